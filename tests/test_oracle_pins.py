@@ -1,0 +1,418 @@
+"""Pins for the CPU oracle: every function is checked against something other than
+itself -- a library routine, a closed form, an invariant, brute force, or a value the
+paper prints (tests/golden/)."""
+import math
+import os
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spts_oracle as O
+from paper_2601_13155_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+SH = replace(synth.TINY, hidden=64, n_q_heads=4, n_kv_heads=2, head_dim=16, ffn_dim=96,
+             ltp_dlow=32, ltp_rank=8)
+
+
+def _layer(shape=SH, seed=7, std=0.2):
+    return synth.layer_weights(shape, seed, 0, std=std)
+
+
+def _x(n, shape=SH, seed=3, heavy=4):
+    X, _ = synth.hidden_states(shape, n, seed, heavy=heavy)
+    return X.astype(np.float64)
+
+
+# ------------------------------------------------------------------ rounding
+def test_round_bf16_matches_torch():
+    rng = np.random.default_rng(0)
+    a = (rng.standard_normal(20000) * np.exp(rng.uniform(-20, 20, 20000))).astype(np.float32)
+    # exact halfway cases between two bf16 values
+    base = synth.bf16_bits_to_f32(rng.integers(0x3000, 0x4800, 4000).astype(np.uint16))
+    half = (base.view(np.uint32) | np.uint32(0x8000)).view(np.float32)
+    a = np.concatenate([a, half, -half])
+    want = torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.round_bf16(a.astype(np.float64))
+    assert np.array_equal(got, want)
+    # and the generator's own rounding agrees with torch too
+    assert np.array_equal(synth.quantize(a, "bf16").astype(np.float64), want)
+
+
+# ------------------------------------------------------------------ rmsnorm / rope / silu
+def test_rmsnorm_matches_torch():
+    x = _x(33)
+    g = np.random.default_rng(1).uniform(0.5, 1.5, x.shape[1])
+    want = torch.nn.functional.rms_norm(torch.from_numpy(x), (x.shape[1],), torch.from_numpy(g), 1e-5)
+    assert np.allclose(O.rmsnorm(x, g, 1e-5), want.numpy(), rtol=1e-12, atol=1e-12)
+
+
+def test_silu_matches_torch():
+    x = np.linspace(-30, 30, 1001)
+    assert np.allclose(O.silu(x), torch.nn.functional.silu(torch.from_numpy(x)).numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_rope_is_complex_rotation_and_relative():
+    rng = np.random.default_rng(2)
+    d, theta = 16, 500000.0
+    x = rng.standard_normal((5, 3, d))
+    pos = np.array([0, 1, 7, 1000, 131071])
+    y = O.rope(x, pos, theta)
+    # independent route: pairs (i, i+d/2) as complex numbers times exp(i*pos*theta^(-2i/d))
+    z = x[..., : d // 2] + 1j * x[..., d // 2:]
+    w = np.exp(1j * pos[:, None] * theta ** (-2.0 * np.arange(d // 2) / d))[:, None, :]
+    zz = z * w
+    assert np.allclose(y, np.concatenate([zz.real, zz.imag], -1), atol=1e-9)
+    assert np.array_equal(y[0], x[0])                       # position 0 is the identity
+    assert np.allclose(np.linalg.norm(y, axis=-1), np.linalg.norm(x, axis=-1))
+    # inner products depend on the position difference only
+    q, k = rng.standard_normal((1, 1, d)), rng.standard_normal((1, 1, d))
+    a = (O.rope(q, [10], theta) * O.rope(k, [3], theta)).sum()
+    b = (O.rope(q, [1010], theta) * O.rope(k, [1003], theta)).sum()
+    assert abs(a - b) < 1e-9
+
+
+def test_rope_matches_hf_llama():
+    tf = pytest.importorskip("transformers")
+    from transformers.models.llama.modeling_llama import apply_rotary_pos_emb, LlamaRotaryEmbedding
+    cfg = _hf_config(SH)
+    rot = LlamaRotaryEmbedding(cfg)
+    rng = np.random.default_rng(4)
+    n = 9
+    q = rng.standard_normal((n, SH.n_q_heads, SH.head_dim))
+    k = rng.standard_normal((n, SH.n_kv_heads, SH.head_dim))
+    pos = np.array([0, 1, 2, 5, 9, 100, 101, 4000, 32767])
+    tq = torch.from_numpy(q).permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).permute(1, 0, 2)[None]
+    cos, sin = rot(tq, torch.from_numpy(pos)[None])
+    cos, sin = cos.double(), sin.double()
+    hq, hk = apply_rotary_pos_emb(tq, tk, cos, sin)
+    # the library evaluates the angles in float32: tight at small positions, looser at large ones
+    gq, gk = O.rope(q, pos, SH.rope_theta), O.rope(k, pos, SH.rope_theta)
+    wq, wk = hq[0].permute(1, 0, 2).numpy(), hk[0].permute(1, 0, 2).numpy()
+    assert np.allclose(gq[:7], wq[:7], atol=2e-5) and np.allclose(gk[:7], wk[:7], atol=2e-5)
+    assert np.allclose(gq, wq, atol=5e-3) and np.allclose(gk, wk, atol=5e-3)
+
+
+# ------------------------------------------------------------------ TopK (P1)
+def _brute_topk(s, k, force_last):
+    n = len(s)
+
+    def key(i):
+        v = s[i]
+        if v != v:
+            v = -math.inf
+        if force_last and i == n - 1:
+            return (0, 0.0, i)
+        return (1, -(v + 0.0), i)
+    return sorted(sorted(range(n), key=key)[:k])
+
+
+@pytest.mark.parametrize("force_last", [False, True])
+def test_topk_bruteforce(force_last):
+    rng = np.random.default_rng(5)
+    cases = [np.array([1.0]), np.array([2.0, 2.0, 2.0, 2.0]), np.array([0.0, -0.0, 0.0, -0.0, 1.0]),
+             np.array([3.0, 1.0, 3.0, 1.0, 3.0, 1.0]), np.array([np.nan, 1.0, -np.inf, np.nan, 0.5])]
+    for n in (2, 3, 17, 64):
+        cases.append(rng.standard_normal(n))
+        cases.append(rng.integers(0, 4, n).astype(np.float64))      # many ties
+    for s in cases:
+        for k in sorted({1, 2, len(s) // 2, len(s) - 1, len(s)} - {0}):
+            if k > len(s):
+                continue
+            got = O.topk_select(s, k, force_last)
+            assert got.tolist() == _brute_topk(list(s), k, force_last), (s, k)
+            assert np.all(np.diff(got) > 0)
+
+
+def test_topk_tie_lowest_index_and_full():
+    s = np.array([1.0, 5.0, 5.0, 5.0, 0.0])
+    assert O.topk_select(s, 2).tolist() == [1, 2]
+    assert O.topk_select(s, 5).tolist() == [0, 1, 2, 3, 4]
+    assert O.topk_select(s, 2, force_last=True).tolist() == [1, 4]
+
+
+# ------------------------------------------------------------------ PAP (P3)
+def _dense_causal_probs_torch(A, pos, W, shape):
+    """Independent route: full causal attention probabilities through torch ops."""
+    N = A.shape[0]
+    H, Hkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    Q = O.rope((A @ W["wq"].T.astype(np.float64)).reshape(N, H, d), pos, shape.rope_theta)
+    K = O.rope((A @ W["wk"].T.astype(np.float64)).reshape(N, Hkv, d), pos, shape.rope_theta)
+    tq = torch.from_numpy(Q).permute(1, 0, 2)
+    tk = torch.from_numpy(K).permute(1, 0, 2).repeat_interleave(H // Hkv, dim=0)
+    z = torch.einsum("hid,hjd->hij", tq, tk) / math.sqrt(d)
+    mask = torch.ones(N, N, dtype=torch.bool).tril()
+    z = z.masked_fill(~mask, float("-inf"))
+    return torch.softmax(z, dim=-1).numpy()
+
+
+def test_pap_score_is_last_row_of_dense_attention():
+    W = _layer()
+    N = 50
+    A = O.rmsnorm(_x(N), np.ones(SH.hidden), SH.rms_eps)
+    pos = np.arange(N) * 3 + 2
+    K, q, S = O.pap_score(A, pos, W["wk"].astype(np.float64), W["wq"].astype(np.float64), SH)
+    P = _dense_causal_probs_torch(A, pos, W, SH)
+    assert np.allclose(S, P[:, N - 1, :].mean(axis=0), rtol=1e-10, atol=1e-14)
+    assert abs(S.sum() - 1.0) < 1e-12
+    assert S.std() > 1e-4           # not degenerate
+
+
+def test_pap_zero_query_is_uniform():
+    W = _layer()
+    N = 23
+    A = O.rmsnorm(_x(N), np.ones(SH.hidden), SH.rms_eps)
+    _, _, S = O.pap_score(A, np.arange(N), W["wk"].astype(np.float64), np.zeros_like(W["wq"], dtype=np.float64), SH)
+    assert np.allclose(S, 1.0 / N, atol=1e-15)
+
+
+# ------------------------------------------------------------------ attention
+def test_attention_matches_torch_sdpa():
+    rng = np.random.default_rng(6)
+    m, H, Hkv, d = 37, 4, 2, 16
+    Q, K, V = rng.standard_normal((m, H, d)), rng.standard_normal((m, Hkv, d)), rng.standard_normal((m, Hkv, d))
+    t = lambda a: torch.from_numpy(a).permute(1, 0, 2)[None]
+    want = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V), is_causal=True, enable_gqa=True)
+    want = want[0].permute(1, 0, 2).reshape(m, H * d).numpy()
+    assert np.allclose(O.causal_gqa_attention(Q, K, V, row_chunk=8), want, atol=1e-12)
+    assert np.allclose(O.causal_gqa_attention(Q, K, V), want, atol=1e-12)
+
+
+# ------------------------------------------------------------------ dense layer vs HF
+def _hf_config(shape):
+    from transformers import LlamaConfig
+    kw = dict(hidden_size=shape.hidden, intermediate_size=shape.ffn_dim,
+              num_attention_heads=shape.n_q_heads, num_key_value_heads=shape.n_kv_heads,
+              head_dim=shape.head_dim, rms_norm_eps=shape.rms_eps, num_hidden_layers=1,
+              vocab_size=32, max_position_embeddings=1 << 17, attention_bias=False, mlp_bias=False)
+    try:
+        cfg = LlamaConfig(rope_theta=shape.rope_theta, **kw)
+    except TypeError:
+        cfg = LlamaConfig(rope_parameters={"rope_type": "default", "rope_theta": shape.rope_theta}, **kw)
+    if getattr(cfg, "rope_parameters", None) is not None and isinstance(cfg.rope_parameters, dict):
+        cfg.rope_parameters["rope_theta"] = shape.rope_theta
+        cfg.rope_parameters.setdefault("rope_type", "default")
+    cfg._attn_implementation = "eager"
+    return cfg
+
+
+def test_dense_layer_matches_hf_llama_decoder_layer():
+    pytest.importorskip("transformers")
+    from transformers.models.llama.modeling_llama import LlamaDecoderLayer, LlamaRotaryEmbedding
+    cfg = _hf_config(SH)
+    W = _layer()
+    rng = np.random.default_rng(8)
+    g1 = rng.uniform(0.5, 1.5, SH.hidden)
+    g2 = rng.uniform(0.5, 1.5, SH.hidden)
+    layer = LlamaDecoderLayer(cfg, 0).double()
+    sd = {"self_attn.q_proj.weight": W["wq"], "self_attn.k_proj.weight": W["wk"],
+          "self_attn.v_proj.weight": W["wv"], "self_attn.o_proj.weight": W["wo"],
+          "mlp.gate_proj.weight": W["w_gate"], "mlp.up_proj.weight": W["w_up"],
+          "mlp.down_proj.weight": W["w_down"], "input_layernorm.weight": g1,
+          "post_attention_layernorm.weight": g2}
+    layer.load_state_dict({k: torch.from_numpy(np.asarray(v, np.float64)) for k, v in sd.items()})
+    N = 29
+    X = _x(N)
+    pos = np.arange(N)
+    tx = torch.from_numpy(X)[None]
+    pid = torch.from_numpy(pos)[None]
+    cos, sin = LlamaRotaryEmbedding(cfg)(tx, pid)
+    mask = torch.zeros(1, 1, N, N, dtype=torch.float64).masked_fill(
+        ~torch.ones(N, N, dtype=torch.bool).tril(), float("-inf"))
+    with torch.no_grad():
+        out = layer(tx, attention_mask=mask, position_ids=pid, position_embeddings=(cos.double(), sin.double()))
+    out = out[0] if isinstance(out, tuple) else out
+    want = out.reshape(N, SH.hidden).numpy()
+    got = O.layer_dense(X, pos, W, SH, g_attn=g1, g_ffn=g2)["X"]
+    assert np.allclose(got, want, atol=5e-5), np.abs(got - want).max()
+
+
+# ------------------------------------------------------------------ Eq. 2 (P2, P6)
+def test_keep_all_equals_dense_and_skipped_rows_untouched():
+    W = _layer()
+    N = 40
+    X = _x(N)
+    pos = np.arange(N)
+    d = O.layer_dense(X, pos, W, SH)
+    s = O.layer_prefill_skip(X, pos, W, SH, N, N)
+    assert np.array_equal(s["X"], d["X"])
+    assert np.array_equal(s["K"], d["K"]) and np.array_equal(s["V"], d["V"])
+    r = O.layer_prefill_skip(X, pos, W, SH, 12, 9)
+    touched = np.union1d(r["idx_attn"], r["idx_ffn"])
+    rest = np.setdiff1d(np.arange(N), touched)
+    assert len(rest) > 0
+    assert np.array_equal(r["X"][rest], X[rest])
+    assert not np.allclose(r["X"][touched], X[touched])
+    assert len(r["idx_attn"]) == 12 and len(r["idx_ffn"]) == 9
+    assert r["idx_attn"][-1] == N - 1 and r["idx_ffn"][-1] == N - 1
+    assert r["K"].shape == (12, SH.n_kv_heads, SH.head_dim)
+    assert np.array_equal(r["cache_pos"], pos[r["idx_attn"]])
+
+
+def test_reduced_attention_is_dense_attention_on_the_subsequence():
+    """Active queries attend to active keys only, causal in token order: the update of the
+    active rows equals a dense attention block run on the gathered rows with their
+    original positions."""
+    W = _layer()
+    N = 36
+    X = _x(N)
+    pos = np.arange(N)
+    Wz = dict(W)
+    Wz["w_down"] = np.zeros_like(W["w_down"])        # FFN contributes nothing
+    r = O.layer_prefill_skip(X, pos, Wz, SH, 14, 5)
+    T = r["idx_attn"]
+    d = O.layer_dense(X[T], pos[T], Wz, SH)
+    assert np.allclose(r["X"][T], d["X"], atol=1e-12)
+    # scores: S_ffn = C * S_mha with S_mha from before the update, C from the updated residual
+    B = O.rmsnorm(r["X"], np.ones(SH.hidden), SH.rms_eps)
+    o = O.ltp_proxy(B, {k: np.asarray(v, np.float64) for k, v in W.items()})
+    assert np.allclose(r["C"], np.linalg.norm(o, axis=1), rtol=1e-12)
+    A = O.rmsnorm(X, np.ones(SH.hidden), SH.rms_eps)
+    _, _, S0 = O.pap_score(A, pos, W["wk"].astype(np.float64), W["wq"].astype(np.float64), SH)
+    assert np.array_equal(r["S_mha"], S0)
+    assert np.allclose(r["S_ffn"], r["C"] * S0, rtol=1e-15)
+
+
+# ------------------------------------------------------------------ LTP (P4, P5)
+def test_full_rank_proxy_reproduces_ffn():
+    W = _layer()
+    D, Dff = SH.hidden, SH.ffn_dim
+    Wp = {k: np.asarray(v, np.float64) for k, v in W.items()}
+    r = min(D, Dff)
+    for name, u, v in (("w_gate", "ug", "vg"), ("w_up", "uu", "vu")):
+        Wm = Wp[name].T                                   # paper orientation [D, Dff]
+        U, s, Vt = np.linalg.svd(Wm, full_matrices=False)
+        Wp[u] = U[:, :r].T.copy()                         # stored [r, D]
+        Wp[v] = (s[:r, None] * Vt[:r]).T.copy()           # stored [Dlow, r]
+    U, s, Vt = np.linalg.svd(Wp["w_down"], full_matrices=False)     # W_down [D, Dff]
+    Wp["ud"] = U[:, :r].copy()                            # [D, r]
+    Wp["vd"] = (s[:r, None] * Vt[:r]).copy()              # [r, Dlow]
+    B = O.rmsnorm(_x(19), np.ones(D), SH.rms_eps)
+    exact = O.ffn(B, Wp["w_gate"], Wp["w_up"], Wp["w_down"])
+    assert np.allclose(O.ltp_proxy(B, Wp), exact, atol=1e-10)
+    C, S = O.ltp_score(B, np.full(19, 0.5), Wp)
+    assert np.allclose(C, np.linalg.norm(exact, axis=1), rtol=1e-9)
+    assert np.allclose(S, 0.5 * C)
+    # the FFN itself against torch
+    t = torch.from_numpy
+    want = (torch.nn.functional.silu(t(B) @ t(Wp["w_gate"]).T) * (t(B) @ t(Wp["w_up"]).T)) @ t(Wp["w_down"]).T
+    assert np.allclose(exact, want.numpy(), atol=1e-12)
+
+
+def test_proxy_cost_matches_table6():
+    rows = [l.split() for l in open(os.path.join(GOLD, "paper_table6_proxy_cost.txt")) if l[0] != "#"]
+    assert len(rows) == 7
+    for dl, r, printed, ok in rows:
+        D = 4096
+        dlow = None if dl == "/" else int(dl)
+        rank = None if r == "/" else int(r)
+        if dlow is None:
+            continue                     # the undecomposed-D_low row needs D_ff; printed value is inconsistent
+        macs = O.proxy_macs_per_projection(D, dlow, rank)
+        if ok == "1":
+            assert round(macs / 1000) == int(printed) or macs // 1000 == int(printed), (dl, r, macs)
+        else:
+            assert macs == 192 * (4096 + 512) == 884736     # printed 855K: digits swapped
+
+
+# ------------------------------------------------------------------ MSDP (P7, P8)
+def test_schedule_reproduces_table3():
+    rows = [l.split() for l in open(os.path.join(GOLD, "paper_table3_kv_cache.txt")) if l[0] != "#"]
+    assert len(rows) == 4
+    for n_ki, full, with_pap, saving in rows:
+        n = int(n_ki) * 1024
+        plan = O.paper_llama_schedule(n)
+        units = O.kv_cache_token_layers(plan) / 1024 / 64.0      # the paper's unit: 32 layers * N Ki / 64
+        full_units = 32 * int(n_ki) / 64.0
+        assert f"{full_units:.2f}" == full
+        # the paper rounds half up (4.125 -> 4.13)
+        assert f"{math.floor(units * 100 + 0.5) / 100:.2f}" == with_pap, (n_ki, units)
+        assert f"{(1 - units / full_units) * 100:.1f}" == saving
+
+
+def test_schedule_budget_rule():
+    plan = O.msdp_schedule(8, 1000, (0, 4), (1000, 600), 700, 400)
+    assert [p["N"] for p in plan] == [1000] * 4 + [600] * 4
+    assert [p["m_attn"] for p in plan] == [700] * 4 + [600] * 4       # M = min(|T|, M_fixed)
+    assert [p["m_ffn"] for p in plan] == [400] * 8
+    assert [p["prune_to"] for p in plan] == [None, None, None, 600, None, None, None, None]
+    w = synth.workload("cfg3")
+    plan = O.msdp_schedule(32, w.n_tokens, w.stage_first_layer, w.stage_tokens,
+                           math.ceil(w.keep_attn * w.n_tokens), math.ceil(w.keep_ffn * w.n_tokens))
+    assert [plan[l]["N"] for l in (0, 8, 16, 24)] == [32768, 24576, 16384, 11469]
+    assert [plan[l]["m_attn"] for l in (0, 8, 16, 24)] == [16384, 16384, 16384, 11469]
+    assert [plan[l]["m_ffn"] for l in (0, 8, 16, 24)] == [13108, 13108, 13108, 11469]
+    assert [l for l in range(32) if plan[l]["prune_to"]] == [7, 15, 23]
+
+
+def test_compaction_preserves_order_and_rows():
+    rng = np.random.default_rng(9)
+    N = 31
+    X = rng.standard_normal((N, 8))
+    pos = np.cumsum(rng.integers(1, 4, N))
+    orig = np.arange(N) + 100
+    S = rng.random(N)
+    Xo, po, oo, T = O.msdp_compact(X, pos, orig, S, 11)
+    assert len(T) == 11 and T[-1] == N - 1
+    assert np.array_equal(Xo, X[T]) and np.array_equal(po, pos[T]) and np.array_equal(oo, orig[T])
+    assert np.all(np.diff(po) > 0)
+    assert set(T.tolist()) == set(_brute_topk(list(S), 11, True))
+    Xi, pi, oi, Ti = O.msdp_compact(X, pos, orig, S, N + 5)
+    assert np.array_equal(Xi, X) and np.array_equal(Ti, np.arange(N))
+
+
+# ------------------------------------------------------------------ Algorithm 1 as a whole, decode (P9)
+def test_model_prefill_follows_plan_and_prunes_with_last_layer_score():
+    sh = replace(SH, n_layers=4)
+    layers = [synth.layer_weights(sh, 11, l, std=0.2) for l in range(4)]
+    N = 48
+    X = _x(N, sh)
+    plan = O.msdp_schedule(4, N, (0, 2), (N, 30), 20, 16)
+    r = O.model_prefill(X, layers, sh, plan)
+    assert r["X"].shape[0] == 30
+    assert [len(c["pos"]) for c in r["caches"]] == [20, 20, 20, 20]
+    T = r["trace"][1]["idx_prune"]
+    assert np.array_equal(T, O.topk_select(r["trace"][1]["S_mha"], 30, True))
+    assert np.array_equal(r["orig"], T)
+    assert np.array_equal(r["caches"][2]["pos"], r["orig"][r["trace"][2]["idx_attn"]])
+    # with every budget = N and no pruning it is a stack of dense layers
+    plan_d = O.msdp_schedule(4, N, (0,), (N,), N, N)
+    rd = O.model_prefill(X, layers, sh, plan_d)
+    Y = X
+    for l in range(4):
+        Y = O.layer_dense(Y, np.arange(N), layers[l], sh)["X"]
+    assert np.array_equal(rd["X"], Y)
+
+
+def test_decode_step_equals_dense_prefill_of_one_more_token():
+    sh = replace(SH, n_layers=3, vocab=40)
+    layers = [synth.layer_weights(sh, 12, l, std=0.2) for l in range(3)]
+    hw = synth.head_weights(sh, 12)
+    N = 21
+    X = _x(N + 1, sh)
+    plan = O.msdp_schedule(3, N, (0,), (N,), N, N)
+    r = O.model_prefill(X[:N], layers, sh, plan)
+    x, logits, tok = O.decode_step(X[N], N, layers, sh, r["caches"], np.ones(sh.hidden), hw["lm_head"])
+    plan1 = O.msdp_schedule(3, N + 1, (0,), (N + 1,), N + 1, N + 1)
+    full = O.model_prefill(X, layers, sh, plan1)
+    assert np.allclose(x, full["X"][N], atol=1e-10)
+    assert all(len(c["pos"]) == N + 1 for c in r["caches"])
+    l2, t2 = O.first_token(full["X"][N], np.ones(sh.hidden), hw["lm_head"], sh.rms_eps)
+    assert tok == t2 == int(torch.argmax(torch.from_numpy(l2)))
+    assert np.allclose(logits, l2, atol=1e-9)
+
+
+def test_bf16_mode_rounds_only_at_storage_points():
+    W = synth.layer_weights(replace(SH, dtype="bf16"), 7, 0, std=0.2)
+    N = 24
+    X = synth.quantize(_x(N).astype(np.float32), "bf16").astype(np.float64)
+    r = O.layer_prefill_skip(X, np.arange(N), W, SH, 10, 8, mode="bf16")
+    for k in ("X", "K", "V"):
+        assert np.array_equal(O.round_bf16(r[k]), r[k])
+    e = O.layer_prefill_skip(X, np.arange(N), W, SH, 10, 8, mode="exact")
+    rel = np.abs(r["X"] - e["X"]).max() / np.sqrt(np.mean(e["X"] ** 2))
+    assert 0 < rel < 0.1
+    assert np.array_equal(r["S_mha"], e["S_mha"])     # PAP scores come from unrounded K
