@@ -1,0 +1,218 @@
+/*
+ * spts.h -- C boundary of the SPTS (Self-Predictive Token Skipping) prefill library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library runs the token-selective transformer prefill layer of the SPTS paper:
+ * Partial Attention Probing (Section 3.2, Eq. 4-5), Low-rank Transformation Probing
+ * (Section 3.3, Eq. 12-15), top-k selection, the reduced attention / FFN blocks with
+ * residual scatter (Eq. 2, Algorithm 1), Multi-Stage Delayed Pruning (Section 3.4, Eq. 16)
+ * and the decode step over the per-layer compressed KV cache.
+ *
+ * General rules
+ *   - Every pointer named in a signature is a DEVICE pointer unless the comment says "host".
+ *     Structs (model_desc, layer_weights, kv_layer, layer_plan) live in HOST memory and hold
+ *     device pointers.
+ *   - The caller owns every buffer, including the workspace given to spts_create().  The
+ *     library allocates no device memory and frees nothing.
+ *   - All work is enqueued on the context's CUDA stream and returns without synchronising.
+ *     Sizes (N, k, m_attn, m_ffn, n_next) are host integers: Algorithm 1 fixes them from the
+ *     schedule (M^l = min(|T^l|, M_fixed), Section 3.4), so no call reads a count back.
+ *   - Storage type: dtype SPTS_BF16 (bf16 in HBM, fp32 accumulation, tensor-core kernels) or
+ *     SPTS_FP32 (verification mode: fp32 storage and CUDA-core fp32 arithmetic).  Scores,
+ *     softmax statistics and norms are fp32 in both modes.
+ *   - Weight matrices are row-major [out_features, in_features].  RMSNorm gains are expected
+ *     to be folded into the columns of the matrices that consume the normalised rows
+ *     (spts_fold_norm_gain()); with unit gains nothing needs to be done.
+ *   - Index lists are int32, strictly ascending.  Ties in a top-k go to the lower index.
+ *   - Errors detectable on the host (null pointer, k > N, unsupported shape, workspace too
+ *     small, misalignment) are returned before anything is launched.  Device-side problems
+ *     (a bounded wait that expired, a non-finite score) set a status word that
+ *     spts_last_device_status() returns after synchronising the stream; kernels never trap.
+ *   - Pointers must be 16-byte aligned; rows of X, K, V are contiguous.
+ */
+#ifndef SPTS_H_
+#define SPTS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SPTS_OK = 0,
+  SPTS_ERR_INVALID_ARG = 1,
+  SPTS_ERR_SHAPE = 2,
+  SPTS_ERR_WORKSPACE = 3,
+  SPTS_ERR_CUDA = 4,
+  SPTS_ERR_TIMEOUT = 5,
+  SPTS_ERR_NONFINITE = 6,
+  SPTS_ERR_UNSUPPORTED = 7
+} spts_status;
+
+enum { SPTS_BF16 = 0, SPTS_FP32 = 1 };
+
+/* flags */
+enum {
+  SPTS_FORCE_LAST = 1u,   /* the last candidate is always selected (it carries the output state) */
+  SPTS_REFERENCE_KERNELS = 2u /* spts_set_option: run the plain CUDA-core kernels also in bf16 mode */
+};
+
+typedef struct {
+  int32_t hidden;      /* D */
+  int32_t n_q_heads;   /* H */
+  int32_t n_kv_heads;  /* Hkv, divides H */
+  int32_t head_dim;    /* d */
+  int32_t ffn_dim;     /* Dff */
+  int32_t ltp_dlow;    /* D_low of the proxy FFN (Eq. 12) */
+  int32_t ltp_rank;    /* r of the proxy FFN */
+  int32_t n_layers;
+  int32_t vocab;
+  float rms_eps;
+  float rope_theta;
+  int32_t dtype;       /* SPTS_BF16 or SPTS_FP32 */
+} spts_model_desc;
+
+/* Device pointers, each [out, in] row-major in the model's storage type. */
+typedef struct {
+  const void* wq;      /* [H*d, D]   */
+  const void* wk;      /* [Hkv*d, D] */
+  const void* wv;      /* [Hkv*d, D] */
+  const void* wo;      /* [D, H*d]   */
+  const void* w_gate;  /* [Dff, D]   */
+  const void* w_up;    /* [Dff, D]   */
+  const void* w_down;  /* [D, Dff]   */
+  const void* ug;      /* [r, D]      U_gate^T  */
+  const void* vg;      /* [Dlow, r]   V_gate^T  */
+  const void* uu;      /* [r, D]      U_up^T    */
+  const void* vu;      /* [Dlow, r]   V_up^T    */
+  const void* vd;      /* [r, Dlow]   V_down    */
+  const void* ud;      /* [D, r]      U_down    */
+} spts_layer_weights;
+
+/* One layer's KV cache: k, v are [capacity, Hkv, d] in the storage type (K after RoPE),
+ * pos [capacity] holds the original position of every cached token.  `len` is host state. */
+typedef struct {
+  void* k;
+  void* v;
+  int32_t* pos;
+  int32_t len;
+  int32_t capacity;
+} spts_kv_layer;
+
+/* Per-layer entry of the MSDP schedule (Section 3.4): active budgets already clipped to the
+ * candidate count, and the candidate count to prune to after this layer (0 = not a stage end). */
+typedef struct {
+  int32_t m_attn;
+  int32_t m_ffn;
+  int32_t prune_to;
+} spts_layer_plan;
+
+typedef struct {
+  const spts_layer_weights* layers; /* host array [n_layers] */
+  const void* lm_head;              /* [vocab, D] */
+  const void* embed;                /* [vocab, D], used by spts_decode_step */
+} spts_model_weights;
+
+typedef struct spts_ctx spts_ctx;
+
+/* Bytes of device workspace spts_create() needs for sequences of up to max_seq candidates. */
+size_t spts_workspace_bytes(const spts_model_desc* desc, int max_seq);
+
+/* Creates a context.  `workspace` is caller-owned device memory of at least
+ * spts_workspace_bytes() bytes, 256-byte aligned; `cuda_stream` is a cudaStream_t (may be 0).
+ * Must be called with the target device current.  Returns SPTS_ERR_SHAPE for shapes the
+ * kernels do not cover (head_dim must be 64 or 128, H a multiple of Hkv, dimensions
+ * multiples of 8; bf16 tensor-core mode additionally needs head_dim 128 and hidden, ffn_dim,
+ * ltp_dlow multiples of 64, ltp_rank a multiple of 16). */
+spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream, spts_ctx** out);
+void spts_destroy(spts_ctx* ctx);
+
+/* Sets SPTS_REFERENCE_KERNELS on/off (value 0/1). */
+spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value);
+
+/* Synchronises the context's stream and returns the device status word (then clears it). */
+spts_status spts_last_device_status(spts_ctx* ctx);
+
+/* Number of kernels the library has launched on this context so far. */
+int64_t spts_launch_count(const spts_ctx* ctx);
+
+/* W[o, i] *= g[i], in place, rounded to the storage type: folds an RMSNorm gain g [in] into a
+ * weight matrix [out, in] that consumes the normalised rows (pre-norm block placement; the
+ * paper's Algorithm 1 leaves normalisation out). */
+spts_status spts_fold_norm_gain(spts_ctx* ctx, void* W, const float* g, int out_features,
+                                int in_features);
+
+/* Partial Attention Probing, Eq. 4 / Algorithm 1 "K <- X W_K, q <- X_N W_Q; S_MHA":
+ * K_out[n] = RoPE(rmsnorm(X[n]) W_K, pos[n]) for all N candidates (storage type, [N,Hkv,d]),
+ * q = RoPE(rmsnorm(X[N-1]) W_Q, pos[N-1]),
+ * S_mha_out[n] = (1/H) sum_h softmax_n(q_h . K_{h / (H/Hkv)} / sqrt(d))[n]   (fp32, [N]).
+ * The logits are taken from the unrounded fp32 keys.  K_out may be NULL (workspace is used). */
+spts_status spts_pap_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X,
+                           const int32_t* pos, int N, void* K_out, float* S_mha_out);
+
+/* Low-rank Transformation Probing, Eq. 12-14: C[n] = || f(rmsnorm(X[n])) ||_2 with
+ * f(x) = (silu(x Ug Vg) * (x Uu Vu)) Vd^T Ud^T, and S_ffn[n] = C[n] * S_mha[n].
+ * C_out may be NULL.  X is the residual stream the FFN block would see. */
+spts_status spts_ltp_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X,
+                           const float* S_mha, int N, float* C_out, float* S_ffn_out);
+
+/* TopK of Eq. 5 / 15 / 16: the k largest of scores[0..N), written ascending by index.
+ * Order: score descending, then index ascending; -0.0 equals +0.0; NaN ranks last (and sets
+ * SPTS_ERR_NONFINITE in the device status).  flags: SPTS_FORCE_LAST.  1 <= k <= N. */
+spts_status spts_topk_select(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags,
+                             int32_t* idx_out);
+
+/* One decoder layer of Algorithm 1 in the prefill phase, in place on X [N, D]:
+ *   S_mha (Eq. 4) -> T_a = TopK(S_mha, m_attn) -> Q, V projected for the rows in T_a, K rows
+ *   reused -> cache <- (K^, V^, pos[T_a]) -> causal GQA attention among the active rows ->
+ *   X[T_a] += O W_O (Eq. 2); then C, S_ffn (Eq. 12-14) on the updated X -> T_f =
+ *   TopK(S_ffn, m_ffn) -> X[T_f] += FFN(rmsnorm(X[T_f])) (Eq. 6).  Rows outside T_a and T_f
+ *   are not written.  m_attn == N / m_ffn == N run that block densely without probing.
+ * cache->len is set to m_attn (capacity must be >= m_attn).  S_mha_out [N], idx_attn_out
+ * [m_attn], idx_ffn_out [m_ffn] are optional outputs (NULL to skip; S_mha is still computed
+ * when a selection needs it).  flags: SPTS_FORCE_LAST. */
+spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, void* X,
+                                    const int32_t* pos, int N, int m_attn, int m_ffn,
+                                    uint32_t flags, spts_kv_layer* cache, float* S_mha_out,
+                                    int32_t* idx_attn_out, int32_t* idx_ffn_out);
+
+/* Stage-end pruning, Eq. 16 / Algorithm 1 "X <- X[T^{l+1}, :]": keeps the
+ * n_next = min(N, N_{s+1}) candidates with the largest S_mha, in token order.  Out of place:
+ * X_out [n_next, D], pos_out, orig_out [n_next] must not alias the inputs; idx_out [n_next]
+ * (optional) receives the kept candidate indices.  flags: SPTS_FORCE_LAST. */
+spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* pos_in,
+                              const int32_t* orig_in, const float* S_mha, int N, int n_next,
+                              uint32_t flags, void* X_out, int32_t* pos_out, int32_t* orig_out,
+                              int32_t* idx_out);
+
+/* End of prefill (the output of Algorithm 1 feeds next-token prediction): RMSNorm of one
+ * hidden row x [D], logits = lm_head x (fp32 [vocab], optional), token = argmax (lowest index). */
+spts_status spts_first_token(spts_ctx* ctx, const void* x_row, const void* lm_head,
+                             float* logits_out, int32_t* token_out);
+
+/* Whole prefill (Algorithm 1, prefill phase) over n_layers layers following `plan` (host
+ * array [n_layers]).  X [N, D] is updated in place; at every stage end the survivors are
+ * compacted into X_alt and the two buffers swap roles, likewise pos/orig with pos_alt/orig_alt
+ * (each sized for N entries).  *n_final (host) receives the final candidate count and
+ * *final_in_alt (host) tells which buffer holds the result.  token_out (device, optional)
+ * receives the first generated token. */
+spts_status spts_prefill(spts_ctx* ctx, const spts_model_weights* mw, const spts_layer_plan* plan,
+                         void* X, int32_t* pos, int32_t* orig, void* X_alt, int32_t* pos_alt,
+                         int32_t* orig_alt, int N, uint32_t flags, spts_kv_layer* caches,
+                         int32_t* n_final, int32_t* final_in_alt, int32_t* token_out);
+
+/* One decode step (Algorithm 1 outside the prefill phase: no skipping).  The new token's
+ * embedding row is x_in [D] (if NULL, row token_in of mw->embed is used); it runs every layer
+ * densely against that layer's cache plus itself at position `pos`, appends its K/V to every
+ * cache (len += 1; capacity must allow it), then the first-token head.  x_out [D] optional. */
+spts_status spts_decode_step(spts_ctx* ctx, const spts_model_weights* mw, spts_kv_layer* caches,
+                             const void* x_in, int32_t token_in, int32_t pos, void* x_out,
+                             float* logits_out, int32_t* token_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPTS_H_ */

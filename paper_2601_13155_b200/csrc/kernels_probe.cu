@@ -1,0 +1,334 @@
+// Memory-bound pieces of the probes: row RMS statistics, the last-token query (Algorithm 1,
+// "q <- X_N W_Q"), the head-mean softmax of Eq. 4, the score fusion of Eq. 13-14, the rotary
+// table, the RMSNorm-gain fold and the first-token head.  fp32 arithmetic throughout.
+#include "spts_common.cuh"
+
+namespace spts {
+
+namespace {
+
+template <typename T> struct Vec16;
+template <> struct Vec16<float> { static constexpr int N = 4; };
+template <> struct Vec16<bf16> { static constexpr int N = 8; };
+
+template <typename T>
+__device__ __forceinline__ void load16(const T* p, float* out);
+template <>
+__device__ __forceinline__ void load16<float>(const float* p, float* out) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <>
+__device__ __forceinline__ void load16<bf16>(const bf16* p, float* out) {
+  uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+// rstd[n] = 1 / sqrt(mean(x_n^2) + eps); one warp per row.
+template <typename T>
+__global__ void rstd_kernel(const T* __restrict__ X, int N, int D, float eps, float* __restrict__ rstd) {
+  constexpr int V = Vec16<T>::N;
+  int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= N) return;
+  int lane = threadIdx.x & 31;
+  const T* x = X + (size_t)row * D;
+  float s = 0.f;
+  for (int c = lane * V; c < D; c += 32 * V) {
+    float v[V];
+    load16<T>(x + c, v);
+#pragma unroll
+    for (int i = 0; i < V; ++i) s = fmaf(v[i], v[i], s);
+  }
+  s = warp_sum(s);
+  if (lane == 0) rstd[row] = 1.0f / sqrtf(s / (float)D + eps);
+}
+
+// cos/sin table for rotary embedding: cs[n, i] = (cos, sin)(pos[n] * theta^(-2i/d)), angles in fp64.
+__global__ void rope_table_kernel(const int32_t* __restrict__ pos, int N, int half, double theta,
+                                  float2* __restrict__ cs) {
+  size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (size_t)N * half) return;
+  int n = (int)(t / half), i = (int)(t - (size_t)n * half);
+  double inv = exp2(-(double)(2 * i) / (double)(2 * half) * log2(theta));
+  double a = (double)pos[n] * inv;
+  double s, c;
+  sincos(a, &s, &c);
+  cs[t] = make_float2((float)c, (float)s);
+}
+
+// q[h, :] = RoPE(rstd * x_last . Wq[h*d + :, :]); one warp per rotary pair (j, j + d/2).
+template <typename T>
+__global__ void q_last_kernel(const T* __restrict__ x, const T* __restrict__ wq, int D, int d, int HD,
+                              float rs_scale_dummy, const float* __restrict__ rstd_last,
+                              const float2* __restrict__ cs_last, float* __restrict__ q) {
+  constexpr int V = Vec16<T>::N;
+  int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  int half = d >> 1;
+  if (pair >= HD / 2) return;
+  int lane = threadIdx.x & 31;
+  int h = pair / half, i = pair - h * half;
+  const T* w1 = wq + (size_t)(h * d + i) * D;
+  const T* w2 = wq + (size_t)(h * d + i + half) * D;
+  float a1 = 0.f, a2 = 0.f;
+  for (int c = lane * V; c < D; c += 32 * V) {
+    float xv[V], u[V], v[V];
+    load16<T>(x + c, xv);
+    load16<T>(w1 + c, u);
+    load16<T>(w2 + c, v);
+#pragma unroll
+    for (int e = 0; e < V; ++e) { a1 = fmaf(xv[e], u[e], a1); a2 = fmaf(xv[e], v[e], a2); }
+  }
+  a1 = warp_sum(a1);
+  a2 = warp_sum(a2);
+  if (lane == 0) {
+    float rs = *rstd_last;
+    a1 *= rs; a2 *= rs;
+    float2 c = cs_last[i];
+    q[h * d + i] = a1 * c.x - a2 * c.y;
+    q[h * d + i + half] = a2 * c.x + a1 * c.y;
+  }
+}
+
+// per-head max and sum of exp over the N logits of one head
+__global__ void __launch_bounds__(1024)
+pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N, float* __restrict__ stats) {
+  __shared__ float red[32];
+  __shared__ float bcast;
+  const float* l = logits + (size_t)blockIdx.x * ld;
+  int tid = threadIdx.x;
+  float m = -INFINITY;
+  for (int n = tid; n < N; n += blockDim.x) m = fmaxf(m, l[n]);
+  m = warp_max(m);
+  if ((tid & 31) == 0) red[tid >> 5] = m;
+  __syncthreads();
+  if (tid < 32) {
+    float v = tid < (blockDim.x >> 5) ? red[tid] : -INFINITY;
+    v = warp_max(v);
+    if (tid == 0) bcast = v;
+  }
+  __syncthreads();
+  m = bcast;
+  float s = 0.f;
+  for (int n = tid; n < N; n += blockDim.x) s += expf(l[n] - m);
+  s = warp_sum(s);
+  __syncthreads();
+  if ((tid & 31) == 0) red[tid >> 5] = s;
+  __syncthreads();
+  if (tid < 32) {
+    float v = tid < (blockDim.x >> 5) ? red[tid] : 0.f;
+    v = warp_sum(v);
+    if (tid == 0) { stats[2 * blockIdx.x] = m; stats[2 * blockIdx.x + 1] = v; }
+  }
+}
+
+// S[n] = (1/H) sum_h exp(l[h, n] - max_h) / sum_h      (Eq. 4)
+__global__ void pap_mean_kernel(const float* __restrict__ logits, int ld, int N, int H,
+                                const float* __restrict__ stats, float* __restrict__ S) {
+  int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float acc = 0.f;
+  for (int h = 0; h < H; ++h) acc += expf(logits[(size_t)h * ld + n] - stats[2 * h]) / stats[2 * h + 1];
+  S[n] = acc / (float)H;
+}
+
+// C[n] = sqrt(sum_p csq[n, p]);  S_ffn[n] = C[n] * S_mha[n]      (Eq. 13-14)
+__global__ void ffn_score_kernel(const float* __restrict__ csq, int parts, const float* __restrict__ S_mha,
+                                 int N, float* __restrict__ C_out, float* __restrict__ S_ffn) {
+  int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  float s = 0.f;
+  for (int p = 0; p < parts; ++p) s += csq[(size_t)n * parts + p];
+  float c = sqrtf(s);
+  if (C_out) C_out[n] = c;
+  S_ffn[n] = c * S_mha[n];
+}
+
+template <typename T>
+__global__ void fold_gain_kernel(T* W, const float* __restrict__ g, size_t total, int in_f) {
+  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (size_t)gridDim.x * blockDim.x)
+    W[t] = from_f32<T>(to_f32(W[t]) * g[t % in_f]);
+}
+
+// out[0] = [vg | 0], out[1] = [0 | vu], each [Dlow, 2r]: lets one dual-weight GEMM evaluate
+// silu(t_g Vg) * (t_u Vu) of Eq. 12 from the concatenated low-rank activations [t_g | t_u].
+template <typename T>
+__global__ void pad_proxy_kernel(const T* __restrict__ vg, const T* __restrict__ vu, int dlow, int r,
+                                 T* __restrict__ out) {
+  int t = blockIdx.x * blockDim.x + threadIdx.x;
+  int total = dlow * 2 * r;
+  if (t >= total) return;
+  int row = t / (2 * r), c = t - row * 2 * r;
+  T zero = from_f32<T>(0.f);
+  out[t] = c < r ? vg[row * r + c] : zero;
+  out[total + t] = c < r ? zero : vu[row * r + (c - r)];
+}
+
+// logits[v] = rstd(x) * x . lm_head[v, :]; one warp per vocabulary row
+template <typename T>
+__global__ void head_logits_kernel(const T* __restrict__ x, const T* __restrict__ lm, int D, int V_,
+                                   float eps, float* __restrict__ logits) {
+  constexpr int V = Vec16<T>::N;
+  extern __shared__ float xs[];
+  __shared__ float red[32];
+  __shared__ float rs_sh;
+  int tid = threadIdx.x;
+  float ss = 0.f;
+  for (int c = tid; c < D; c += blockDim.x) { float v = to_f32(x[c]); xs[c] = v; ss = fmaf(v, v, ss); }
+  ss = warp_sum(ss);
+  if ((tid & 31) == 0) red[tid >> 5] = ss;
+  __syncthreads();
+  if (tid < 32) {
+    float v = tid < (blockDim.x >> 5) ? red[tid] : 0.f;
+    v = warp_sum(v);
+    if (tid == 0) rs_sh = 1.0f / sqrtf(v / (float)D + eps);
+  }
+  __syncthreads();
+  int row = blockIdx.x * (blockDim.x >> 5) + (tid >> 5);
+  if (row >= V_) return;
+  int lane = tid & 31;
+  const T* w = lm + (size_t)row * D;
+  float a = 0.f;
+  for (int c = lane * V; c < D; c += 32 * V) {
+    float u[V];
+    load16<T>(w + c, u);
+#pragma unroll
+    for (int e = 0; e < V; ++e) a = fmaf(xs[c + e], u[e], a);
+  }
+  a = warp_sum(a);
+  if (lane == 0) logits[row] = a * rs_sh;
+}
+
+// argmax with the lowest index on ties (single block)
+__global__ void __launch_bounds__(1024)
+argmax_kernel(const float* __restrict__ logits, int n, int32_t* __restrict__ out) {
+  __shared__ float bv[32];
+  __shared__ int bi[32];
+  int tid = threadIdx.x;
+  float best = -INFINITY;
+  int besti = 0x7FFFFFFF;
+  for (int i = tid; i < n; i += blockDim.x) {
+    float v = logits[i];
+    if (v > best || (v == best && i < besti)) { best = v; besti = i; }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+    if (ov > best || (ov == best && oi < besti)) { best = ov; besti = oi; }
+  }
+  if ((tid & 31) == 0) { bv[tid >> 5] = best; bi[tid >> 5] = besti; }
+  __syncthreads();
+  if (tid < 32) {
+    best = tid < (blockDim.x >> 5) ? bv[tid] : -INFINITY;
+    besti = tid < (blockDim.x >> 5) ? bi[tid] : 0x7FFFFFFF;
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+      if (ov > best || (ov == best && oi < besti)) { best = ov; besti = oi; }
+    }
+    if (tid == 0) *out = besti == 0x7FFFFFFF ? 0 : besti;
+  }
+}
+
+}  // namespace
+
+spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd) {
+  const int D = ctx->desc.hidden;
+  const int wpb = 8;
+  if (ctx->desc.dtype == SPTS_BF16)
+    rstd_kernel<bf16><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const bf16*)X, N, D, ctx->desc.rms_eps, rstd);
+  else
+    rstd_kernel<float><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const float*)X, N, D, ctx->desc.rms_eps, rstd);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_rope_table(spts_ctx* ctx, const int32_t* pos, int N, float2* cs) {
+  const int half = ctx->desc.head_dim / 2;
+  size_t total = (size_t)N * half;
+  rope_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, ctx->stream>>>(pos, N, half,
+                                                                             (double)ctx->desc.rope_theta, cs);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N, const void* wq,
+                          const float* rstd, float* q) {
+  const auto& d = ctx->desc;
+  const int HD = d.n_q_heads * d.head_dim;
+  const int wpb = 8;
+  const int half = d.head_dim / 2;
+  dim3 grid(ceil_div(HD / 2, wpb));
+  if (d.dtype == SPTS_BF16)
+    q_last_kernel<bf16><<<grid, wpb * 32, 0, ctx->stream>>>((const bf16*)X + (size_t)(N - 1) * d.hidden,
+        (const bf16*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q);
+  else
+    q_last_kernel<float><<<grid, wpb * 32, 0, ctx->stream>>>((const float*)X + (size_t)(N - 1) * d.hidden,
+        (const float*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, float* S) {
+  const int H = ctx->desc.n_q_heads;
+  pap_head_stats_kernel<<<H, 1024, 0, ctx->stream>>>(logits, ld_logits, N, ctx->ws.head_stats);
+  SPTS_CUDA_OK(ctx);
+  pap_mean_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(logits, ld_logits, N, H, ctx->ws.head_stats, S);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
+                             float* C_out, float* S_ffn) {
+  ffn_score_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(csq, parts, S_mha, N, C_out, S_ffn);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_fold_gain(spts_ctx* ctx, void* W, const float* g, int out_f, int in_f) {
+  size_t total = (size_t)out_f * in_f;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+  if (ctx->desc.dtype == SPTS_BF16)
+    fold_gain_kernel<bf16><<<blocks, 256, 0, ctx->stream>>>((bf16*)W, g, total, in_f);
+  else
+    fold_gain_kernel<float><<<blocks, 256, 0, ctx->stream>>>((float*)W, g, total, in_f);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void* out) {
+  const auto& d = ctx->desc;
+  int total = d.ltp_dlow * 2 * d.ltp_rank;
+  if (d.dtype == SPTS_BF16)
+    pad_proxy_kernel<bf16><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const bf16*)vg, (const bf16*)vu, d.ltp_dlow, d.ltp_rank, (bf16*)out);
+  else
+    pad_proxy_kernel<float><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const float*)vg, (const float*)vu, d.ltp_dlow, d.ltp_rank, (float*)out);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_head(spts_ctx* ctx, const void* x_row, const void* lm_head, float* logits,
+                        int32_t* token_out) {
+  const auto& d = ctx->desc;
+  const int wpb = 8;
+  size_t sm = (size_t)d.hidden * sizeof(float);
+  if (d.dtype == SPTS_BF16)
+    head_logits_kernel<bf16><<<ceil_div(d.vocab, wpb), wpb * 32, sm, ctx->stream>>>(
+        (const bf16*)x_row, (const bf16*)lm_head, d.hidden, d.vocab, d.rms_eps, logits);
+  else
+    head_logits_kernel<float><<<ceil_div(d.vocab, wpb), wpb * 32, sm, ctx->stream>>>(
+        (const float*)x_row, (const float*)lm_head, d.hidden, d.vocab, d.rms_eps, logits);
+  SPTS_CUDA_OK(ctx);
+  if (token_out != nullptr) {
+    argmax_kernel<<<1, 1024, 0, ctx->stream>>>(logits, d.vocab, token_out);
+    SPTS_CUDA_OK(ctx);
+  }
+  return SPTS_OK;
+}
+
+}  // namespace spts

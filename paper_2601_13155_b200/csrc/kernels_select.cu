@@ -1,0 +1,299 @@
+// Top-k selection (Eq. 5 / 15 / 16) by radix select, and the gathers used by stage-end
+// compaction (Algorithm 1, "X <- X[T, :]").  Integer / compare work only: results are exact.
+//
+// Selection rule: score descending, then index ascending; -0.0 == +0.0; NaN ranks with -inf;
+// with SPTS_FORCE_LAST the last element ranks first.  Output indices are ascending.
+#include "spts_common.cuh"
+
+namespace spts {
+
+namespace {
+
+constexpr int TK_THREADS = 256;
+constexpr int TK_PER_THREAD = TOPK_CHUNK / TK_THREADS;  // 8
+
+// scratch layout (uint32 words)
+constexpr int SC_HIST = 0;            // [4][256]
+constexpr int SC_PREFIX = 4 * 256;    // threshold key bits found so far
+constexpr int SC_KREM = SC_PREFIX + 1;  // how many still to take inside the current bucket
+constexpr int SC_DONE = SC_PREFIX + 2;  // blocks finished (reset by the last block)
+constexpr int SC_NAN = SC_PREFIX + 3;
+constexpr int SC_CTA = SC_PREFIX + 16;  // [2][TOPK_MAX_CTAS]: out_base, eq_base
+
+__device__ __forceinline__ uint32_t score_key(float s, bool* nonfinite) {
+  uint32_t u = __float_as_uint(s);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) {  // NaN ranks with -inf
+    *nonfinite = true;
+    return 0x007FFFFFu;
+  }
+  if (u == 0x80000000u) u = 0u;  // -0.0 -> +0.0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ uint32_t load_key(const float* scores, int i, int N, bool force_last,
+                                             bool* nonfinite) {
+  if (force_last && i == N - 1) return 0xFFFFFFFFu;
+  return score_key(scores[i], nonfinite);
+}
+
+// One radix pass: histogram of the 8-bit digit at `shift` over the keys that match the prefix
+// found so far; the last block to finish picks the bucket holding the k-th largest key.
+__global__ void __launch_bounds__(TK_THREADS)
+topk_hist_kernel(const float* __restrict__ scores, int N, int k, int pass, int force_last,
+                 uint32_t* __restrict__ sc, int* status) {
+  __shared__ uint32_t h[256];
+  __shared__ uint32_t scan[256];
+  __shared__ bool is_last;
+  const int tid = threadIdx.x;
+  h[tid] = 0;
+  __syncthreads();
+  const int shift = 24 - 8 * pass;
+  const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (32 - 8 * pass));
+  const uint32_t prefix = pass == 0 ? 0u : sc[SC_PREFIX];
+  bool nonfinite = false;
+  const int base = blockIdx.x * TOPK_CHUNK;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    int i = base + e * TK_THREADS + tid;
+    if (i < N) {
+      uint32_t key = load_key(scores, i, N, force_last != 0, &nonfinite);
+      if ((key & mask) == prefix) atomicAdd(&h[(key >> shift) & 0xFFu], 1u);
+    }
+  }
+  if (nonfinite && pass == 0) set_status(status, SPTS_ERR_NONFINITE);
+  __syncthreads();
+  if (h[tid] != 0) atomicAdd(&sc[SC_HIST + pass * 256 + tid], h[tid]);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t done = atomicAdd(&sc[SC_DONE], 1u);
+    is_last = (done == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // inclusive scan from the top digit downwards: scan[t] = sum of hist[255 - t .. 255]
+  uint32_t mine = ((volatile uint32_t*)sc)[SC_HIST + pass * 256 + (255 - tid)];
+  scan[tid] = mine;
+  __syncthreads();
+  for (int o = 1; o < 256; o <<= 1) {
+    uint32_t v = tid >= o ? scan[tid - o] : 0u;
+    __syncthreads();
+    scan[tid] += v;
+    __syncthreads();
+  }
+  const uint32_t krem = pass == 0 ? (uint32_t)k : ((volatile uint32_t*)sc)[SC_KREM];
+  const uint32_t above = scan[tid] - mine;  // keys in strictly higher buckets
+  __syncthreads();
+  if (above < krem && krem <= scan[tid]) {  // exactly one thread
+    sc[SC_PREFIX] = prefix | ((uint32_t)(255 - tid) << shift);
+    sc[SC_KREM] = krem - above;
+  }
+  if (tid == 0) sc[SC_DONE] = 0u;
+}
+
+// Per-chunk counts of keys above / equal to the threshold; the last block turns them into
+// output offsets so that the emit kernel writes ascending indices without further sync.
+__global__ void __launch_bounds__(TK_THREADS)
+topk_count_kernel(const float* __restrict__ scores, int N, int force_last, uint32_t* __restrict__ sc) {
+  __shared__ uint32_t s_gt[TK_THREADS / 32], s_eq[TK_THREADS / 32];
+  __shared__ bool is_last;
+  __shared__ uint32_t carry_out, carry_eq;
+  __shared__ uint32_t sa[TK_THREADS], sb[TK_THREADS];
+  const int tid = threadIdx.x;
+  const uint32_t T = sc[SC_PREFIX];
+  uint32_t* cta_a = sc + SC_CTA;
+  uint32_t* cta_b = sc + SC_CTA + TOPK_MAX_CTAS;
+  bool nf = false;
+  uint32_t gt = 0, eq = 0;
+  const int base = blockIdx.x * TOPK_CHUNK;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    int i = base + e * TK_THREADS + tid;
+    if (i < N) {
+      uint32_t key = load_key(scores, i, N, force_last != 0, &nf);
+      gt += key > T;
+      eq += key == T;
+    }
+  }
+  gt = __reduce_add_sync(0xffffffffu, gt);
+  eq = __reduce_add_sync(0xffffffffu, eq);
+  if ((tid & 31) == 0) { s_gt[tid >> 5] = gt; s_eq[tid >> 5] = eq; }
+  __syncthreads();
+  if (tid == 0) {
+    uint32_t a = 0, b = 0;
+    for (int w = 0; w < TK_THREADS / 32; ++w) { a += s_gt[w]; b += s_eq[w]; }
+    cta_a[blockIdx.x] = a;
+    cta_b[blockIdx.x] = b;
+    __threadfence();
+    uint32_t done = atomicAdd(&sc[SC_DONE], 1u);
+    is_last = (done == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const uint32_t need_eq = ((volatile uint32_t*)sc)[SC_KREM];
+  if (tid == 0) { carry_out = 0; carry_eq = 0; }
+  __syncthreads();
+  const int nb = gridDim.x;
+  for (int c0 = 0; c0 < nb; c0 += TK_THREADS) {
+    int b = c0 + tid;
+    uint32_t g = 0, e = 0;
+    if (b < nb) { g = ((volatile uint32_t*)cta_a)[b]; e = ((volatile uint32_t*)cta_b)[b]; }
+    // exclusive scan of eq counts first (needed to clip the equal keys taken per chunk)
+    sb[tid] = e;
+    __syncthreads();
+    for (int o = 1; o < TK_THREADS; o <<= 1) {
+      uint32_t v = tid >= o ? sb[tid - o] : 0u;
+      __syncthreads();
+      sb[tid] += v;
+      __syncthreads();
+    }
+    uint32_t eq_base = carry_eq + sb[tid] - e;
+    uint32_t take = 0;
+    if (eq_base < need_eq) take = min(e, need_eq - eq_base);
+    sa[tid] = g + take;
+    __syncthreads();
+    for (int o = 1; o < TK_THREADS; o <<= 1) {
+      uint32_t v = tid >= o ? sa[tid - o] : 0u;
+      __syncthreads();
+      sa[tid] += v;
+      __syncthreads();
+    }
+    uint32_t out_base = carry_out + sa[tid] - (g + take);
+    if (b < nb) { cta_a[b] = out_base; cta_b[b] = eq_base; }
+    __syncthreads();
+    if (tid == TK_THREADS - 1) { carry_out += sa[tid]; carry_eq += sb[tid]; }
+    __syncthreads();
+  }
+  if (tid == 0) sc[SC_DONE] = 0u;
+}
+
+__global__ void __launch_bounds__(TK_THREADS)
+topk_emit_kernel(const float* __restrict__ scores, int N, int k, int force_last,
+                 const uint32_t* __restrict__ sc, int32_t* __restrict__ idx_out) {
+  __shared__ uint32_t s_sel[TK_THREADS], s_eq[TK_THREADS];
+  const int tid = threadIdx.x;
+  const uint32_t T = sc[SC_PREFIX];
+  const uint32_t need_eq = sc[SC_KREM];
+  const uint32_t out_base = sc[SC_CTA + blockIdx.x];
+  const uint32_t eq_base = sc[SC_CTA + TOPK_MAX_CTAS + blockIdx.x];
+  bool nf = false;
+  // thread t owns TK_PER_THREAD consecutive elements so that a scan over threads is index order
+  const int i0 = blockIdx.x * TOPK_CHUNK + tid * TK_PER_THREAD;
+  uint32_t keys[TK_PER_THREAD];
+  uint32_t eq = 0;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    int i = i0 + e;
+    keys[e] = i < N ? load_key(scores, i, N, force_last != 0, &nf) : 0u;
+    eq += (i < N && keys[e] == T);
+  }
+  s_eq[tid] = eq;
+  __syncthreads();
+  for (int o = 1; o < TK_THREADS; o <<= 1) {
+    uint32_t v = tid >= o ? s_eq[tid - o] : 0u;
+    __syncthreads();
+    s_eq[tid] += v;
+    __syncthreads();
+  }
+  uint32_t eq_rank = eq_base + s_eq[tid] - eq;  // rank of my first equal key among all equal keys
+  uint32_t flags = 0, sel = 0;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    int i = i0 + e;
+    if (i < N) {
+      bool take = keys[e] > T;
+      if (keys[e] == T) { take = eq_rank < need_eq; ++eq_rank; }
+      if (take) { flags |= 1u << e; ++sel; }
+    }
+  }
+  s_sel[tid] = sel;
+  __syncthreads();
+  for (int o = 1; o < TK_THREADS; o <<= 1) {
+    uint32_t v = tid >= o ? s_sel[tid - o] : 0u;
+    __syncthreads();
+    s_sel[tid] += v;
+    __syncthreads();
+  }
+  uint32_t w = out_base + s_sel[tid] - sel;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    if (flags & (1u << e)) {
+      if (w < (uint32_t)k) idx_out[w] = i0 + e;
+      ++w;
+    }
+  }
+}
+
+__global__ void iota_kernel(int32_t* out, int n) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = i;
+}
+
+// dst[i, :] = src[idx[i], :], 16 bytes per thread.
+__global__ void gather_rows_kernel(const uint4* __restrict__ src, const int32_t* __restrict__ idx,
+                                   int n_rows, int row_vec, uint4* __restrict__ dst) {
+  size_t total = (size_t)n_rows * row_vec;
+  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
+       t += (size_t)gridDim.x * blockDim.x) {
+    int r = (int)(t / row_vec);
+    int c = (int)(t - (size_t)r * row_vec);
+    dst[t] = src[(size_t)idx[r] * row_vec + c];
+  }
+}
+
+__global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ idx,
+                                  int n, int32_t* __restrict__ dst) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[idx[i]];
+}
+
+}  // namespace
+
+spts_status launch_topk(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags,
+                        int32_t* idx_out, uint32_t* scratch) {
+  if (scores == nullptr || idx_out == nullptr || N < 1 || k < 1 || k > N) return SPTS_ERR_INVALID_ARG;
+  const int nb = ceil_div(N, TOPK_CHUNK);
+  if (nb > TOPK_MAX_CTAS) return SPTS_ERR_SHAPE;
+  cudaStream_t st = ctx->stream;
+  if (k == N) {  // TopK of everything: the identity list
+    iota_kernel<<<ceil_div(N, 256), 256, 0, st>>>(idx_out, N);
+    SPTS_CUDA_OK(ctx);
+    return SPTS_OK;
+  }
+  const int fl = (flags & SPTS_FORCE_LAST) ? 1 : 0;
+  if (cudaMemsetAsync(scratch, 0, (4 * 256 + 16) * sizeof(uint32_t), st) != cudaSuccess) return SPTS_ERR_CUDA;
+  for (int pass = 0; pass < 4; ++pass) {
+    topk_hist_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, pass, fl, scratch, ctx->ws.status);
+    SPTS_CUDA_OK(ctx);
+  }
+  topk_count_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, fl, scratch);
+  SPTS_CUDA_OK(ctx);
+  topk_emit_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, fl, scratch, idx_out);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* idx, int n_rows,
+                               int row_bytes, void* dst) {
+  if (row_bytes % 16 != 0) return SPTS_ERR_SHAPE;
+  if (n_rows == 0) return SPTS_OK;
+  int row_vec = row_bytes / 16;
+  size_t total = (size_t)n_rows * row_vec;
+  int blocks = (int)((total + 255) / 256);
+  int cap = ctx->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  gather_rows_kernel<<<blocks, 256, 0, ctx->stream>>>((const uint4*)src, idx, n_rows, row_vec, (uint4*)dst);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst) {
+  if (n == 0) return SPTS_OK;
+  gather_i32_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(src, idx, n, dst);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+}  // namespace spts

@@ -1,0 +1,445 @@
+// C boundary of the SPTS library: argument checks, workspace carving and the per-layer
+// schedule of Algorithm 1.  Everything here is host code that enqueues kernels on the context's
+// stream; no call synchronises except spts_last_device_status().
+#include <new>
+#include <cstring>
+
+#include "spts_common.cuh"
+
+using namespace spts;
+
+namespace {
+
+struct Carver {
+  char* base;
+  size_t off;
+  template <typename T> T* take(size_t count) {
+    off = align_up(off, 256);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+size_t elt_size(const spts_model_desc& d) { return d.dtype == SPTS_BF16 ? 2 : 4; }
+
+bool shape_ok(const spts_model_desc& d) {
+  if (d.hidden <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.ffn_dim <= 0) return false;
+  if (d.n_q_heads % d.n_kv_heads != 0) return false;
+  if (d.head_dim != 64 && d.head_dim != 128) return false;
+  if (d.hidden % 8 || d.ffn_dim % 8 || d.ltp_dlow % 8 || d.ltp_rank % 8) return false;
+  if (d.ltp_dlow <= 0 || d.ltp_rank <= 0) return false;
+  if (d.dtype != SPTS_BF16 && d.dtype != SPTS_FP32) return false;
+  if (d.n_layers <= 0) return false;
+  return true;
+}
+
+// Shapes the tcgen05 kernels cover.
+bool tc_shape_ok(const spts_model_desc& d) {
+  return d.dtype == SPTS_BF16 && d.head_dim == 128 && d.hidden % 64 == 0 && d.ffn_dim % 64 == 0 &&
+         d.ltp_dlow % 64 == 0 && d.ltp_rank % 16 == 0 && (d.n_q_heads * d.head_dim) % 64 == 0;
+}
+
+size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws) {
+  Carver c{reinterpret_cast<char*>(base), 0};
+  Workspace w;
+  memset(&w, 0, sizeof(w));
+  const size_t es = elt_size(d);
+  const size_t N = (size_t)Nmax;
+  const size_t HD = (size_t)d.n_q_heads * d.head_dim, KD = (size_t)d.n_kv_heads * d.head_dim;
+  const size_t Npad = align_up(N, 128);
+  w.status = c.take<int>(64);
+  w.rstd = c.take<float>(N);
+  w.q = c.take<float>(HD);
+  w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
+  w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
+  w.logits = c.take<float>((size_t)d.n_q_heads * Npad);
+  w.head_stats = c.take<float>(2 * (size_t)d.n_q_heads);
+  w.s_mha = c.take<float>(N);
+  w.s_ffn = c.take<float>(N);
+  w.csq_parts = ceil_div(d.hidden, 64);
+  w.csq = c.take<float>(N * w.csq_parts);
+  w.idx_a = c.take<int32_t>(Npad);
+  w.idx_f = c.take<int32_t>(Npad);
+  w.idx_p = c.take<int32_t>(Npad);
+  w.topk_scratch = c.take<uint32_t>(TOPK_SCRATCH_WORDS);
+  w.k_all = c.take<char>(N * KD * es);
+  w.q_act = c.take<char>(Npad * HD * es);
+  w.v_t = c.take<char>(KD * Npad * es);
+  w.o_att = c.take<char>(Npad * HD * es);
+  w.hm = c.take<char>(Npad * (size_t)d.ffn_dim * es);
+  w.t1 = c.take<char>(Npad * 2 * (size_t)d.ltp_rank * es);
+  w.hlow = c.take<char>(Npad * (size_t)d.ltp_dlow * es);
+  w.t2 = c.take<char>(Npad * (size_t)d.ltp_rank * es);
+  w.acc32_elems = N * KD;
+  w.acc32 = c.take<float>(w.acc32_elems);
+  w.dec = c.take<float>(decode_scratch_floats(d));
+  w.logits_v = c.take<float>((size_t)(d.vocab > 0 ? d.vocab : 1));
+  w.xrow = c.take<char>((size_t)d.hidden * es);
+  if (ws) *ws = w;
+  return align_up(c.off, 256);
+}
+
+bool use_tc(const spts_ctx* ctx) { return ctx->desc.dtype == SPTS_BF16 && !ctx->reference_kernels; }
+
+// One GEMM with fused epilogue on whichever kernel family the context uses.
+struct Gemm {
+  const void* A; int lda; int a_rows;
+  const int32_t* idx; const int32_t* dst_idx;
+  const void* W; const void* W2;
+  int M, Nout, K;
+  const float* rowscale;
+  void* out; int ldo;
+  void* out_t; int ldt;
+  const float* q; float* logits; int ld_logits;
+  float* csq;
+};
+
+spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
+  if (g.M <= 0) return SPTS_OK;
+  const auto& d = ctx->desc;
+  if (use_tc(ctx)) {
+    TcGemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = (const bf16*)g.A; a.lda = g.lda; a.a_rows = g.a_rows; a.idx = g.idx; a.dst_idx = g.dst_idx;
+    a.W = (const bf16*)g.W; a.W2 = (const bf16*)g.W2; a.M = g.M; a.Nout = g.Nout; a.K = g.K;
+    a.rowscale = g.rowscale; a.out = (bf16*)g.out; a.ldo = g.ldo; a.out_t = (bf16*)g.out_t; a.ldt = g.ldt;
+    a.q = g.q; a.logits = g.logits; a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads;
+    a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts;
+    return launch_tc_gemm(ctx, epi, a);
+  }
+  RefGemmArgs a;
+  memset(&a, 0, sizeof(a));
+  a.A = g.A; a.lda = g.lda; a.idx = g.idx; a.dst_idx = g.dst_idx; a.W = g.W; a.W2 = g.W2;
+  a.M = g.M; a.Nout = g.Nout; a.K = g.K; a.rowscale = g.rowscale; a.out = g.out; a.ldo = g.ldo;
+  a.out_t = g.out_t; a.ldt = g.ldt; a.head_dim = d.head_dim; a.q = g.q; a.logits = g.logits;
+  a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads; a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts;
+  return launch_ref_gemm(ctx, epi, a);
+}
+
+#define TRY(x) do { spts_status s__ = (x); if (s__ != SPTS_OK) return s__; } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// PAP (Eq. 4): rstd, rotary table, q of the last row, K of every row with the logits taken from
+// the unrounded keys in the projection's epilogue, then the head-mean softmax.
+spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const int32_t* pos, int N,
+                         void* K_out, bool want_scores, float* S_out) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int KD = d.n_kv_heads * d.head_dim;
+  const int ld = (int)align_up((size_t)N, 128);
+  TRY(launch_rstd(ctx, X, N, ws.rstd));
+  TRY(launch_rope_table(ctx, pos, N, ws.rope_cs));
+  if (want_scores) TRY(launch_q_last(ctx, X, ws.rope_cs, N, w->wq, ws.rstd, ws.q));
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->wk; g.M = N; g.Nout = KD; g.K = d.hidden;
+  g.rowscale = ws.rstd; g.out = K_out; g.ldo = KD;
+  if (want_scores) { g.q = ws.q; g.logits = ws.logits; g.ld_logits = ld; }
+  TRY(run_gemm(ctx, REF_ROPE, g));
+  if (want_scores) TRY(launch_pap_softmax(ctx, ws.logits, ld, N, S_out));
+  return SPTS_OK;
+}
+
+// LTP (Eq. 12-14) on rows already normalised through `rstd`.
+spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const float* S_mha, int N,
+                         float* C_out, float* S_ffn_out) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int r = d.ltp_rank, Dl = d.ltp_dlow;
+  const size_t es = elt_size(d);
+  TRY(launch_pad_proxy(ctx, w->vg, w->vu, ws.vgu_pad));
+  Gemm g;
+  // t1 = [x Ug | x Uu]  (two column blocks of one [N, 2r] matrix)
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->ug; g.M = N; g.Nout = r; g.K = d.hidden;
+  g.rowscale = ws.rstd; g.out = ws.t1; g.ldo = 2 * r;
+  TRY(run_gemm(ctx, REF_STORE, g));
+  g.W = w->uu; g.out = (char*)ws.t1 + (size_t)r * es;
+  TRY(run_gemm(ctx, REF_STORE, g));
+  // hlow = silu(t_g Vg) * (t_u Vu)
+  memset(&g, 0, sizeof(g));
+  g.A = ws.t1; g.lda = 2 * r; g.a_rows = N; g.W = ws.vgu_pad; g.W2 = (char*)ws.vgu_pad + (size_t)Dl * 2 * r * es;
+  g.M = N; g.Nout = Dl; g.K = 2 * r; g.out = ws.hlow; g.ldo = Dl;
+  TRY(run_gemm(ctx, REF_SWIGLU, g));
+  // t2 = hlow Vd^T
+  memset(&g, 0, sizeof(g));
+  g.A = ws.hlow; g.lda = Dl; g.a_rows = N; g.W = w->vd; g.M = N; g.Nout = r; g.K = Dl; g.out = ws.t2; g.ldo = r;
+  TRY(run_gemm(ctx, REF_STORE, g));
+  // C^2 = || t2 Ud^T ||^2, summed in the epilogue
+  memset(&g, 0, sizeof(g));
+  g.A = ws.t2; g.lda = r; g.a_rows = N; g.W = w->ud; g.M = N; g.Nout = d.hidden; g.K = r; g.csq = ws.csq;
+  TRY(run_gemm(ctx, REF_SUMSQ, g));
+  const int parts = use_tc(ctx) ? tc_sumsq_parts(d.hidden) : ceil_div(d.hidden, 64);
+  TRY(launch_ffn_score(ctx, ws.csq, parts, S_mha, N, C_out, S_ffn_out));
+  return SPTS_OK;
+}
+
+spts_status check_ctx(const spts_ctx* ctx) { return ctx == nullptr ? SPTS_ERR_INVALID_ARG : SPTS_OK; }
+
+}  // namespace
+
+extern "C" {
+
+size_t spts_workspace_bytes(const spts_model_desc* desc, int max_seq) {
+  if (desc == nullptr || max_seq < 1 || !shape_ok(*desc)) return 0;
+  return carve(*desc, max_seq, nullptr, nullptr);
+}
+
+spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream, spts_ctx** out) {
+  if (desc == nullptr || out == nullptr || workspace == nullptr || max_seq < 1) return SPTS_ERR_INVALID_ARG;
+  if (!shape_ok(*desc)) return SPTS_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return SPTS_ERR_INVALID_ARG;
+  if (carve(*desc, max_seq, nullptr, nullptr) > workspace_bytes) return SPTS_ERR_WORKSPACE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SPTS_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SPTS_ERR_CUDA;
+  if (desc->dtype == SPTS_BF16 && prop.major != 10) return SPTS_ERR_UNSUPPORTED;   // sm_100a only
+  spts_ctx* ctx = new (std::nothrow) spts_ctx;
+  if (ctx == nullptr) return SPTS_ERR_INVALID_ARG;
+  ctx->desc = *desc;
+  ctx->max_seq = max_seq;
+  ctx->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  ctx->launches = 0;
+  ctx->sm_count = prop.multiProcessorCount;
+  ctx->encode_tiled = nullptr;
+  carve(*desc, max_seq, workspace, &ctx->ws);
+  ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
+  if (!ctx->reference_kernels) {
+    spts_status s = tc_init(ctx);
+    if (s != SPTS_OK) { delete ctx; return s; }
+  }
+  if (cudaMemsetAsync(ctx->ws.status, 0, 64 * sizeof(int), ctx->stream) != cudaSuccess) { delete ctx; return SPTS_ERR_CUDA; }
+  if (cudaMemsetAsync(ctx->ws.topk_scratch, 0, TOPK_SCRATCH_WORDS * sizeof(uint32_t), ctx->stream) != cudaSuccess) {
+    delete ctx;
+    return SPTS_ERR_CUDA;
+  }
+  *out = ctx;
+  return SPTS_OK;
+}
+
+void spts_destroy(spts_ctx* ctx) { delete ctx; }
+
+spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
+  TRY(check_ctx(ctx));
+  if (option == SPTS_REFERENCE_KERNELS) {
+    if (ctx->desc.dtype == SPTS_FP32 || !tc_shape_ok(ctx->desc)) return value ? SPTS_OK : SPTS_ERR_UNSUPPORTED;
+    if (!value && ctx->encode_tiled == nullptr) TRY(tc_init(ctx));
+    ctx->reference_kernels = value != 0;
+    return SPTS_OK;
+  }
+  return SPTS_ERR_INVALID_ARG;
+}
+
+spts_status spts_last_device_status(spts_ctx* ctx) {
+  TRY(check_ctx(ctx));
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return SPTS_ERR_CUDA;
+  int st = 0;
+  if (cudaMemcpy(&st, ctx->ws.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SPTS_ERR_CUDA;
+  if (st != 0 && cudaMemset(ctx->ws.status, 0, sizeof(int)) != cudaSuccess) return SPTS_ERR_CUDA;
+  return (spts_status)st;
+}
+
+int64_t spts_launch_count(const spts_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+spts_status spts_fold_norm_gain(spts_ctx* ctx, void* W, const float* g, int out_features, int in_features) {
+  TRY(check_ctx(ctx));
+  if (W == nullptr || g == nullptr || out_features < 1 || in_features < 1) return SPTS_ERR_INVALID_ARG;
+  return launch_fold_gain(ctx, W, g, out_features, in_features);
+}
+
+spts_status spts_pap_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const int32_t* pos, int N,
+                           void* K_out, float* S_mha_out) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || X == nullptr || pos == nullptr || S_mha_out == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || N > ctx->max_seq) return SPTS_ERR_SHAPE;
+  if (!aligned16(X) || !aligned16(K_out) || !aligned16(w->wk) || !aligned16(w->wq)) return SPTS_ERR_INVALID_ARG;
+  return pap_pipeline(ctx, w, X, pos, N, K_out ? K_out : ctx->ws.k_all, true, S_mha_out);
+}
+
+spts_status spts_ltp_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const float* S_mha, int N,
+                           float* C_out, float* S_ffn_out) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || X == nullptr || S_mha == nullptr || S_ffn_out == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || N > ctx->max_seq) return SPTS_ERR_SHAPE;
+  if (!aligned16(X)) return SPTS_ERR_INVALID_ARG;
+  TRY(launch_rstd(ctx, X, N, ctx->ws.rstd));
+  return ltp_pipeline(ctx, w, X, S_mha, N, C_out, S_ffn_out);
+}
+
+spts_status spts_topk_select(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags, int32_t* idx_out) {
+  TRY(check_ctx(ctx));
+  if (scores == nullptr || idx_out == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || k < 1 || k > N) return SPTS_ERR_INVALID_ARG;
+  return launch_topk(ctx, scores, N, k, flags, idx_out, ctx->ws.topk_scratch);
+}
+
+spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos, int N,
+                                    int m_attn, int m_ffn, uint32_t flags, spts_kv_layer* cache, float* S_mha_out,
+                                    int32_t* idx_attn_out, int32_t* idx_ffn_out) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || X == nullptr || pos == nullptr || cache == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (cache->k == nullptr || cache->v == nullptr || cache->pos == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || N > ctx->max_seq) return SPTS_ERR_SHAPE;
+  if (m_attn < 1 || m_attn > N || m_ffn < 1 || m_ffn > N) return SPTS_ERR_INVALID_ARG;
+  if (cache->capacity < m_attn) return SPTS_ERR_WORKSPACE;
+  if (!aligned16(X) || !aligned16(cache->k) || !aligned16(cache->v)) return SPTS_ERR_INVALID_ARG;
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int D = d.hidden, HD = d.n_q_heads * d.head_dim, KD = d.n_kv_heads * d.head_dim;
+  const size_t es = elt_size(d);
+  const bool sel_a = m_attn < N, sel_f = m_ffn < N;
+  const bool want_scores = sel_a || sel_f || S_mha_out != nullptr;
+  float* S = S_mha_out ? S_mha_out : ws.s_mha;
+  const bool tc = use_tc(ctx);
+
+  // ---- PAP + reduced MHA
+  void* k_dst = sel_a ? ws.k_all : cache->k;
+  TRY(pap_pipeline(ctx, w, X, pos, N, k_dst, want_scores, S));
+  const int32_t* idx_a = nullptr;
+  if (sel_a) {
+    int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
+    TRY(launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
+    TRY(launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
+    TRY(launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
+    idx_a = ia;
+  } else {
+    if (cudaMemcpyAsync(cache->pos, pos, (size_t)N * sizeof(int32_t), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+      return SPTS_ERR_CUDA;
+    if (idx_attn_out) TRY(launch_topk(ctx, S, N, N, flags, idx_attn_out, ws.topk_scratch));
+  }
+  const int ldvt = (int)align_up((size_t)m_attn, 128);
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_a; g.W = w->wq; g.M = m_attn; g.Nout = HD; g.K = D;
+  g.rowscale = ws.rstd; g.out = ws.q_act; g.ldo = HD;
+  TRY(run_gemm(ctx, REF_ROPE, g));
+  g.W = w->wv; g.Nout = KD; g.out = cache->v; g.ldo = KD;
+  if (tc) { g.out_t = ws.v_t; g.ldt = ldvt; }
+  TRY(run_gemm(ctx, REF_STORE, g));
+  if (tc) TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)ws.v_t, ldvt, m_attn,
+                                  (bf16*)ws.o_att));
+  else TRY(launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att));
+  memset(&g, 0, sizeof(g));
+  g.A = ws.o_att; g.lda = HD; g.a_rows = m_attn; g.dst_idx = idx_a; g.W = w->wo; g.M = m_attn; g.Nout = D; g.K = HD;
+  g.out = X; g.ldo = D;
+  TRY(run_gemm(ctx, REF_RESID, g));
+  cache->len = m_attn;
+
+  // ---- LTP + reduced FFN on the updated residual
+  TRY(launch_rstd(ctx, X, N, ws.rstd));
+  const int32_t* idx_f = nullptr;
+  if (sel_f) {
+    int32_t* jf = idx_ffn_out ? idx_ffn_out : ws.idx_f;
+    TRY(ltp_pipeline(ctx, w, X, S, N, nullptr, ws.s_ffn));
+    TRY(launch_topk(ctx, ws.s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
+    idx_f = jf;
+  } else if (idx_ffn_out) {
+    TRY(launch_topk(ctx, S, N, N, flags, idx_ffn_out, ws.topk_scratch));
+  }
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_f; g.W = w->w_gate; g.W2 = w->w_up; g.M = m_ffn; g.Nout = d.ffn_dim;
+  g.K = D; g.rowscale = ws.rstd; g.out = ws.hm; g.ldo = d.ffn_dim;
+  TRY(run_gemm(ctx, REF_SWIGLU, g));
+  memset(&g, 0, sizeof(g));
+  g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = m_ffn; g.dst_idx = idx_f; g.W = w->w_down; g.M = m_ffn; g.Nout = D;
+  g.K = d.ffn_dim; g.out = X; g.ldo = D;
+  TRY(run_gemm(ctx, REF_RESID, g));
+  return SPTS_OK;
+}
+
+spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* pos_in, const int32_t* orig_in,
+                              const float* S_mha, int N, int n_next, uint32_t flags, void* X_out, int32_t* pos_out,
+                              int32_t* orig_out, int32_t* idx_out) {
+  TRY(check_ctx(ctx));
+  if (X_in == nullptr || pos_in == nullptr || orig_in == nullptr || S_mha == nullptr || X_out == nullptr ||
+      pos_out == nullptr || orig_out == nullptr)
+    return SPTS_ERR_INVALID_ARG;
+  if (X_in == X_out || pos_in == pos_out || orig_in == orig_out) return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || N > ctx->max_seq || n_next < 1) return SPTS_ERR_SHAPE;
+  if (n_next > N) n_next = N;
+  if (!aligned16(X_in) || !aligned16(X_out)) return SPTS_ERR_INVALID_ARG;
+  int32_t* idx = idx_out ? idx_out : ctx->ws.idx_p;
+  TRY(launch_topk(ctx, S_mha, N, n_next, flags, idx, ctx->ws.topk_scratch));
+  TRY(launch_gather_rows(ctx, X_in, idx, n_next, (int)(ctx->desc.hidden * elt_size(ctx->desc)), X_out));
+  TRY(launch_gather_i32(ctx, pos_in, idx, n_next, pos_out));
+  TRY(launch_gather_i32(ctx, orig_in, idx, n_next, orig_out));
+  return SPTS_OK;
+}
+
+spts_status spts_first_token(spts_ctx* ctx, const void* x_row, const void* lm_head, float* logits_out,
+                             int32_t* token_out) {
+  TRY(check_ctx(ctx));
+  if (x_row == nullptr || lm_head == nullptr || ctx->desc.vocab < 1) return SPTS_ERR_INVALID_ARG;
+  if (!aligned16(x_row) || !aligned16(lm_head)) return SPTS_ERR_INVALID_ARG;
+  return launch_head(ctx, x_row, lm_head, logits_out ? logits_out : ctx->ws.logits_v, token_out);
+}
+
+spts_status spts_prefill(spts_ctx* ctx, const spts_model_weights* mw, const spts_layer_plan* plan, void* X,
+                         int32_t* pos, int32_t* orig, void* X_alt, int32_t* pos_alt, int32_t* orig_alt, int N,
+                         uint32_t flags, spts_kv_layer* caches, int32_t* n_final, int32_t* final_in_alt,
+                         int32_t* token_out) {
+  TRY(check_ctx(ctx));
+  if (mw == nullptr || mw->layers == nullptr || plan == nullptr || X == nullptr || pos == nullptr || orig == nullptr ||
+      caches == nullptr)
+    return SPTS_ERR_INVALID_ARG;
+  if (N < 1 || N > ctx->max_seq) return SPTS_ERR_SHAPE;
+  const auto& d = ctx->desc;
+  void* xc = X; int32_t* pc = pos; int32_t* oc = orig;
+  void* xa = X_alt; int32_t* pa = pos_alt; int32_t* oa = orig_alt;
+  int cur = N, in_alt = 0;
+  for (int l = 0; l < d.n_layers; ++l) {
+    const spts_layer_plan& p = plan[l];
+    if (p.m_attn < 1 || p.m_attn > cur || p.m_ffn < 1 || p.m_ffn > cur) return SPTS_ERR_INVALID_ARG;
+    const bool prune = p.prune_to > 0 && p.prune_to < cur;
+    if (prune && (xa == nullptr || pa == nullptr || oa == nullptr)) return SPTS_ERR_INVALID_ARG;
+    TRY(spts_layer_prefill_skip(ctx, &mw->layers[l], xc, pc, cur, p.m_attn, p.m_ffn, flags, &caches[l],
+                                prune ? ctx->ws.s_mha : nullptr, nullptr, nullptr));
+    if (prune) {
+      TRY(spts_msdp_compact(ctx, xc, pc, oc, ctx->ws.s_mha, cur, p.prune_to, flags, xa, pa, oa, nullptr));
+      void* tx = xc; xc = xa; xa = tx;
+      int32_t* tp = pc; pc = pa; pa = tp;
+      int32_t* to = oc; oc = oa; oa = to;
+      cur = p.prune_to;
+      in_alt ^= 1;
+    }
+  }
+  if (n_final) *n_final = cur;
+  if (final_in_alt) *final_in_alt = in_alt;
+  if (token_out != nullptr) {
+    if (mw->lm_head == nullptr) return SPTS_ERR_INVALID_ARG;
+    const char* last = (const char*)xc + (size_t)(cur - 1) * d.hidden * elt_size(d);
+    TRY(spts_first_token(ctx, last, mw->lm_head, nullptr, token_out));
+  }
+  return SPTS_OK;
+}
+
+spts_status spts_decode_step(spts_ctx* ctx, const spts_model_weights* mw, spts_kv_layer* caches, const void* x_in,
+                             int32_t token_in, int32_t pos, void* x_out, float* logits_out, int32_t* token_out) {
+  TRY(check_ctx(ctx));
+  if (mw == nullptr || mw->layers == nullptr || caches == nullptr) return SPTS_ERR_INVALID_ARG;
+  const auto& d = ctx->desc;
+  const size_t es = elt_size(d);
+  const void* x = x_in;
+  if (x == nullptr) {
+    if (mw->embed == nullptr || token_in < 0 || token_in >= d.vocab) return SPTS_ERR_INVALID_ARG;
+    x = (const char*)mw->embed + (size_t)token_in * d.hidden * es;
+  }
+  for (int l = 0; l < d.n_layers; ++l)
+    if (caches[l].len + 1 > caches[l].capacity) return SPTS_ERR_WORKSPACE;
+  TRY(launch_decode_load(ctx, x));
+  for (int l = 0; l < d.n_layers; ++l) TRY(launch_decode_layer(ctx, &mw->layers[l], &caches[l], pos));
+  // the residual is already rounded through the storage type; park it where the head can read it
+  void* xo = x_out ? x_out : ctx->ws.xrow;
+  TRY(launch_decode_store(ctx, xo));
+  if (logits_out != nullptr || token_out != nullptr) {
+    if (mw->lm_head == nullptr) return SPTS_ERR_INVALID_ARG;
+    TRY(launch_head(ctx, xo, mw->lm_head, logits_out ? logits_out : ctx->ws.logits_v, token_out));
+  }
+  return SPTS_OK;
+}
+
+}  // extern "C"

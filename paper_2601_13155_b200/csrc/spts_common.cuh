@@ -1,0 +1,179 @@
+// Shared declarations of the SPTS CUDA library (internal; the public boundary is include/spts.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "spts.h"
+
+namespace spts {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------------------------------------
+// device status word: kernels record problems here instead of trapping
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void set_status(int* status, int code) {
+  if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+// ---------------------------------------------------------------------------------------------
+// storage-type helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__host__ __device__ __forceinline__ size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+__host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------------------------
+struct Workspace {
+  // all device pointers, carved from the caller's workspace
+  int* status;          // [1] device status word
+  float* rstd;          // [Nmax]
+  float* q;             // [H*d]
+  float2* rope_cs;      // [Nmax, d/2] cos/sin of the rotary angles
+  void* vgu_pad;        // [2, Dlow, 2r] zero-padded proxy factors (gate | up)
+  float* logits;        // [H, Nmax]
+  float* head_stats;    // [2*H] max and sum of exp per head
+  float* s_mha;         // [Nmax]
+  float* s_ffn;         // [Nmax]
+  float* csq;           // [Nmax * csq_parts] partial sums of squares of the proxy output
+  int32_t* idx_a;       // [Nmax]
+  int32_t* idx_f;       // [Nmax]
+  int32_t* idx_p;       // [Nmax]
+  uint32_t* topk_scratch;  // radix-select scratch
+  void* k_all;          // [Nmax, Hkv*d]
+  void* q_act;          // [Nmax, H*d]
+  void* v_t;            // [Hkv*d, Nmax_pad] transposed V for the tensor-core attention
+  void* o_att;          // [Nmax, H*d]
+  void* hm;             // [Nmax, Dff]
+  void* t1;             // [Nmax, 2r]
+  void* hlow;           // [Nmax, Dlow]
+  void* t2;             // [Nmax, r]
+  float* acc32;         // fp32 accumulator scratch of the reference GEMM path
+  size_t acc32_elems;
+  void* dec;            // decode-step scratch
+  float* logits_v;      // [vocab]
+  void* xrow;           // [D] one hidden row in the storage type
+  int csq_parts;
+};
+
+}  // namespace spts
+
+struct spts_ctx {
+  spts_model_desc desc;
+  int max_seq;
+  cudaStream_t stream;
+  spts::Workspace ws;
+  bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
+  int64_t launches;
+  int sm_count;
+  void* encode_tiled;       // cuTensorMapEncodeTiled entry point (tensor-core mode)
+};
+
+namespace spts {
+
+// top-k scratch size in uint32 words
+static const int TOPK_CHUNK = 2048;           // elements per CTA in the select / emit kernels
+static const int TOPK_MAX_CTAS = 4096;        // supports N up to 8M
+static const int TOPK_SCRATCH_WORDS = 4 * 256 + 16 + 2 * TOPK_MAX_CTAS;
+
+// ---- kernels_select.cu
+spts_status launch_topk(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags,
+                        int32_t* idx_out, uint32_t* scratch);
+spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* idx, int n_rows,
+                               int row_bytes, void* dst);
+spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst);
+
+// ---- kernels_probe.cu
+spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd);
+spts_status launch_rope_table(spts_ctx* ctx, const int32_t* pos, int N, float2* cs);
+spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N, const void* wq,
+                          const float* rstd, float* q);
+spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void* out);
+spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, float* S);
+spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
+                             float* C_out, float* S_ffn);
+spts_status launch_fold_gain(spts_ctx* ctx, void* W, const float* g, int out_f, int in_f);
+spts_status launch_head(spts_ctx* ctx, const void* x_row, const void* lm_head, float* logits,
+                        int32_t* token_out);
+
+// ---- kernels_ref.cu : plain CUDA-core path (fp32 verification mode, bf16 cross-check)
+enum RefEpi {
+  REF_STORE = 0,       // out[i, j] = T(acc * rowscale)
+  REF_ROPE = 1,        // out[i, j] = T(rope(acc * rowscale)) ; optional PAP logits from unrounded values
+  REF_SWIGLU = 2,      // out[i, j] = T(silu(acc1 * rowscale) * (acc2 * rowscale))
+  REF_RESID = 3,       // X[dst(i), j] = T(X[dst(i), j] + acc)
+  REF_SUMSQ = 4        // csq[i, part] = sum_j acc^2 (deterministic partials)
+};
+struct RefGemmArgs {
+  const void* A; int lda;            // A [*, K] rows addressed through idx (or i when idx == nullptr)
+  const int32_t* idx;                // gather list for A rows, row scales and positions
+  const int32_t* dst_idx;            // REF_RESID: residual rows to update (nullptr: row i)
+  const void* W; const void* W2;     // [Nout, K] row-major; W2 for REF_SWIGLU
+  int M, Nout, K;
+  const float* rowscale;             // [*] indexed like A rows, or nullptr
+  void* out; int ldo;                // output matrix (REF_RESID: the residual stream X, row stride ldo)
+  void* out_t; int ldt;              // optional transposed copy out_t[j, i] (REF_STORE)
+  int head_dim;                      // REF_ROPE: rotary table rows are indexed like A rows
+  const float* q; float* logits; int ld_logits; int group;   // REF_ROPE + PAP: q [H, d], logits [H, ld]
+  float* csq; int csq_parts;         // REF_SUMSQ
+};
+spts_status launch_ref_gemm(spts_ctx* ctx, int epi, const RefGemmArgs& a);
+spts_status launch_ref_attention(spts_ctx* ctx, const void* Q, const void* K, const void* V, int m,
+                                 void* O);
+
+// ---- kernels_decode.cu
+size_t decode_scratch_floats(const spts_model_desc& d);
+spts_status launch_decode_load(spts_ctx* ctx, const void* x);     // x [D] -> fp32 residual scratch
+spts_status launch_decode_store(spts_ctx* ctx, void* x);          // fp32 residual scratch -> x [D]
+spts_status launch_decode_layer(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_layer* cache,
+                                int32_t pos);
+
+// ---- kernels_tc_gemm.cu / kernels_tc_attn.cu : tcgen05 path (bf16)
+enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4 };
+struct TcGemmArgs {
+  const bf16* A; int lda; int a_rows;   // A [a_rows, K]
+  const int32_t* idx;                   // optional gather list (TMA gather4)
+  const int32_t* dst_idx;               // TC_RESID scatter rows
+  const bf16* W; const bf16* W2;        // [Nout, K]
+  int M, Nout, K;
+  const float* rowscale;
+  bf16* out; int ldo;
+  bf16* out_t; int ldt;
+  const float* q; float* logits; int ld_logits; int group;
+  float* csq; int csq_parts;
+};
+spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
+spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* Vt, int ldvt,
+                                int m, bf16* O);
+spts_status tc_init(spts_ctx* ctx);          // resolves the tensor-map encoder, sets kernel attributes
+int tc_sumsq_parts(int n_out);               // partial sums per row written by TC_SUMSQ
+
+#define SPTS_CUDA_OK(ctx)                                   \
+  do {                                                      \
+    cudaError_t e__ = cudaGetLastError();                   \
+    if (e__ != cudaSuccess) return SPTS_ERR_CUDA;           \
+    (ctx)->launches++;                                      \
+  } while (0)
+
+}  // namespace spts

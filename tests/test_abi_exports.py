@@ -1,0 +1,71 @@
+"""The C-ABI library builds, loads without a GPU and exports every symbol include/spts.h declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib_path():
+    from paper_2601_13155_b200 import build
+    return build.build()
+
+
+def _declared():
+    src = open(os.path.join(ROOT, "include", "spts.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(spts_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_exports_match_header(lib_path):
+    lib = ctypes.CDLL(lib_path)
+    names = _declared()
+    assert {"spts_pap_score", "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip",
+            "spts_msdp_compact", "spts_decode_step"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    from paper_2601_13155_b200 import binding
+    assert set(binding.EXPORTS) == set(names)
+    binding.load_library()
+
+
+def test_workspace_bytes_is_host_arithmetic(lib_path):
+    from paper_2601_13155_b200 import binding, synth
+    lib = binding.load_library()
+    s = synth.LLAMA8B
+    d = binding.ModelDesc(s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn_dim, s.ltp_dlow, s.ltp_rank,
+                          s.n_layers, s.vocab, s.rms_eps, s.rope_theta, 0)
+    small = lib.spts_workspace_bytes(ctypes.byref(d), 8192)
+    big = lib.spts_workspace_bytes(ctypes.byref(d), 131072)
+    assert 0 < small < big < 40 * 2 ** 30
+    d.head_dim = 96                      # unsupported shape -> 0
+    assert lib.spts_workspace_bytes(ctypes.byref(d), 8192) == 0
+    assert lib.spts_workspace_bytes(None, 8192) == 0
+
+
+def test_host_argument_checks_need_no_gpu(lib_path):
+    from paper_2601_13155_b200 import binding
+    lib = binding.load_library()
+    assert lib.spts_topk_select(None, None, 4, 2, 0, None) == 1        # SPTS_ERR_INVALID_ARG
+    assert lib.spts_launch_count(None) == 0
+
+
+def test_product_schedule_matches_budget_rule():
+    from paper_2601_13155_b200 import schedule, synth
+    w = synth.workload("cfg3")
+    plan = schedule.workload_plan(w)
+    assert [plan[l] for l in (0, 7, 8, 23, 24, 31)] == [
+        (16384, 13108, 0), (16384, 13108, 24576), (16384, 13108, 0), (16384, 13108, 11469),
+        (11469, 11469, 0), (11469, 11469, 0)]
+    w4 = synth.workload("cfg4")
+    p4 = schedule.workload_plan(w4)
+    assert p4[0] == (65536, 52429, 0) and p4[31] == (45875, 45875, 0)
+    # agrees with the oracle's independent statement of the rule
+    from oracle import spts_oracle as O
+    import math
+    op = O.msdp_schedule(32, w.n_tokens, w.stage_first_layer, w.stage_tokens,
+                         math.ceil(w.keep_attn * w.n_tokens), math.ceil(w.keep_ffn * w.n_tokens))
+    assert [(p["m_attn"], p["m_ffn"], p["prune_to"] or 0) for p in op] == plan

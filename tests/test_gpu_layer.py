@@ -1,0 +1,184 @@
+"""GPU parity of the probes, the skip layer, the whole prefill and the decode step against the oracle.
+
+Tolerances: bf16 storage -> max-abs error <= 2e-2 of the output RMS; fp32 verification mode -> 1e-4.
+Index sets must equal the oracle's except for tokens within 1e-3 (relative) of the k-th score."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spts_oracle as O
+from paper_2601_13155_b200 import synth, schedule
+from parity_utils import TOL, check_index_set, dev, host, i32, rel_rms_err, up
+
+pytestmark = pytest.mark.gpu
+
+SMALL_BF16 = replace(synth.LLAMA8B, hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn_dim=1024,
+                     ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
+
+
+def _mk(shape, max_seq, reference=None):
+    from paper_2601_13155_b200 import binding
+    lib = binding.Spts(shape, max_seq=max_seq)
+    if reference is not None:
+        lib.set_reference_kernels(reference)
+    return lib
+
+
+def _layer_case(shape, n, seed, heavy, std=0.02):
+    from paper_2601_13155_b200 import binding
+    W = synth.layer_weights(shape, seed, 0, std=std)
+    X, _ = synth.hidden_states(shape, n, seed, heavy=heavy)
+    return W, X, binding.LayerWeights(W, shape.dtype)
+
+
+def _modes():
+    # (shape, N, m_attn, m_ffn, reference kernels)
+    return [
+        pytest.param(synth.TINY, 512, 256, 256, None, id="cfg1-fp32"),
+        pytest.param(synth.TINY, 389, 100, 57, None, id="tiny-fp32-ragged"),
+        pytest.param(replace(synth.TINY, dtype="bf16"), 512, 256, 256, True, id="cfg1-bf16-refkernels"),
+        pytest.param(SMALL_BF16, 777, 300, 211, True, id="small8b-bf16-refkernels"),
+        pytest.param(SMALL_BF16, 777, 300, 211, False, id="small8b-bf16-tensorcore"),
+        pytest.param(SMALL_BF16, 1024, 1024, 1024, False, id="small8b-bf16-tensorcore-dense"),
+        pytest.param(SMALL_BF16, 640, 640, 200, False, id="small8b-bf16-tensorcore-attn-dense"),
+    ]
+
+
+@pytest.mark.parametrize("shape,N,ma,mf,ref", _modes())
+def test_probes_match_oracle(shape, N, ma, mf, ref):
+    lib = _mk(shape, 2048, ref)
+    W, X, Wd = _layer_case(shape, N, 1001, 32, std=0.05)
+    pos = (np.arange(N) * 2 + 5).astype(np.int32)
+    tol = TOL[shape.dtype]
+    Xd = up(X, shape.dtype)
+    Kd = torch.empty(N, shape.n_kv_heads, shape.head_dim, dtype=lib.dtype, device=dev())
+    S = lib.pap_score(Wd, Xd, i32(pos), K_out=Kd)
+    A = O.rmsnorm(X, np.ones(shape.hidden), shape.rms_eps)
+    Ko, qo, So = O.pap_score(A, pos, W["wk"].astype(np.float64), W["wq"].astype(np.float64), shape)
+    assert rel_rms_err(host(Kd), Ko) <= tol
+    assert np.abs(host(S) - So).max() <= 2e-4 * So.max()
+    assert abs(host(S).sum() - 1.0) < 1e-4
+    # LTP on the same rows
+    Cd = torch.empty(N, dtype=torch.float32, device=dev())
+    Sf = lib.ltp_score(Wd, Xd, S, C_out=Cd)
+    Co, Sfo = O.ltp_score(A, So, {k: v.astype(np.float64) for k, v in W.items()}, O.rounding("bf16" if shape.dtype == "bf16" else "exact"))
+    ctol = 2e-3 if shape.dtype == "bf16" else 1e-4
+    assert np.abs(host(Cd) - Co).max() <= ctol * Co.max()
+    assert np.abs(host(Sf) - Sfo).max() <= ctol * Sfo.max()
+    assert lib.device_status() == 0
+    lib.close()
+
+
+@pytest.mark.parametrize("shape,N,ma,mf,ref", _modes())
+def test_layer_matches_oracle(shape, N, ma, mf, ref):
+    from paper_2601_13155_b200 import binding
+    lib = _mk(shape, 2048, ref)
+    W, X, Wd = _layer_case(shape, N, 1001, 32)
+    pos = np.arange(N, dtype=np.int32)
+    mode = "bf16" if shape.dtype == "bf16" else "exact"
+    want = O.layer_prefill_skip(X, pos, W, shape, ma, mf, mode=mode)
+    Xd = up(X, shape.dtype)
+    X0 = Xd.clone()
+    cache = binding.KvCache(shape, 1, N)
+    S = torch.empty(N, dtype=torch.float32, device=dev())
+    ia = torch.empty(ma, dtype=torch.int32, device=dev())
+    jf = torch.empty(mf, dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip(Wd, Xd, i32(pos), ma, mf, cache, S_out=S, idx_attn_out=ia, idx_ffn_out=jf)
+    assert lib.device_status() == 0
+    tol = TOL[shape.dtype]
+    assert np.abs(host(S) - want["S_mha"]).max() <= 2e-4 * want["S_mha"].max()
+    swaps_a = check_index_set(ia.cpu().numpy(), want["S_mha"], ma)
+    swaps_f = check_index_set(jf.cpu().numpy(), want["S_ffn"], mf)
+    got = host(Xd)
+    # rows outside both sets are bit-identical (Eq. 2)
+    touched = np.union1d(ia.cpu().numpy(), jf.cpu().numpy())
+    rest = np.setdiff1d(np.arange(N), touched)
+    assert torch.equal(Xd[torch.from_numpy(rest).to(dev())], X0[torch.from_numpy(rest).to(dev())])
+    if swaps_a == 0 and swaps_f == 0:
+        assert rel_rms_err(got, want["X"]) <= tol
+        assert cache.length(0) == ma
+        assert rel_rms_err(host(cache.k[0][:ma]), want["K"]) <= tol
+        assert rel_rms_err(host(cache.v[0][:ma]), want["V"]) <= tol
+        assert np.array_equal(cache.pos[0][:ma].cpu().numpy(), want["cache_pos"])
+    else:       # boundary tokens swapped inside the allowed band: compare the rows both sides updated alike
+        same = np.setdiff1d(np.arange(N), np.setxor1d(ia.cpu().numpy(), want["idx_attn"]))
+        same = np.setdiff1d(same, np.setxor1d(jf.cpu().numpy(), want["idx_ffn"]))
+        assert rel_rms_err(got[same], want["X"][same]) <= 5 * tol
+    lib.close()
+
+
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", True), ("bf16", False)])
+def test_keep_all_equals_dense_and_is_deterministic(dtype, ref):
+    from paper_2601_13155_b200 import binding
+    shape = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    lib = _mk(shape, 1024, ref)
+    N = 300
+    W, X, Wd = _layer_case(shape, N, 5, 8)
+    pos = i32(np.arange(N))
+    outs = []
+    for _ in range(2):
+        Xd = up(X, shape.dtype)
+        cache = binding.KvCache(shape, 1, N)
+        lib.layer_prefill_skip(Wd, Xd, pos, N, N, cache)
+        outs.append(Xd)
+    assert torch.equal(outs[0], outs[1])
+    want = O.layer_dense(X, np.arange(N), W, shape, mode="bf16" if dtype == "bf16" else "exact")
+    assert rel_rms_err(host(outs[0]), want["X"]) <= TOL[dtype]
+    assert lib.device_status() == 0
+    lib.close()
+
+
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", True), ("bf16", False)])
+def test_prefill_and_decode_match_oracle(dtype, ref):
+    from paper_2601_13155_b200 import binding
+    base = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    L = 4
+    shape = replace(base, n_layers=L, vocab=1000)
+    lib = _mk(shape, 1024, ref)
+    N = 384
+    layers = [synth.layer_weights(shape, 1010, l, std=0.03) for l in range(L)]
+    hw = synth.head_weights(shape, 1010)
+    X, _ = synth.hidden_states(shape, N, 1010, heavy=24)
+    plan = schedule.stage_plan(L, N, (0, 2), (N, 288), 192, 150)
+    oplan = O.msdp_schedule(L, N, (0, 2), (N, 288), 192, 150)
+    mode = "bf16" if dtype == "bf16" else "exact"
+    want = O.model_prefill(X, layers, shape, oplan, mode=mode)
+    model = binding.Model([binding.LayerWeights(w, dtype) for w in layers], up(hw["lm_head"], dtype), up(hw["embed"], dtype))
+    cache = binding.KvCache(shape, L, [p[0] + 4 for p in plan])
+    Xd, Xa = up(X, dtype), torch.empty(N, shape.hidden, dtype=lib.dtype, device=dev())
+    pos, orig = i32(np.arange(N)), i32(np.arange(N))
+    pa, oa = torch.empty_like(pos), torch.empty_like(orig)
+    tok = torch.zeros(1, dtype=torch.int32, device=dev())
+    nf, in_alt = lib.prefill(model, plan, Xd, pos, orig, Xa, pa, oa, cache, token_out=tok)
+    assert lib.device_status() == 0
+    assert nf == want["X"].shape[0] == 288 and in_alt
+    Xf, of = (Xa, oa) if in_alt else (Xd, orig)
+    got_orig = of[:nf].cpu().numpy()
+    tol = TOL[dtype]
+    if np.array_equal(got_orig, want["orig"]):
+        assert rel_rms_err(host(Xf[:nf]), want["X"]) <= 3 * tol
+        lg, tk = O.first_token(want["X"][-1], np.ones(shape.hidden), hw["lm_head"], shape.rms_eps)
+        top2 = np.sort(lg)[-2:]
+        if top2[1] - top2[0] > 10 * tol * np.abs(lg).max():
+            assert int(tok.item()) == tk
+    else:   # a boundary token swapped at the prune: the surviving common rows still agree
+        check_index_set(got_orig, want["trace"][1]["S_mha"], 288)
+    for l in range(L):
+        assert cache.length(l) == len(want["caches"][l]["pos"])
+    # ---- decode two steps against the compressed caches, oracle side by side
+    if np.array_equal(got_orig, want["orig"]) and all(
+            np.array_equal(cache.pos[l][:cache.length(l)].cpu().numpy(), want["caches"][l]["pos"]) for l in range(L)):
+        emb = hw["embed"]
+        for step, token in enumerate((17, 523)):
+            xo = torch.empty(shape.hidden, dtype=lib.dtype, device=dev())
+            lgd = torch.empty(shape.vocab, dtype=torch.float32, device=dev())
+            lib.decode_step(model, cache, N + step, token_in=token, x_out=xo, logits_out=lgd, token_out=tok)
+            x, lg, tk = O.decode_step(emb[token], N + step, layers, shape, want["caches"], np.ones(shape.hidden),
+                                      hw["lm_head"], mode=mode)
+            assert rel_rms_err(host(xo), x) <= 3 * tol
+            assert rel_rms_err(host(lgd), lg) <= 3 * tol
+        assert all(cache.length(l) == len(want["caches"][l]["pos"]) for l in range(L))
+    assert lib.device_status() == 0
+    lib.close()
