@@ -137,12 +137,13 @@ __global__ void pap_mean_kernel(const float* __restrict__ logits, int ld, int N,
 }
 
 // C[n] = sqrt(sum_p csq[n, p]);  S_ffn[n] = C[n] * S_mha[n]      (Eq. 13-14)
-__global__ void ffn_score_kernel(const float* __restrict__ csq, int parts, const float* __restrict__ S_mha,
-                                 int N, float* __restrict__ C_out, float* __restrict__ S_ffn) {
+__global__ void ffn_score_kernel(const float* __restrict__ csq, int stride, int parts,
+                                 const float* __restrict__ S_mha, int N, float* __restrict__ C_out,
+                                 float* __restrict__ S_ffn) {
   int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= N) return;
   float s = 0.f;
-  for (int p = 0; p < parts; ++p) s += csq[(size_t)n * parts + p];
+  for (int p = 0; p < parts; ++p) s += csq[(size_t)n * stride + p];
   float c = sqrtf(s);
   if (C_out) C_out[n] = c;
   S_ffn[n] = c * S_mha[n];
@@ -284,7 +285,7 @@ spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits
 
 spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
                              float* C_out, float* S_ffn) {
-  ffn_score_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(csq, parts, S_mha, N, C_out, S_ffn);
+  ffn_score_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(csq, ctx->ws.csq_parts, parts, S_mha, N, C_out, S_ffn);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

@@ -1,0 +1,455 @@
+// bf16 GEMM on the 5th-generation tensor cores with the SPTS epilogues fused in:
+//
+//   acc[i, j] = sum_k A[src(i), k] * W[j, k]          A rows optionally gathered by an index list
+//
+// Persistent, warp-specialised CTA (one per SM):
+//   warp 0      TMA producer: A tile by a tiled load, or -- for the gathered rows of the reduced
+//               attention / FFN blocks (Algorithm 1, X^ = X[T_active, :]) -- by 32 tile::gather4
+//               loads, one per lane, straight into the 128B-swizzled operand layout; W tile(s) tiled
+//   warp 1      TMEM allocation and the single-thread tcgen05.mma issue loop
+//   warps 2-5   epilogue: tcgen05.ld of the fp32 accumulator (each warp its lane quarter, one
+//               row per thread), then one of
+//                 TC_STORE   out = bf16(acc * rstd[row])            (+ transposed copy for V)
+//                 TC_ROPE    rotary embedding on 128-wide heads; optional PAP logits q_h . k
+//                            from the unrounded keys (Eq. 4)
+//                 TC_SWIGLU  tile = 128 gate | 128 up columns; out = bf16(silu(g) * u)   (Eq. 6)
+//                 TC_RESID   X[dst(i), :] += acc, in place (Eq. 2 residual scatter)
+//                 TC_SUMSQ   per-row sum of squares of the tile (Eq. 13), no matrix written
+// Accumulators are double-buffered in TMEM so the epilogue of tile t overlaps the MMAs of t+1.
+#include "spts_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace spts {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;
+constexpr int BK = 64;                        // 64 bf16 = one 128-byte swizzle row
+constexpr int A_STAGE_BYTES = BM * BK * 2;    // 16 KiB
+constexpr int GEMM_THREADS = 192;
+constexpr int GROUP_M = 8;
+
+template <int BN> struct Cfg {
+  static constexpr int B_STAGE_BYTES = BN * BK * 2;
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 + 256;
+  static constexpr int TMEM_COLS = 2 * BN;
+};
+
+struct TcParams {
+  const int32_t* idx;
+  const int32_t* dst_idx;
+  int M, Nout, K, a_rows;
+  const float* rowscale;
+  bf16* out; int ldo;
+  bf16* out_t; int ldt;
+  const float2* cs;             // rotary table [rows, 64]
+  const float* q; float* logits; int ld_logits; int group;
+  float* csq; int csq_parts;
+  int* status;
+  int num_m, num_n;
+};
+
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mb, int& nb) {
+  const int per_group = GROUP_M * num_n;
+  const int g = t / per_group;
+  const int rem = t - g * per_group;
+  const int gm = min(GROUP_M, num_m - g * GROUP_M);
+  mb = g * GROUP_M + rem % gm;
+  nb = rem / gm;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void unpack_bf16(uint32_t w, float& a, float& b) {
+  a = __uint_as_float(w << 16);
+  b = __uint_as_float(w & 0xFFFF0000u);
+}
+
+// 32 fp32 values -> 32 bf16 stored to p (64 bytes, 16-byte aligned), columns [c0, c0+32) clipped to ncols
+__device__ __forceinline__ void store32_bf16(bf16* p, const float* v, int c0, int ncols) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    if (c0 + g * 8 < ncols) {
+      uint4 w;
+      w.x = pack_bf16(v[g * 8 + 0], v[g * 8 + 1]);
+      w.y = pack_bf16(v[g * 8 + 2], v[g * 8 + 3]);
+      w.z = pack_bf16(v[g * 8 + 4], v[g * 8 + 5]);
+      w.w = pack_bf16(v[g * 8 + 6], v[g * 8 + 7]);
+      *reinterpret_cast<uint4*>(p + g * 8) = w;
+    }
+  }
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
+  using C = Cfg<BN>;
+  constexpr int STAGES = C::STAGES;
+  constexpr int NT = (EPI == TC_SWIGLU) ? BN / 2 : BN;   // output columns per tile
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sA = base;
+  const uint32_t sB = base + STAGES * A_STAGE_BYTES;
+  const uint32_t bars = sB + STAGES * C::B_STAGE_BYTES;          // 8-byte aligned barrier block
+  const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
+  const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 16;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + STAGES * (A_STAGE_BYTES + C::B_STAGE_BYTES) + 16 * STAGES + 32);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint64_t t0 = globaltimer_ns();
+  const int total_tiles = p.num_m * p.num_n;
+  const int kblocks = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + 8 * b, 1); mbar_init(tempty_bar + 8 * b, 4); }
+    fence_mbar_init();
+    prefetch_tensormap(&tmA);
+    prefetch_tensormap(&tmB);
+    if (EPI == TC_SWIGLU) prefetch_tensormap(&tmB2);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), C::TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    int stage = 0; uint32_t phase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      int mb, nb;
+      tile_coords(t, p.num_m, p.num_n, mb, nb);
+      const int m0 = mb * BM, n0 = nb * NT;
+      int r[4] = {0, 0, 0, 0};
+      if (p.idx != nullptr) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          int gi = m0 + lane * 4 + e;
+          r[e] = gi < p.M ? p.idx[gi] : 0;       // rows past the end load row 0 and are masked later
+        }
+      }
+      for (int kb = 0; kb < kblocks; ++kb) {
+        if (lane == 0) {
+          ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag, t0);
+          if (ok) mbar_expect_tx(full_bar + 8 * stage, A_STAGE_BYTES + C::B_STAGE_BYTES);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        const int k0 = kb * BK;
+        const uint32_t a_dst = sA + stage * A_STAGE_BYTES, b_dst = sB + stage * C::B_STAGE_BYTES;
+        if (p.idx != nullptr) {
+          tma_gather4(a_dst + lane * 512, &tmA, full_bar + 8 * stage, k0, r[0], r[1], r[2], r[3]);
+        } else if (lane == 0) {
+          tma_load_2d(a_dst, &tmA, full_bar + 8 * stage, k0, m0);
+        }
+        if (lane == 0) {
+          tma_load_2d(b_dst, &tmB, full_bar + 8 * stage, k0, n0);
+          if (EPI == TC_SWIGLU) tma_load_2d(b_dst + (BN / 2) * BK * 2, &tmB2, full_bar + 8 * stage, k0, n0);
+        }
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BM, BN);
+      int stage = 0; uint32_t phase = 0;
+      int abuf = 0; uint32_t aphase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        ok = mbar_wait(tempty_bar + 8 * abuf, aphase ^ 1, abort_flag, t0);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + abuf * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, t0);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_addr = sA + stage * A_STAGE_BYTES, b_addr = sB + stage * C::B_STAGE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            mma_bf16(d_tmem, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32), idesc,
+                     (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          mma_commit(empty_bar + 8 * stage);          // frees the smem stage when these MMAs finish
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        mma_commit(tfull_bar + 8 * abuf);             // accumulator complete
+        if (++abuf == 2) { abuf = 0; aphase ^= 1; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;
+    const int row_in_tile = quarter * 32 + lane;
+    int abuf = 0; uint32_t aphase = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+      int mb, nb;
+      tile_coords(t, p.num_m, p.num_n, mb, nb);
+      const int grow = mb * BM + row_in_tile;
+      const int n0 = nb * NT;
+      const bool row_ok = grow < p.M;
+      int src = 0;
+      float rs = 1.0f;
+      if (row_ok) {
+        src = p.idx ? p.idx[grow] : grow;
+        if (p.rowscale) rs = p.rowscale[src];
+      }
+      ok = mbar_wait(tfull_bar + 8 * abuf, aphase, abort_flag, t0);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + abuf * BN + ((uint32_t)(quarter * 32) << 16);
+
+      if (EPI == TC_STORE) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tacc + c, r);
+          tmem_ld_wait();
+          if (row_ok && n0 + c < p.Nout) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * rs;
+            store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
+            if (p.out_t != nullptr) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n0 + c + i < p.Nout) p.out_t[(size_t)(n0 + c + i) * p.ldt + grow] = __float2bfloat16_rn(v[i]);
+            }
+          }
+        }
+      } else if (EPI == TC_ROPE) {
+        const float inv_sqrt_d = 0.08838834764831845f;   // 1 / sqrt(128)
+#pragma unroll 1
+        for (int hh = 0; hh < BN / 128; ++hh) {
+          const int hcol = n0 + hh * 128;               // first column of this head
+          float dots[8];
+#pragma unroll
+          for (int g = 0; g < 8; ++g) dots[g] = 0.f;
+#pragma unroll 1
+          for (int jj = 0; jj < 2; ++jj) {
+            uint32_t lo[32], hi[32];
+            tmem_ld32(tacc + hh * 128 + jj * 32, lo);
+            tmem_ld32(tacc + hh * 128 + 64 + jj * 32, hi);
+            tmem_ld_wait();
+            if (row_ok && hcol < p.Nout) {
+              float a[32], b[32];
+              const float4* cs4 = reinterpret_cast<const float4*>(p.cs + (size_t)src * 64 + jj * 32);
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                float4 c2 = cs4[i >> 1];                 // (cos, sin) of two consecutive frequencies
+                float x0 = __uint_as_float(lo[i]) * rs, y0 = __uint_as_float(hi[i]) * rs;
+                float x1 = __uint_as_float(lo[i + 1]) * rs, y1 = __uint_as_float(hi[i + 1]) * rs;
+                a[i] = x0 * c2.x - y0 * c2.y;
+                b[i] = y0 * c2.x + x0 * c2.y;
+                a[i + 1] = x1 * c2.z - y1 * c2.w;
+                b[i + 1] = y1 * c2.z + x1 * c2.w;
+              }
+              bf16* o = p.out + (size_t)grow * p.ldo + hcol + jj * 32;
+              store32_bf16(o, a, 0, 32);
+              store32_bf16(o + 64, b, 0, 32);
+              if (p.logits != nullptr) {
+                const int kvh = hcol >> 7;
+                for (int g = 0; g < p.group && g < 8; ++g) {
+                  const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
+                  float d = dots[g];
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
+                  dots[g] = d;
+                }
+              }
+            }
+          }
+          if (p.logits != nullptr && row_ok && hcol < p.Nout) {
+            const int kvh = hcol >> 7;
+            for (int g = 0; g < p.group && g < 8; ++g)
+              p.logits[(size_t)(kvh * p.group + g) * p.ld_logits + grow] = dots[g] * inv_sqrt_d;
+          }
+        }
+      } else if (EPI == TC_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 2; c += 32) {
+          uint32_t g[32], u[32];
+          tmem_ld32(tacc + c, g);
+          tmem_ld32(tacc + BN / 2 + c, u);
+          tmem_ld_wait();
+          if (row_ok && n0 + c < p.Nout) {
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              float a = __uint_as_float(g[i]) * rs, b = __uint_as_float(u[i]) * rs;
+              v[i] = a / (1.0f + expf(-a)) * b;
+            }
+            store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
+          }
+        }
+      } else if (EPI == TC_RESID) {
+        int dst = grow;
+        if (row_ok && p.dst_idx) dst = p.dst_idx[grow];
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tacc + c, r);
+          tmem_ld_wait();
+          if (row_ok && n0 + c < p.Nout) {
+            bf16* xp = p.out + (size_t)dst * p.ldo + n0 + c;
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (n0 + c + g * 8 < p.Nout) {
+                uint4 w = *reinterpret_cast<const uint4*>(xp + g * 8);
+                uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  float x0, x1;
+                  unpack_bf16(ww[e], x0, x1);
+                  ww[e] = pack_bf16(x0 + __uint_as_float(r[g * 8 + 2 * e]), x1 + __uint_as_float(r[g * 8 + 2 * e + 1]));
+                }
+                *reinterpret_cast<uint4*>(xp + g * 8) = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+              }
+            }
+          }
+        }
+      } else {   // TC_SUMSQ
+        float s = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tacc + c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float v = __uint_as_float(r[i]);
+            if (n0 + c + i < p.Nout) s = fmaf(v, v, s);
+          }
+        }
+        if (row_ok) p.csq[(size_t)grow * p.csq_parts + nb] = s;
+      }
+      // accumulator buffer drained: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * abuf);
+      if (++abuf == 2) { abuf = 0; aphase ^= 1; }
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // a wait ran out: give copies still in flight time to land before shared memory is released
+    if (threadIdx.x == 0) set_status(p.status, SPTS_ERR_TIMEOUT);
+    const uint64_t t1 = globaltimer_ns();
+    while (globaltimer_ns() - t1 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, C::TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor [rows, cols] with row stride ld (elements), box [box_rows, 64 cols], 128B swizzle.
+bool make_map(spts_ctx* ctx, CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+              uint32_t box_rows) {
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {ld * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
+  constexpr int NT = (EPI == TC_SWIGLU) ? BN / 2 : BN;
+  TcParams p;
+  p.idx = a.idx; p.dst_idx = a.dst_idx; p.M = a.M; p.Nout = a.Nout; p.K = a.K; p.a_rows = a.a_rows;
+  p.rowscale = a.rowscale; p.out = a.out; p.ldo = a.ldo; p.out_t = a.out_t; p.ldt = a.ldt;
+  p.cs = ctx->ws.rope_cs; p.q = a.q; p.logits = a.logits; p.ld_logits = a.ld_logits; p.group = a.group;
+  p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
+  p.num_m = ceil_div(a.M, BM);
+  p.num_n = ceil_div(a.Nout, NT);
+  if (EPI == TC_SUMSQ && p.num_n > a.csq_parts) return SPTS_ERR_WORKSPACE;
+  CUtensorMap tmA, tmB, tmB2;
+  if (!make_map(ctx, &tmA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, (uint64_t)a.lda, a.idx ? 1u : (uint32_t)BM))
+    return SPTS_ERR_CUDA;
+  if (!make_map(ctx, &tmB, a.W, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
+  if (EPI == TC_SWIGLU) {
+    if (!make_map(ctx, &tmB2, a.W2, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
+  } else {
+    tmB2 = tmB;
+  }
+  const int tiles = p.num_m * p.num_n;
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  tc_gemm_kernel<BN, EPI><<<grid, GEMM_THREADS, Cfg<BN>::SMEM_BYTES, ctx->stream>>>(tmA, tmB, tmB2, p);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+template <int BN, int EPI>
+bool set_smem_attr() {
+  return cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+}
+
+}  // namespace
+
+int tc_sumsq_parts(int n_out) { return ceil_div(n_out, 256); }
+
+spts_status tc_gemm_init(spts_ctx* ctx) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || fn == nullptr)
+    return SPTS_ERR_CUDA;
+  ctx->encode_tiled = fn;
+  bool ok = set_smem_attr<256, TC_STORE>() && set_smem_attr<256, TC_ROPE>() && set_smem_attr<256, TC_SWIGLU>() &&
+            set_smem_attr<256, TC_RESID>() && set_smem_attr<256, TC_SUMSQ>() && set_smem_attr<128, TC_STORE>() &&
+            set_smem_attr<128, TC_ROPE>() && set_smem_attr<128, TC_SWIGLU>();
+  return ok ? SPTS_OK : SPTS_ERR_CUDA;
+}
+
+spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a) {
+  if (a.M <= 0) return SPTS_OK;
+  if (ctx->encode_tiled == nullptr) return SPTS_ERR_UNSUPPORTED;
+  if ((a.K % 8) || (a.lda % 8) || (reinterpret_cast<uintptr_t>(a.A) & 15) || (reinterpret_cast<uintptr_t>(a.W) & 15))
+    return SPTS_ERR_SHAPE;
+  if (a.out != nullptr && ((a.ldo % 8) || (reinterpret_cast<uintptr_t>(a.out) & 15))) return SPTS_ERR_SHAPE;
+  if (a.Nout % 8) return SPTS_ERR_SHAPE;
+  const bool narrow = a.Nout <= 128;       // a 128-wide tile wastes less on the skinny proxy factors
+  switch (epi) {
+    case TC_STORE: return narrow ? launch_one<128, TC_STORE>(ctx, a) : launch_one<256, TC_STORE>(ctx, a);
+    case TC_ROPE:
+      if (a.Nout % 128) return SPTS_ERR_SHAPE;
+      return narrow ? launch_one<128, TC_ROPE>(ctx, a) : launch_one<256, TC_ROPE>(ctx, a);
+    case TC_SWIGLU: return (a.Nout <= 64) ? launch_one<128, TC_SWIGLU>(ctx, a) : launch_one<256, TC_SWIGLU>(ctx, a);
+    case TC_RESID: return launch_one<256, TC_RESID>(ctx, a);
+    case TC_SUMSQ: return launch_one<256, TC_SUMSQ>(ctx, a);
+    default: return SPTS_ERR_INVALID_ARG;
+  }
+}
+
+}  // namespace spts

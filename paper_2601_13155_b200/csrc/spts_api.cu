@@ -320,7 +320,7 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   g.W = w->wv; g.Nout = KD; g.out = cache->v; g.ldo = KD;
   if (tc) { g.out_t = ws.v_t; g.ldt = ldvt; }
   TRY(run_gemm(ctx, REF_STORE, g));
-  if (tc) TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)ws.v_t, ldvt, m_attn,
+  if (tc) TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)cache->v, (const bf16*)ws.v_t, ldvt, m_attn,
                                   (bf16*)ws.o_att));
   else TRY(launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att));
   memset(&g, 0, sizeof(g));

@@ -164,7 +164,7 @@ struct TcGemmArgs {
   float* csq; int csq_parts;
 };
 spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
-spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* Vt, int ldvt,
+spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,
                                 int m, bf16* O);
 spts_status tc_init(spts_ctx* ctx);          // resolves the tensor-map encoder, sets kernel attributes
 int tc_sumsq_parts(int n_out);               // partial sums per row written by TC_SUMSQ
