@@ -76,3 +76,66 @@ def check_output(got, want, dtype, scale=1.0):
     assert not bad.any(), f"max-abs error {err[bad].max() / rms:.3e} of RMS exceeds {tol:.1e} (beyond one bf16 ulp)"
     assert flips.sum() <= max(1, 1e-3 * want.size), f"{int(flips.sum())} one-ulp disagreements"
     return float(err[~over].max() / rms) if (~over).any() else 0.0
+
+
+def zero_down(W):
+    """Same layer with W_down = 0: the FFN block becomes a no-op, exposing the residual after attention."""
+    Wz = dict(W)
+    Wz["w_down"] = np.zeros_like(W["w_down"])
+    return Wz
+
+
+def check_layer_blocks(lib, shape, W, lw, lw_mid, Xd, pos_t, ma, mf, cache, layer=0):
+    """Runs spts_layer_prefill_skip on Xd (in place) and checks it against the oracle block by block.
+
+    The attention block is compared on the layer's input.  The FFN block's decision (T_f) and
+    update are compared on the GPU's own post-attention residual (obtained by a second run with
+    W_down = 0), because a single one-ulp bf16 disagreement in that residual moves the LTP score of
+    its token by more than the 1e-3 band.  Returns the outputs of the real run."""
+    import torch
+    from paper_2601_13155_b200 import binding
+    dtype = shape.dtype
+    mode = "bf16" if dtype == "bf16" else "exact"
+    n = Xd.shape[0]
+    x_in, pos_in = host(Xd), pos_t.cpu().numpy()
+    X0 = Xd.clone()
+    # GPU: attention block only
+    Xmid = Xd.clone()
+    scratch = binding.KvCache(shape, 1, n)
+    lib.layer_prefill_skip(lw_mid, Xmid, pos_t, ma, n, scratch)
+    # GPU: the real layer
+    S = torch.empty(n, dtype=torch.float32, device=dev())
+    ia = torch.empty(ma, dtype=torch.int32, device=dev())
+    jf = torch.empty(mf, dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip(lw, Xd, pos_t, ma, mf, cache, layer=layer, S_out=S, idx_attn_out=ia, idx_ffn_out=jf)
+    assert lib.device_status() == 0
+    ia_h, jf_h = ia.cpu().numpy(), jf.cpu().numpy()
+    # oracle: attention block from the layer input
+    wa = O.layer_prefill_skip(x_in, pos_in, zero_down(W), shape, ma, n, mode=mode)
+    assert np.abs(host(S) - wa["S_mha"]).max() <= 2e-4 * wa["S_mha"].max()
+    swaps_a = check_index_set(ia_h, wa["S_mha"], ma)
+    same = np.setdiff1d(np.arange(n), np.setxor1d(ia_h, wa["idx_attn"]))
+    check_output(host(Xmid)[same], wa["X"][same], dtype)
+    assert cache.length(layer) == ma
+    assert np.array_equal(cache.pos[layer][:ma].cpu().numpy(), pos_in[ia_h])
+    if swaps_a == 0:
+        check_output(host(cache.k[layer][:ma]), wa["K"], dtype)
+        check_output(host(cache.v[layer][:ma]), wa["V"], dtype)
+    # oracle: FFN block from the GPU's post-attention residual and the oracle's S_mha
+    rnd = O.rounding(mode)
+    W64 = {k: np.asarray(v, np.float64) for k, v in W.items()}
+    xm = host(Xmid)
+    B = O.rmsnorm(xm, np.ones(shape.hidden), shape.rms_eps)
+    Cw, Sf = O.ltp_score(B, wa["S_mha"], W64, rnd)
+    swaps_f = check_index_set(jf_h, Sf, mf)
+    Tf = O.topk_select(Sf, mf, True)
+    xo = xm.copy()
+    xo[Tf] = rnd(xo[Tf] + O.ffn(B[Tf], W64["w_gate"], W64["w_up"], W64["w_down"], rnd))
+    samef = np.setdiff1d(np.arange(n), np.setxor1d(jf_h, Tf))
+    check_output(host(Xd)[samef], xo[samef], dtype)
+    # Eq. 2: rows outside both sets are bit-identical to the input
+    rest = np.setdiff1d(np.arange(n), np.union1d(ia_h, jf_h))
+    if len(rest):
+        r = torch.from_numpy(rest).to(dev())
+        assert torch.equal(Xd[r], X0[r])
+    return {"S": S, "idx_attn": ia, "idx_ffn": jf, "swaps": swaps_a + swaps_f}
