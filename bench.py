@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the SPTS prefill path on B200.
+
+One step = one whole prefill of the 32-layer LLaMA-3.1-8B-shaped model (random-init weights,
+synthetic hidden states with heavy tokens) through Algorithm 1: per layer PAP score, top-k,
+reduced attention, LTP score, top-k, reduced FFN; stage-end pruning; first-token head.
+The default workload is BASELINE config 3 (32768-token prompt, four MSDP stages).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` = prompt tokens / second over all replicas with inputs
+resident in HBM; `e2e` = the same through host buffers (pinned H2D of the prompt's hidden states,
+D2H of the first token) every step; `dense` = the same code with skipping disabled.
+More than one GPU = independent replicas (the path has no inter-GPU exchange).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="spts", choices=["spts", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
+    ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--breakdown", action="store_true", help="also print a per-operation table to stderr")
+    return ap.parse_args()
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "hw_thermal_slowdown": 0x40,
+                 "sw_thermal_slowdown": 0x20, "hw_power_brake": 0x80, "sync_boost": 0x10}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for n, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(0.05)
+
+    def start(self):
+        if self.nv is not None:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._t is not None:
+            self._t.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------
+# CPU oracle leg (bounded sample)
+# --------------------------------------------------------------------------------------------
+def oracle_sample(w, seconds_hint=20.0):
+    """One skip layer of the workload's shape on a shortened prompt, on the host cores.
+    Returns (tokens_per_s extrapolated to the full depth, cores, description, seconds)."""
+    from oracle import spts_oracle as O
+    from paper_2601_13155_b200 import synth
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    n = 1024
+    shape = w.shape
+    W = synth.layer_weights(shape, w.seed, 0)
+    X, _ = synth.hidden_states(shape, n, w.seed, heavy=max(1, n // 100))
+    ma, mf = math.ceil(w.keep_attn * n), math.ceil(w.keep_ffn * n)
+    t = time.perf_counter()
+    O.layer_prefill_skip(X, np.arange(n), W, shape, ma, mf, mode="bf16" if shape.dtype == "bf16" else "exact")
+    dt = time.perf_counter() - t
+    layers = shape.n_layers
+    tps = n / (dt * layers)
+    desc = (f"one SPTS layer of the {shape.hidden}-wide model on a {n}-token prompt (keep {w.keep_attn}/{w.keep_ffn}), "
+            f"fp64 numpy oracle, {dt:.2f} s; tokens/s = {n} / ({dt:.2f} s x {layers} layers)")
+    return tps, cores, desc, dt
+
+
+def run_reference(args):
+    """--impl reference: the oracle as it stands, timed on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2601_13155_b200 import synth
+    w = synth.workload(args.workload)
+    vals = []
+    for i in range(args.warmup + args.steps):
+        tps, cores, desc, dt = oracle_sample(w)
+        if i >= args.warmup:
+            vals.append((tps, dt))
+        if i == 0 and dt * (args.warmup + args.steps) > 240:      # keep the run within minutes
+            args.warmup, args.steps = 0, max(1, min(args.steps, int(240 / dt)))
+            vals.append((tps, dt))
+            if len(vals) >= args.steps:
+                break
+    tps = float(np.mean([v[0] for v in vals]))
+    ms = float(np.mean([v[1] for v in vals])) * 1e3
+    line = {"impl": "reference", "metric": "prefill_tokens_per_s", "value": tps, "unit": "tokens/s",
+            "n_gpus": args.gpus, "steps": len(vals), "warmup": args.warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload + " (bounded sample)", "sample": desc},
+            "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------
+# the SPTS arm
+# --------------------------------------------------------------------------------------------
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    import torch
+    from paper_2601_13155_b200 import binding, schedule, synth, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    dev = f"cuda:{local}"
+    torch.cuda.set_device(dev)
+    if rank == 0 and not os.path.exists(binding.LIB_PATH):
+        build.build()
+    if dist is not None:
+        dist.barrier()
+
+    w = synth.workload(args.workload)
+    shape = w.shape
+    if args.layers:
+        from dataclasses import replace
+        shape = replace(shape, n_layers=args.layers)
+        w = replace(w, shape=shape, stage_first_layer=tuple(f for f in w.stage_first_layer if f < args.layers),
+                    stage_tokens=w.stage_tokens[:len([f for f in w.stage_first_layer if f < args.layers])])
+    L, N = shape.n_layers, w.n_tokens
+    plan = schedule.workload_plan(w)
+    plan_dense = schedule.workload_plan(w, dense=True)
+
+    # weights and inputs (seeded, drawn on the device)
+    layers = []
+    for l in range(L):
+        t = synth.device_layer_weights(shape, w.seed, l, dev)
+        lw = binding.LayerWeights.__new__(binding.LayerWeights)
+        lw.t = t
+        lw.c = binding.LayerWeightsC(**{n: t[n].data_ptr() for n in binding.WEIGHT_NAMES})
+        layers.append(lw)
+    hw = synth.device_head_weights(shape, w.seed, dev)
+    model = binding.Model(layers, hw["lm_head"], hw["embed"])
+    X0, _ = synth.device_hidden_states(w, dev)
+    X0_host = torch.empty(X0.shape, dtype=X0.dtype, pin_memory=True)
+    X0_host.copy_(X0)
+    lib = binding.Spts(shape, max_seq=N, device=dev)
+    cache = binding.KvCache(shape, L, [N] * L if not args.no_dense else schedule.cache_capacities(plan), dev)
+    X = torch.empty_like(X0)
+    Xa = torch.empty_like(X0)
+    ar = torch.arange(N, dtype=torch.int32, device=dev)
+    pos, orig, pa, oa = ar.clone(), ar.clone(), ar.clone(), ar.clone()
+    tok = torch.zeros(1, dtype=torch.int32, device=dev)
+    tok_host = torch.zeros(1, dtype=torch.int32, pin_memory=True)
+
+    def step(pl, from_host=False):
+        if from_host:
+            X.copy_(X0_host, non_blocking=True)
+        else:
+            X.copy_(X0)
+        pos.copy_(ar)
+        orig.copy_(ar)
+        lib.prefill(model, pl, X, pos, orig, Xa, pa, oa, cache, token_out=tok)
+        if from_host:
+            tok_host.copy_(tok, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(pl, steps, from_host=False, profile_op=0):
+        barrier()
+        if profile_op:
+            lib.profile_begin(profile_op)
+        l0 = lib.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            step(pl, from_host)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        prof = lib.profile_end() if profile_op else {}
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, lib.launch_count() - l0, prof
+
+    for _ in range(max(args.warmup, 3)):
+        step(plan)
+    status = lib.device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} after warm-up")
+
+    # which operation dominates?  one untimed, fully instrumented pass
+    lib.profile_begin(-1)
+    step(plan)
+    table = lib.profile_end()
+    dom = max(table.items(), key=lambda kv: kv[1]["ms"])[0]
+    dom_id = {v: k for k, v in binding.OP_NAMES.items()}[dom]
+
+    clocks = ClockSampler(local)
+    clocks.start()
+    ms, launches, prof = timed(plan, args.steps, profile_op=dom_id)
+    clk = clocks.stop()
+    ms_step = ms / args.steps
+    value = N * world / (ms_step * 1e-3)
+
+    ms_e2e, _, _ = timed(plan, args.steps, from_host=True)
+    e2e = N * world / (ms_e2e / args.steps * 1e-3)
+
+    dense = None
+    if not args.no_dense:
+        for _ in range(2):
+            step(plan_dense)
+        ms_d, _, _ = timed(plan_dense, max(1, args.steps))
+        ms_d /= max(1, args.steps)
+        dense = {"value": N * world / (ms_d * 1e-3), "unit": "tokens/s", "ms_per_step": ms_d,
+                 "ttft_ms": ms_d, "speedup_spts_vs_dense": ms_d / ms_step}
+    status = lib.device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+
+    # roofline of the dominant kernel, from the events recorded inside the timed region
+    peaks = {}
+    pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk_path):
+        peaks = json.load(open(pk_path))
+    d = prof[dom]
+    tensor_ops = {"kproj_pap", "qv_proj", "attention", "o_proj", "ltp", "gate_up", "down"}
+    per_launch_ms = d["ms"] / d["calls"]
+    if dom in tensor_ops:
+        peak = peaks.get("bf16_tflops_sustained", 1400.0)
+        achieved = d["flops"] / d["calls"] / (per_launch_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": None, "kernel": dom, "launches": d["calls"], "ms_per_launch": per_launch_ms,
+                "peak_source": "measured (sustained cuBLAS bf16)" if peaks else "fallback"}
+    else:
+        peak = peaks.get("hbm_gbs", 6650.0)
+        achieved = d["bytes"] / d["calls"] / (per_launch_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "kernel": dom, "launches": d["calls"], "ms_per_launch": per_launch_ms,
+                "peak_source": "measured (copy)" if peaks else "fallback"}
+
+    total_flops = sum(v["flops"] for v in table.values())
+    if rank == 0:
+        tps_cpu, cores, desc, _ = oracle_sample(w)
+        line = {
+            "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ttft_ms": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": {"workload": f"{w.name}: {L}-layer LLaMA-3.1-8B shape, prompt {N}, MSDP stages at layers "
+                                   f"{list(w.stage_first_layer)} with {list(w.stage_tokens)} candidates, keep "
+                                   f"{w.keep_attn}/{w.keep_ffn}, LTP (D_low, r) = ({shape.ltp_dlow}, {shape.ltp_rank})",
+                       "global_batch": world, "seq_len": N, "parallelism": f"replicas x{world}",
+                       "l2": "inputs larger than L2 (14 GB of weights streamed per step)"},
+            "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": int(X0_host.numel() * X0_host.element_size()),
+                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": int(launches),
+            "clocks": clk,
+            "roofline": roof,
+            "cpu_baseline": {"value": tps_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "dense": dense,
+            "algorithmic_tflop_per_step": total_flops / 1e12,
+            "achieved_tflops_whole_step": total_flops / 1e12 / (ms_step * 1e-3),
+            "breakdown_ms": {k: round(v["ms"], 3) for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"])},
+        }
+        if args.breakdown:
+            for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"]):
+                tf = v["flops"] / max(v["ms"], 1e-9) / 1e9
+                gb = v["bytes"] / max(v["ms"], 1e-9) / 1e6
+                sys.stderr.write(f"{k:12s} {v['ms']:9.3f} ms  {v['calls']:4d} calls  {tf:8.1f} TFLOP/s  {gb:8.1f} GB/s\n")
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

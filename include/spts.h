@@ -115,6 +115,25 @@ typedef struct {
   const void* embed;                /* [vocab, D], used by spts_decode_step */
 } spts_model_weights;
 
+/* Operation tags of the per-operation timer (spts_profile_begin / spts_profile_end). */
+enum {
+  SPTS_OP_PREP = 1,        /* row RMS statistics, rotary table, last-token query            */
+  SPTS_OP_KPROJ = 2,       /* K projection of all candidates + RoPE + PAP logits (Eq. 4)   */
+  SPTS_OP_PAP_SOFTMAX = 3, /* head-mean softmax of Eq. 4                                    */
+  SPTS_OP_TOPK = 4,        /* Eq. 5 / 15 / 16                                               */
+  SPTS_OP_KV_GATHER = 5,   /* K^ = K[T_a], cache positions                                  */
+  SPTS_OP_QVPROJ = 6,      /* gathered Q (RoPE) and V projections                           */
+  SPTS_OP_ATTN = 7,        /* causal GQA attention among the active rows                    */
+  SPTS_OP_OPROJ = 8,       /* O projection + residual scatter                               */
+  SPTS_OP_LTP = 9,         /* proxy FFN chain, row norms and score fusion (Eq. 12-14)       */
+  SPTS_OP_GATEUP = 10,     /* gathered gate/up GEMM + SwiGLU                                */
+  SPTS_OP_DOWN = 11,       /* down GEMM + residual scatter                                  */
+  SPTS_OP_COMPACT = 12,    /* stage-end row compaction (Eq. 16)                             */
+  SPTS_OP_HEAD = 13,       /* final norm, LM head, argmax                                   */
+  SPTS_OP_DECODE = 14,     /* all layers of one decode step                                 */
+  SPTS_OP_COUNT = 16
+};
+
 typedef struct spts_ctx spts_ctx;
 
 /* Bytes of device workspace spts_create() needs for sequences of up to max_seq candidates. */
@@ -138,6 +157,14 @@ spts_status spts_last_device_status(spts_ctx* ctx);
 
 /* Number of kernels the library has launched on this context so far. */
 int64_t spts_launch_count(const spts_ctx* ctx);
+
+/* Per-operation timing with CUDA events recorded on the context's stream (the paper has no
+ * counterpart; this is measurement plumbing).  spts_profile_begin starts recording event pairs
+ * around every operation with tag `op` (-1: every tagged operation); spts_profile_end stops,
+ * synchronises the stream and fills four host arrays of SPTS_OP_COUNT entries indexed by tag:
+ * elapsed milliseconds, number of timed operations, algorithmic FLOPs and algorithmic bytes. */
+spts_status spts_profile_begin(spts_ctx* ctx, int op);
+spts_status spts_profile_end(spts_ctx* ctx, float* ms, int64_t* calls, double* flops, double* bytes);
 
 /* W[o, i] *= g[i], in place, rounded to the storage type: folds an RMSNorm gain g [in] into a
  * weight matrix [out, in] that consumes the normalised rows (pre-norm block placement; the

@@ -59,7 +59,11 @@ class ModelWeightsC(C.Structure):
 EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_option",
            "spts_last_device_status", "spts_launch_count", "spts_fold_norm_gain", "spts_pap_score",
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
-           "spts_first_token", "spts_prefill", "spts_decode_step")
+           "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end")
+
+OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
+            8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
+OP_COUNT = 16
 
 
 def load_library() -> C.CDLL:
@@ -89,6 +93,9 @@ def load_library() -> C.CDLL:
                                  i32, u32, C.POINTER(KvLayerC), C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
     lib.spts_decode_step.argtypes = [vp, C.POINTER(ModelWeightsC), C.POINTER(KvLayerC), vp, C.c_int32,
                                      C.c_int32, vp, vp, vp]
+    lib.spts_profile_begin.argtypes = [vp, i32]
+    lib.spts_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64), C.POINTER(C.c_double),
+                                     C.POINTER(C.c_double)]
     for n in EXPORTS:
         if n not in ("spts_workspace_bytes", "spts_destroy", "spts_launch_count"):
             getattr(lib, n).restype = C.c_int
@@ -194,6 +201,19 @@ class Spts:
     def fold_norm_gain(self, W: torch.Tensor, g: torch.Tensor):
         self._check(self.lib.spts_fold_norm_gain(self.h, _ptr(W), _ptr(g), W.shape[0], W.shape[1]),
                     "spts_fold_norm_gain")
+
+    def profile_begin(self, op: int = -1):
+        self._check(self.lib.spts_profile_begin(self.h, op), "spts_profile_begin")
+
+    def profile_end(self):
+        """Returns {op name: {"ms", "calls", "flops", "bytes"}} for the operations timed since profile_begin."""
+        ms = (C.c_float * OP_COUNT)()
+        calls = (C.c_int64 * OP_COUNT)()
+        fl = (C.c_double * OP_COUNT)()
+        by = (C.c_double * OP_COUNT)()
+        self._check(self.lib.spts_profile_end(self.h, ms, calls, fl, by), "spts_profile_end")
+        return {OP_NAMES[i]: {"ms": float(ms[i]), "calls": int(calls[i]), "flops": float(fl[i]), "bytes": float(by[i])}
+                for i in OP_NAMES if calls[i] > 0}
 
     # ------------------------------------------------------------------ the six calls
     def pap_score(self, w: LayerWeights, X, pos, K_out=None, S_out=None):

@@ -3,6 +3,7 @@
 // stream; no call synchronises except spts_last_device_status().
 #include <new>
 #include <cstring>
+#include <vector>
 
 #include "spts_common.cuh"
 
@@ -119,6 +120,40 @@ spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
 
 #define TRY(x) do { spts_status s__ = (x); if (s__ != SPTS_OK) return s__; } while (0)
 
+// ---- optional per-operation timing with CUDA events on the context's stream
+struct ProfRecord { cudaEvent_t a, b; int tag; double flops, bytes; };
+struct Profiler {
+  int filter = 0;                 // 0 off, -1 every operation, else one SPTS_OP_* tag
+  std::vector<ProfRecord> recs;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  cudaEvent_t get() {
+    if (used == pool.size()) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+      pool.push_back(e);
+    }
+    return pool[used++];
+  }
+};
+Profiler* prof_of(spts_ctx* ctx) { return reinterpret_cast<Profiler*>(ctx->prof); }
+
+struct ProfScope {
+  spts_ctx* ctx; ProfRecord r; bool on;
+  ProfScope(spts_ctx* c, int tag, double flops, double bytes) : ctx(c), on(false) {
+    Profiler* p = prof_of(c);
+    if (p == nullptr || p->filter == 0 || (p->filter != -1 && p->filter != tag) || p->recs.size() >= 65536) return;
+    r.a = p->get(); r.b = p->get();
+    if (r.a == nullptr || r.b == nullptr) return;
+    r.tag = tag; r.flops = flops; r.bytes = bytes;
+    on = cudaEventRecord(r.a, c->stream) == cudaSuccess;
+  }
+  ~ProfScope() {
+    if (on && cudaEventRecord(r.b, ctx->stream) == cudaSuccess) prof_of(ctx)->recs.push_back(r);
+  }
+};
+#define OP(tag, flops, bytes, call) do { ProfScope ps__(ctx, tag, flops, bytes); TRY(call); } while (0)
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 // PAP (Eq. 4): rstd, rotary table, q of the last row, K of every row with the logits taken from
@@ -129,16 +164,20 @@ spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   Workspace& ws = ctx->ws;
   const int KD = d.n_kv_heads * d.head_dim;
   const int ld = (int)align_up((size_t)N, 128);
-  TRY(launch_rstd(ctx, X, N, ws.rstd));
-  TRY(launch_rope_table(ctx, pos, N, ws.rope_cs));
-  if (want_scores) TRY(launch_q_last(ctx, X, ws.rope_cs, N, w->wq, ws.rstd, ws.q));
+  const double es = (double)elt_size(d), Nd = (double)N, Dd = (double)d.hidden;
+  OP(SPTS_OP_PREP, 0.0, Nd * Dd * es + 4.0 * Nd, launch_rstd(ctx, X, N, ws.rstd));
+  OP(SPTS_OP_PREP, 0.0, Nd * (4.0 + 4.0 * d.head_dim), launch_rope_table(ctx, pos, N, ws.rope_cs));
+  if (want_scores)
+    OP(SPTS_OP_PREP, 2.0 * Dd * d.n_q_heads * d.head_dim, Dd * d.n_q_heads * d.head_dim * es,
+       launch_q_last(ctx, X, ws.rope_cs, N, w->wq, ws.rstd, ws.q));
   Gemm g;
   memset(&g, 0, sizeof(g));
   g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->wk; g.M = N; g.Nout = KD; g.K = d.hidden;
   g.rowscale = ws.rstd; g.out = K_out; g.ldo = KD;
   if (want_scores) { g.q = ws.q; g.logits = ws.logits; g.ld_logits = ld; }
-  TRY(run_gemm(ctx, REF_ROPE, g));
-  if (want_scores) TRY(launch_pap_softmax(ctx, ws.logits, ld, N, S_out));
+  OP(SPTS_OP_KPROJ, 2.0 * Nd * Dd * KD, (Nd * Dd + Nd * KD + Dd * KD) * es, run_gemm(ctx, REF_ROPE, g));
+  if (want_scores)
+    OP(SPTS_OP_PAP_SOFTMAX, 0.0, Nd * 4.0 * (2.0 * d.n_q_heads + 1.0), launch_pap_softmax(ctx, ws.logits, ld, N, S_out));
   return SPTS_OK;
 }
 
@@ -149,6 +188,9 @@ spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   Workspace& ws = ctx->ws;
   const int r = d.ltp_rank, Dl = d.ltp_dlow;
   const size_t es = elt_size(d);
+  const double Nd = (double)N;
+  ProfScope ps_ltp(ctx, SPTS_OP_LTP, 6.0 * Nd * r * ((double)d.hidden + Dl),
+                   Nd * d.hidden * (double)es + 3.0 * r * ((double)d.hidden + Dl) * (double)es + 8.0 * Nd);
   TRY(launch_pad_proxy(ctx, w->vg, w->vu, ws.vgu_pad));
   Gemm g;
   // t1 = [x Ug | x Uu]  (two column blocks of one [N, 2r] matrix)
@@ -206,6 +248,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->launches = 0;
   ctx->sm_count = prop.multiProcessorCount;
   ctx->encode_tiled = nullptr;
+  ctx->prof = new (std::nothrow) Profiler;
   carve(*desc, max_seq, workspace, &ctx->ws);
   ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
   if (!ctx->reference_kernels) {
@@ -221,7 +264,41 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   return SPTS_OK;
 }
 
-void spts_destroy(spts_ctx* ctx) { delete ctx; }
+void spts_destroy(spts_ctx* ctx) {
+  if (ctx == nullptr) return;
+  if (Profiler* p = prof_of(ctx)) {
+    for (cudaEvent_t e : p->pool) cudaEventDestroy(e);
+    delete p;
+  }
+  delete ctx;
+}
+
+spts_status spts_profile_begin(spts_ctx* ctx, int op) {
+  TRY(check_ctx(ctx));
+  Profiler* p = prof_of(ctx);
+  if (p == nullptr || op < -1 || op >= SPTS_OP_COUNT) return SPTS_ERR_INVALID_ARG;
+  p->filter = op;
+  p->recs.clear();
+  p->used = 0;
+  return SPTS_OK;
+}
+
+spts_status spts_profile_end(spts_ctx* ctx, float* ms, int64_t* calls, double* flops, double* bytes) {
+  TRY(check_ctx(ctx));
+  Profiler* p = prof_of(ctx);
+  if (p == nullptr || ms == nullptr || calls == nullptr || flops == nullptr || bytes == nullptr) return SPTS_ERR_INVALID_ARG;
+  p->filter = 0;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return SPTS_ERR_CUDA;
+  for (int i = 0; i < SPTS_OP_COUNT; ++i) { ms[i] = 0.f; calls[i] = 0; flops[i] = 0.0; bytes[i] = 0.0; }
+  for (const ProfRecord& r : p->recs) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) return SPTS_ERR_CUDA;
+    ms[r.tag] += t; calls[r.tag] += 1; flops[r.tag] += r.flops; bytes[r.tag] += r.bytes;
+  }
+  p->recs.clear();
+  p->used = 0;
+  return SPTS_OK;
+}
 
 spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
   TRY(check_ctx(ctx));
@@ -302,9 +379,10 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   const int32_t* idx_a = nullptr;
   if (sel_a) {
     int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
-    TRY(launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
-    TRY(launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
-    TRY(launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
+    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_attn, launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
+    OP(SPTS_OP_KV_GATHER, 0.0, 2.0 * m_attn * (double)KD * es + 8.0 * m_attn,
+       launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
+    OP(SPTS_OP_KV_GATHER, 0.0, 12.0 * m_attn, launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
     idx_a = ia;
   } else {
     if (cudaMemcpyAsync(cache->pos, pos, (size_t)N * sizeof(int32_t), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
@@ -316,26 +394,31 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   memset(&g, 0, sizeof(g));
   g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_a; g.W = w->wq; g.M = m_attn; g.Nout = HD; g.K = D;
   g.rowscale = ws.rstd; g.out = ws.q_act; g.ldo = HD;
-  TRY(run_gemm(ctx, REF_ROPE, g));
+  const double Ma = (double)m_attn, Mf = (double)m_ffn, Dd = (double)D, esd = (double)es;
+  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * HD, (Ma * Dd + Ma * HD + Dd * HD) * esd, run_gemm(ctx, REF_ROPE, g));
   g.W = w->wv; g.Nout = KD; g.out = cache->v; g.ldo = KD;
   if (tc) { g.out_t = ws.v_t; g.ldt = ldvt; }
-  TRY(run_gemm(ctx, REF_STORE, g));
-  if (tc) TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)cache->v, (const bf16*)ws.v_t, ldvt, m_attn,
+  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * KD, (Ma * Dd + 2.0 * Ma * KD + Dd * KD) * esd, run_gemm(ctx, REF_STORE, g));
+  ProfScope* ps_att = new ProfScope(ctx, SPTS_OP_ATTN, 2.0 * HD * Ma * (Ma + 1.0), (2.0 * Ma * HD + 2.0 * Ma * KD) * esd);
+  spts_status s_att = SPTS_OK;
+  if (tc) s_att = (launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)cache->v, (const bf16*)ws.v_t, ldvt, m_attn,
                                   (bf16*)ws.o_att));
-  else TRY(launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att));
+  else s_att = launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att);
+  delete ps_att;
+  TRY(s_att);
   memset(&g, 0, sizeof(g));
   g.A = ws.o_att; g.lda = HD; g.a_rows = m_attn; g.dst_idx = idx_a; g.W = w->wo; g.M = m_attn; g.Nout = D; g.K = HD;
   g.out = X; g.ldo = D;
-  TRY(run_gemm(ctx, REF_RESID, g));
+  OP(SPTS_OP_OPROJ, 2.0 * Ma * Dd * HD, (Ma * HD + 2.0 * Ma * Dd + Dd * HD) * esd, run_gemm(ctx, REF_RESID, g));
   cache->len = m_attn;
 
   // ---- LTP + reduced FFN on the updated residual
-  TRY(launch_rstd(ctx, X, N, ws.rstd));
+  OP(SPTS_OP_PREP, 0.0, (double)N * Dd * esd + 4.0 * N, launch_rstd(ctx, X, N, ws.rstd));
   const int32_t* idx_f = nullptr;
   if (sel_f) {
     int32_t* jf = idx_ffn_out ? idx_ffn_out : ws.idx_f;
     TRY(ltp_pipeline(ctx, w, X, S, N, nullptr, ws.s_ffn));
-    TRY(launch_topk(ctx, ws.s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
+    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_ffn, launch_topk(ctx, ws.s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
     idx_f = jf;
   } else if (idx_ffn_out) {
     TRY(launch_topk(ctx, S, N, N, flags, idx_ffn_out, ws.topk_scratch));
@@ -343,11 +426,13 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   memset(&g, 0, sizeof(g));
   g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_f; g.W = w->w_gate; g.W2 = w->w_up; g.M = m_ffn; g.Nout = d.ffn_dim;
   g.K = D; g.rowscale = ws.rstd; g.out = ws.hm; g.ldo = d.ffn_dim;
-  TRY(run_gemm(ctx, REF_SWIGLU, g));
+  OP(SPTS_OP_GATEUP, 4.0 * Mf * Dd * d.ffn_dim, (Mf * Dd + Mf * d.ffn_dim + 2.0 * Dd * d.ffn_dim) * esd,
+     run_gemm(ctx, REF_SWIGLU, g));
   memset(&g, 0, sizeof(g));
   g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = m_ffn; g.dst_idx = idx_f; g.W = w->w_down; g.M = m_ffn; g.Nout = D;
   g.K = d.ffn_dim; g.out = X; g.ldo = D;
-  TRY(run_gemm(ctx, REF_RESID, g));
+  OP(SPTS_OP_DOWN, 2.0 * Mf * Dd * d.ffn_dim, (Mf * d.ffn_dim + 2.0 * Mf * Dd + Dd * d.ffn_dim) * esd,
+     run_gemm(ctx, REF_RESID, g));
   return SPTS_OK;
 }
 
@@ -363,7 +448,8 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
   if (n_next > N) n_next = N;
   if (!aligned16(X_in) || !aligned16(X_out)) return SPTS_ERR_INVALID_ARG;
   int32_t* idx = idx_out ? idx_out : ctx->ws.idx_p;
-  TRY(launch_topk(ctx, S_mha, N, n_next, flags, idx, ctx->ws.topk_scratch));
+  OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * n_next, launch_topk(ctx, S_mha, N, n_next, flags, idx, ctx->ws.topk_scratch));
+  ProfScope ps_c(ctx, SPTS_OP_COMPACT, 0.0, 2.0 * n_next * (double)ctx->desc.hidden * (double)elt_size(ctx->desc) + 28.0 * n_next);
   TRY(launch_gather_rows(ctx, X_in, idx, n_next, (int)(ctx->desc.hidden * elt_size(ctx->desc)), X_out));
   TRY(launch_gather_i32(ctx, pos_in, idx, n_next, pos_out));
   TRY(launch_gather_i32(ctx, orig_in, idx, n_next, orig_out));
@@ -375,6 +461,8 @@ spts_status spts_first_token(spts_ctx* ctx, const void* x_row, const void* lm_he
   TRY(check_ctx(ctx));
   if (x_row == nullptr || lm_head == nullptr || ctx->desc.vocab < 1) return SPTS_ERR_INVALID_ARG;
   if (!aligned16(x_row) || !aligned16(lm_head)) return SPTS_ERR_INVALID_ARG;
+  ProfScope ps_h(ctx, SPTS_OP_HEAD, 2.0 * ctx->desc.vocab * (double)ctx->desc.hidden,
+                 ctx->desc.vocab * ((double)ctx->desc.hidden * (double)elt_size(ctx->desc) + 8.0));
   return launch_head(ctx, x_row, lm_head, logits_out ? logits_out : ctx->ws.logits_v, token_out);
 }
 
@@ -430,11 +518,17 @@ spts_status spts_decode_step(spts_ctx* ctx, const spts_model_weights* mw, spts_k
   }
   for (int l = 0; l < d.n_layers; ++l)
     if (caches[l].len + 1 > caches[l].capacity) return SPTS_ERR_WORKSPACE;
+  double kvb = 0.0;
+  for (int l = 0; l < d.n_layers; ++l) kvb += 2.0 * (caches[l].len + 1.0) * d.n_kv_heads * d.head_dim * (double)es;
+  const double wl = ((2.0 * d.n_q_heads + 2.0 * d.n_kv_heads) * d.head_dim + 3.0 * d.ffn_dim) * (double)d.hidden;
+  ProfScope* ps_d = new ProfScope(ctx, SPTS_OP_DECODE, 2.0 * wl * d.n_layers, wl * d.n_layers * (double)es + kvb);
+  struct Guard { ProfScope* p; ~Guard() { delete p; } } guard_d{ps_d};
   TRY(launch_decode_load(ctx, x));
   for (int l = 0; l < d.n_layers; ++l) TRY(launch_decode_layer(ctx, &mw->layers[l], &caches[l], pos));
   // the residual is already rounded through the storage type; park it where the head can read it
   void* xo = x_out ? x_out : ctx->ws.xrow;
   TRY(launch_decode_store(ctx, xo));
+  delete guard_d.p; guard_d.p = nullptr;
   if (logits_out != nullptr || token_out != nullptr) {
     if (mw->lm_head == nullptr) return SPTS_ERR_INVALID_ARG;
     TRY(launch_head(ctx, xo, mw->lm_head, logits_out ? logits_out : ctx->ws.logits_v, token_out));

@@ -88,6 +88,7 @@ struct spts_ctx {
   int64_t launches;
   int sm_count;
   void* encode_tiled;       // cuTensorMapEncodeTiled entry point (tensor-core mode)
+  void* prof;               // per-operation CUDA-event timing (host state)
 };
 
 namespace spts {

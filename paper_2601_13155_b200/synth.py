@@ -170,3 +170,53 @@ def tiny_multilayer(n_layers: int = 4, n_tokens: int = 384, dtype: str = "fp32")
     firsts = tuple(range(0, n_layers, max(1, n_layers // 2)))[:2]
     toks = (n_tokens, (n_tokens * 3) // 4)[: len(firsts)]
     return Workload("tiny_ml", s, n_tokens, 1010, 24, 1, firsts, toks, 0.5, 0.4)
+
+
+# ----------------------------------------------------------------------------------------------
+# full-size workloads: drawn on the device (seeded torch generator) because 7 G parameters take
+# too long through numpy; the CPU oracle receives copies of the same tensors.
+# ----------------------------------------------------------------------------------------------
+def device_layer_weights(shape: ModelShape, seed: int, layer: int, device="cuda:0", std: float = 0.02):
+    """Same recipe as layer_weights (N(0, std), [out, in], rounded to the storage type) as torch tensors."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed * 100 + layer)
+    dt = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
+    out = {}
+    for name, fn in LAYER_WEIGHT_SHAPES.items():
+        w = torch.randn(fn(shape), generator=g, device=device, dtype=torch.float32) * std
+        out[name] = w.to(dt).contiguous()
+    return out
+
+
+def device_head_weights(shape: ModelShape, seed: int, device="cuda:0", std: float = 0.02):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed * 100 + 99)
+    dt = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
+    lm = (torch.randn((shape.vocab, shape.hidden), generator=g, device=device, dtype=torch.float32) * std).to(dt)
+    emb = torch.randn((shape.vocab, shape.hidden), generator=g, device=device, dtype=torch.float32).to(dt)
+    return {"lm_head": lm.contiguous(), "embed": emb.contiguous()}
+
+
+def device_hidden_states(w: "Workload", device="cuda:0", n_tokens: Optional[int] = None):
+    """X [N, hidden] ~ N(0,1) on the device with the workload's heavy rows (x8); returns (X, heavy_rows)."""
+    import torch
+    n = w.n_tokens if n_tokens is None else n_tokens
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed)
+    X = torch.randn((n, w.shape.hidden), generator=g, device=device, dtype=torch.float32)
+    rng = np.random.default_rng(w.seed)
+    heavy = max(1, int(round(w.heavy * n / w.n_tokens))) if w.heavy else 0
+    if heavy:
+        if w.cluster <= 1:
+            rows = np.sort(rng.choice(n, size=heavy, replace=False))
+        else:
+            n_cl = max(1, heavy // w.cluster)
+            starts = np.sort(rng.choice(n // w.cluster, size=n_cl, replace=False)) * w.cluster
+            rows = (starts[:, None] + np.arange(w.cluster)[None, :]).reshape(-1)
+        X[torch.from_numpy(rows).to(device)] *= 8.0
+    else:
+        rows = np.zeros((0,), np.int64)
+    dt = torch.bfloat16 if w.shape.dtype == "bf16" else torch.float32
+    return X.to(dt).contiguous(), rows
