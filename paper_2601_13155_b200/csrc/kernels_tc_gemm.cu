@@ -3,9 +3,10 @@
 //   acc[i, j] = sum_k A[src(i), k] * W[j, k]          A rows optionally gathered by an index list
 //
 // Persistent, warp-specialised CTA (one per SM):
-//   warp 0      TMA producer: A tile by a tiled load, or -- for the gathered rows of the reduced
-//               attention / FFN blocks (Algorithm 1, X^ = X[T_active, :]) -- by 32 tile::gather4
-//               loads, one per lane, straight into the 128B-swizzled operand layout; W tile(s) tiled
+//   warp 0      TMA producer: W tile(s) and, when A is contiguous, the A tile
+//   warps 6-9   (gather variant only) fetch the rows X[T_active, :] of the reduced attention / FFN
+//               blocks (Algorithm 1, X^ = X[T_active, :]) straight into the 128B-swizzled operand
+//               layout, so the gather costs no pass of its own
 //   warp 1      TMEM allocation and the single-thread tcgen05.mma issue loop
 //   warps 2-5   epilogue: tcgen05.ld of the fp32 accumulator (each warp its lane quarter, one
 //               row per thread), then one of
@@ -42,6 +43,7 @@ struct TcParams {
   const int32_t* idx;
   const int32_t* dst_idx;
   int M, Nout, K, a_rows;
+  const void* a_ptr; int lda;   // A base and row stride (elements) for the gather producers
   const float* rowscale;
   bf16* out; int ldo;
   bf16* out_t; int ldt;
@@ -85,8 +87,24 @@ __device__ __forceinline__ void store32_bf16(bf16* p, const float* v, int c0, in
   }
 }
 
-template <int BN, int EPI>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+// 16-byte asynchronous copy global -> shared; src_bytes == 0 writes zeros
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int GATHER_WARPS = 4;      // extra producer warps of the row-gather variant
+constexpr int GATHER_LAG = 2;        // k-blocks a gather thread keeps in flight before publishing
+
+// GATHER: the A rows are X[idx[i], :].  Warps 6..9 fetch them with 16-byte cp.async copies --
+// eight lanes per 128-byte row slice, written straight into the swizzled operand layout -- while
+// warp 0 keeps feeding W through TMA.  (A tile::gather4 TMA load does the same job in one
+// instruction per four rows, but was measured at a third of the tiled-load rate on this part.)
+template <int BN, int EPI, bool GATHER>
+__global__ void __launch_bounds__(GATHER ? GEMM_THREADS + 32 * GATHER_WARPS : GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const TcParams p) {
   using C = Cfg<BN>;
@@ -110,7 +128,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar + 8 * s, GATHER ? 1 + 32 * GATHER_WARPS : 1);
+      mbar_init(empty_bar + 8 * s, 1);
+    }
     for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar + 8 * b, 1); mbar_init(tempty_bar + 8 * b, 4); }
     fence_mbar_init();
     prefetch_tensormap(&tmA);
@@ -127,41 +148,79 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ producer
-    int stage = 0; uint32_t phase = 0;
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        int mb, nb;
+        tile_coords(t, p.num_m, p.num_n, mb, nb);
+        const int m0 = mb * BM, n0 = nb * NT;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag, t0);
+          if (!ok) break;
+          mbar_expect_tx(full_bar + 8 * stage, (GATHER ? 0 : A_STAGE_BYTES) + C::B_STAGE_BYTES);
+          const int k0 = kb * BK;
+          const uint32_t a_dst = sA + stage * A_STAGE_BYTES, b_dst = sB + stage * C::B_STAGE_BYTES;
+          if (!GATHER) tma_load_2d(a_dst, &tmA, full_bar + 8 * stage, k0, m0);
+          tma_load_2d(b_dst, &tmB, full_bar + 8 * stage, k0, n0);
+          if (EPI == TC_SWIGLU) tma_load_2d(b_dst + (BN / 2) * BK * 2, &tmB2, full_bar + 8 * stage, k0, n0);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (GATHER && warp >= 6) {
+    // ------------------------------------------------------------------ row-gather producers
+    // lane -> (row offset lane / 8 inside a group of four rows, 16-byte chunk lane % 8)
+    const int pw = warp - 6;
+    const int chunk = lane & 7;
+    const bf16* Abase = reinterpret_cast<const bf16*>(p.a_ptr);
+    int stage = 0; uint32_t phase = 0;      // stage being filled
+    int pstage = 0;                         // next stage to publish
+    int inflight = 0;                       // committed, unpublished k-blocks
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
       int mb, nb;
       tile_coords(t, p.num_m, p.num_n, mb, nb);
-      const int m0 = mb * BM, n0 = nb * NT;
-      int r[4] = {0, 0, 0, 0};
-      if (p.idx != nullptr) {
+      const int m0 = mb * BM;
+      const bf16* rowp[8];
+      uint32_t soff[8];
+      bool rvalid[8];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          int gi = m0 + lane * 4 + e;
-          r[e] = gi < p.M ? p.idx[gi] : 0;       // rows past the end load row 0 and are masked later
-        }
+      for (int e = 0; e < 8; ++e) {
+        const int rt = pw * 32 + e * 4 + (lane >> 3);          // row inside the tile
+        const int gi = m0 + rt;
+        rvalid[e] = gi < p.M;
+        const int src = rvalid[e] ? p.idx[gi] : 0;
+        rowp[e] = Abase + (size_t)src * p.lda + chunk * 8;
+        soff[e] = (uint32_t)(rt * 128 + ((chunk ^ (rt & 7)) << 4));
       }
       for (int kb = 0; kb < kblocks; ++kb) {
-        if (lane == 0) {
-          ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag, t0);
-          if (ok) mbar_expect_tx(full_bar + 8 * stage, A_STAGE_BYTES + C::B_STAGE_BYTES);
-        }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
+        ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag, t0);
         if (!ok) break;
         const int k0 = kb * BK;
-        const uint32_t a_dst = sA + stage * A_STAGE_BYTES, b_dst = sB + stage * C::B_STAGE_BYTES;
-        if (p.idx != nullptr) {
-          tma_gather4(a_dst + lane * 512, &tmA, full_bar + 8 * stage, k0, r[0], r[1], r[2], r[3]);
-        } else if (lane == 0) {
-          tma_load_2d(a_dst, &tmA, full_bar + 8 * stage, k0, m0);
-        }
-        if (lane == 0) {
-          tma_load_2d(b_dst, &tmB, full_bar + 8 * stage, k0, n0);
-          if (EPI == TC_SWIGLU) tma_load_2d(b_dst + (BN / 2) * BK * 2, &tmB2, full_bar + 8 * stage, k0, n0);
-        }
+        const bool kin = k0 + chunk * 8 < p.K;
+        const uint32_t a_dst = sA + stage * A_STAGE_BYTES;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) cp_async16(a_dst + soff[e], rowp[e] + k0, (rvalid[e] && kin) ? 16u : 0u);
+        cp_async_commit();
+        ++inflight;
         if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        if (inflight > GATHER_LAG) {
+          cp_async_wait<GATHER_LAG>();
+          fence_proxy_async_smem();
+          mbar_arrive(full_bar + 8 * pstage);
+          if (++pstage == STAGES) pstage = 0;
+          --inflight;
+        }
       }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    while (ok && inflight > 0) {
+      mbar_arrive(full_bar + 8 * pstage);
+      if (++pstage == STAGES) pstage = 0;
+      --inflight;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -383,11 +442,12 @@ bool make_map(spts_ctx* ctx, CUtensorMap* tm, const void* base, uint64_t rows, u
   return r == CUDA_SUCCESS;
 }
 
-template <int BN, int EPI>
-spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
+template <int BN, int EPI, bool GATHER>
+spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   constexpr int NT = (EPI == TC_SWIGLU) ? BN / 2 : BN;
   TcParams p;
   p.idx = a.idx; p.dst_idx = a.dst_idx; p.M = a.M; p.Nout = a.Nout; p.K = a.K; p.a_rows = a.a_rows;
+  p.a_ptr = a.A; p.lda = a.lda;
   p.rowscale = a.rowscale; p.out = a.out; p.ldo = a.ldo; p.out_t = a.out_t; p.ldt = a.ldt;
   p.cs = ctx->ws.rope_cs; p.q = a.q; p.logits = a.logits; p.ld_logits = a.ld_logits; p.group = a.group;
   p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
@@ -395,8 +455,7 @@ spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
   p.num_n = ceil_div(a.Nout, NT);
   if (EPI == TC_SUMSQ && p.num_n > a.csq_parts) return SPTS_ERR_WORKSPACE;
   CUtensorMap tmA, tmB, tmB2;
-  if (!make_map(ctx, &tmA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, (uint64_t)a.lda, a.idx ? 1u : (uint32_t)BM))
-    return SPTS_ERR_CUDA;
+  if (!make_map(ctx, &tmA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, (uint64_t)a.lda, (uint32_t)BM)) return SPTS_ERR_CUDA;
   if (!make_map(ctx, &tmB, a.W, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
   if (EPI == TC_SWIGLU) {
     if (!make_map(ctx, &tmB2, a.W2, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
@@ -405,15 +464,30 @@ spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
   }
   const int tiles = p.num_m * p.num_n;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-  tc_gemm_kernel<BN, EPI><<<grid, GEMM_THREADS, Cfg<BN>::SMEM_BYTES, ctx->stream>>>(tmA, tmB, tmB2, p);
+  tc_gemm_kernel<BN, EPI, GATHER><<<grid, GATHER ? GEMM_THREADS + 32 * GATHER_WARPS : GEMM_THREADS, Cfg<BN>::SMEM_BYTES,
+                                    ctx->stream>>>(tmA, tmB, tmB2, p);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }
 
 template <int BN, int EPI>
+spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
+  if (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU) {
+    if (a.idx != nullptr) return launch_one_g<BN, EPI, (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU)>(ctx, a);
+  } else if (a.idx != nullptr) {
+    return SPTS_ERR_UNSUPPORTED;
+  }
+  return launch_one_g<BN, EPI, false>(ctx, a);
+}
+
+template <int BN, int EPI>
 bool set_smem_attr() {
-  return cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+  bool ok = cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+  if (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU)
+    ok = ok && cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI, (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU)>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+  return ok;
 }
 
 }  // namespace

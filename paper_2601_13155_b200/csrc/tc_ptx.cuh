@@ -1,5 +1,5 @@
 // Thin wrappers over the sm_100a PTX used by the tensor-core kernels: mbarrier, TMA
-// (cp.async.bulk.tensor, tiled and tile::gather4), tcgen05 (TMEM alloc, mma, commit, ld) and the
+// (cp.async.bulk.tensor tiled loads), tcgen05 (TMEM alloc, mma, commit, ld) and the
 // shared-memory / instruction descriptors.  Every wait is bounded: when it runs out the kernel
 // records SPTS_ERR_TIMEOUT, raises a CTA-wide abort flag and unwinds (no trap, no endless spin).
 #pragma once
@@ -74,15 +74,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-// Four rows (r0..r3) of `cols` starting at column c0; the tensor map's box is one row high.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int r0, int r1,
-                                            int r2, int r3) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
-      "%5, %6, %7}], [%2];" ::"r"(dst),
-      "l"(tm), "r"(bar), "r"(c0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
       : "memory");
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* tm) {
