@@ -158,19 +158,15 @@ def main():
     import torch
     from paper_2601_13155_b200 import binding, schedule, synth, build
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2601_13155_b200.replicas import Replicas
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     dev = f"cuda:{local}"
     torch.cuda.set_device(dev)
+    rep = Replicas(backend="nccl", device=torch.device(dev))
+    rank, world = rep.rank, rep.world
     if rank == 0 and not os.path.exists(binding.LIB_PATH):
         build.build()
-    if dist is not None:
-        dist.barrier()
+    rep.barrier()
 
     w = synth.workload(args.workload)
     shape = w.shape
@@ -216,11 +212,7 @@ def main():
         if from_host:
             tok_host.copy_(tok, non_blocking=True)
 
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+    barrier = rep.barrier
 
     def timed(pl, steps, from_host=False, profile_op=0):
         barrier()
@@ -235,11 +227,7 @@ def main():
         barrier()
         ms = e0.elapsed_time(e1)
         prof = lib.profile_end() if profile_op else {}
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, lib.launch_count() - l0, prof
+        return rep.max_over_ranks(ms), lib.launch_count() - l0, prof
 
     for _ in range(max(args.warmup, 3)):
         step(plan)
@@ -327,9 +315,7 @@ def main():
                 gb = v["bytes"] / max(v["ms"], 1e-9) / 1e6
                 sys.stderr.write(f"{k:12s} {v['ms']:9.3f} ms  {v['calls']:4d} calls  {tf:8.1f} TFLOP/s  {gb:8.1f} GB/s\n")
         print(json.dumps(line))
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    rep.close()
 
 
 if __name__ == "__main__":

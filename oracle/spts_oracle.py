@@ -154,6 +154,23 @@ def causal_gqa_attention(Q, K, V, row_chunk=1024):
     return out.reshape(m, H * d)
 
 
+def causal_gqa_attention_rows(Q_rows, rows, K, V):
+    """The rows `rows` of causal_gqa_attention(Q, K, V) without forming the others:
+    Q_rows [s,H,d] holds the queries of those rows; row i attends to K[j], V[j] for j <= i
+    (compact order, Algorithm 1's F_MHA on the active rows).  Returns [s, H*d]."""
+    Q_rows = np.asarray(Q_rows, F64)
+    s, H, d = Q_rows.shape
+    G = H // K.shape[1]
+    out = np.zeros((s, H, d), F64)
+    for a, i in enumerate(rows):
+        for h in range(H):
+            z = K[: i + 1, h // G, :] @ Q_rows[a, h] / math.sqrt(d)
+            z = z - z.max()
+            e = np.exp(z)
+            out[a, h] = (e / e.sum()) @ V[: i + 1, h // G, :]
+    return out.reshape(s, H * d)
+
+
 # ----------------------------------------------------------------------------
 # Eq. 6 and Eq. 12-14
 # ----------------------------------------------------------------------------
@@ -219,6 +236,36 @@ def layer_prefill_skip(X, pos, W, shape, m_attn, m_ffn, g_attn=None, g_ffn=None,
 
     return {"X": X, "S_mha": S_mha, "idx_attn": Ta, "C": C, "S_ffn": S_ffn, "idx_ffn": Tf,
             "K": Kh, "V": Vh, "cache_pos": pos[Ta].copy(), "K_all": K, "q": q}
+
+
+def attention_block_rows(X, pos, W, shape, Ta, K_all, sample, mode="exact"):
+    """Eq. 2 for the attention block on a sample of the active rows: returns the updated
+    hidden rows X[Ta[sample]] + F_MHA(...) W_O given the active set Ta (ascending) and the
+    post-RoPE keys K_all [N,Hkv,d] of every candidate.  V is projected for all active rows
+    (every later active row attends to it), Q only for the sampled rows."""
+    rnd = rounding(mode)
+    W = _w64(W)
+    X = np.asarray(X)
+    pos = np.asarray(pos)
+    H, Hkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    Ta = np.asarray(Ta)
+    sample = np.asarray(sample)
+    ones = np.ones(X.shape[1])
+    Aa = rmsnorm(X[Ta], ones, shape.rms_eps)
+    Vh = rnd((Aa @ W["wv"].T).reshape(len(Ta), Hkv, d))
+    Kh = rnd(np.asarray(K_all, F64)[Ta])
+    Qs = rnd(rope((Aa[sample] @ W["wq"].T).reshape(len(sample), H, d), pos[Ta[sample]], shape.rope_theta))
+    att = rnd(causal_gqa_attention_rows(Qs, sample, Kh, Vh))
+    return rnd(np.asarray(X[Ta[sample]], F64) + att @ W["wo"].T), Kh, Vh
+
+
+def ffn_block_rows(X, W, shape, rows, mode="exact"):
+    """Eq. 2 + Eq. 6 for the FFN block on the given rows of the (post-attention) residual X."""
+    rnd = rounding(mode)
+    W = _w64(W)
+    xr = np.asarray(X[np.asarray(rows)], F64)
+    B = rmsnorm(xr, np.ones(xr.shape[1]), shape.rms_eps)
+    return rnd(xr + ffn(B, W["w_gate"], W["w_up"], W["w_down"], rnd))
 
 
 def layer_dense(X, pos, W, shape, g_attn=None, g_ffn=None, mode="exact"):

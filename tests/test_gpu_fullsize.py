@@ -1,0 +1,139 @@
+"""GPU parity at the sizes and launch shapes the benchmark times (LLaMA-3.1-8B layer shape, bf16).
+
+The fp64 oracle cannot run a whole layer at these sizes in test time, so: score vectors and index sets are
+compared in full (they are cheap), hidden-state updates on a seeded sample of rows the oracle computes one
+by one (attention rows against all earlier active keys), skipped rows bit for bit.  Inputs are drawn with
+the benchmark's own generators.  Same tolerances as the small cases: index sets equal to the oracle's
+outside a 1e-3 relative band at the k-th score, outputs within 2e-2 of the output RMS."""
+import math
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import spts_oracle as O
+from paper_2601_13155_b200 import synth
+from parity_utils import check_index_set, check_output, dev, host
+
+pytestmark = pytest.mark.gpu
+
+
+def _host_weights(t):
+    return {k: v.float().cpu().numpy().astype(np.float64) for k, v in t.items()}
+
+
+def _sample(m, n_rand, seed):
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 2, 63, 64, 127, 128, 129, 255, 256, m // 2, m - 130, m - 129, m - 128, m - 2, m - 1]
+    s = set(i for i in fixed if 0 <= i < m)
+    s.update(int(i) for i in rng.choice(m, size=min(m, n_rand), replace=False))
+    return np.array(sorted(s))
+
+
+def _run_layer_case(name, N, ma, mf, n_rows):
+    from paper_2601_13155_b200 import binding
+    w = synth.workload(name)
+    shape = replace(w.shape, n_layers=1)
+    wt = synth.device_layer_weights(shape, w.seed, 0, dev())
+    lw = binding.LayerWeights.__new__(binding.LayerWeights)
+    lw.t = wt
+    lw.c = binding.LayerWeightsC(**{k: wt[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    wz = dict(wt)
+    wz["w_down"] = torch.zeros_like(wt["w_down"])
+    lz = binding.LayerWeights.__new__(binding.LayerWeights)
+    lz.t = wz
+    lz.c = binding.LayerWeightsC(**{k: wz[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    X0, _ = synth.device_hidden_states(w, dev(), n_tokens=N)
+    pos_h = np.arange(N, dtype=np.int32) * 2 + 3          # original positions need not be 0..N-1
+    pos = torch.from_numpy(pos_h).to(dev())
+    lib = binding.Spts(shape, max_seq=N)
+
+    # GPU: attention block alone (W_down = 0, FFN dense), then the real layer
+    Xmid = X0.clone()
+    lib.layer_prefill_skip(lz, Xmid, pos, ma, N, binding.KvCache(shape, 1, N))
+    Xd = X0.clone()
+    cache = binding.KvCache(shape, 1, ma)
+    S = torch.empty(N, dtype=torch.float32, device=dev())
+    ia = torch.empty(ma, dtype=torch.int32, device=dev())
+    jf = torch.empty(mf, dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip(lw, Xd, pos, ma, mf, cache, S_out=S, idx_attn_out=ia, idx_ffn_out=jf)
+    assert lib.device_status() == 0
+    ia_h, jf_h = ia.cpu().numpy().astype(np.int64), jf.cpu().numpy().astype(np.int64)
+
+    # ---- oracle: scores and the attention index set in full
+    W = _host_weights(wt)
+    x_in = host(X0)
+    ones = np.ones(shape.hidden)
+    A = O.rmsnorm(x_in, ones, shape.rms_eps)
+    K_all, _, S_o = O.pap_score(A, pos_h, W["wk"], W["wq"], shape)
+    del A
+    if ma < N or mf < N:
+        assert np.abs(host(S) - S_o).max() <= 2e-4 * S_o.max()
+        assert abs(float(host(S).sum()) - 1.0) < 1e-4
+    swaps_a = check_index_set(ia_h, S_o, ma) if ma < N else 0
+    if ma == N:
+        assert np.array_equal(ia_h, np.arange(N))
+    # ---- attention block on sampled active rows, with the (validated) GPU index set
+    smp = _sample(ma, n_rows, 11)
+    want_rows, Kh, Vh = O.attention_block_rows(x_in, pos_h, W, shape, ia_h, K_all, smp, mode="bf16")
+    xm = host(Xmid)
+    check_output(xm[ia_h[smp]], want_rows, "bf16")
+    assert cache.length(0) == ma
+    assert np.array_equal(cache.pos[0][:ma].cpu().numpy(), pos_h[ia_h])
+    check_output(host(cache.k[0][:ma]), Kh, "bf16")
+    check_output(host(cache.v[0][:ma]), Vh, "bf16")
+    del K_all, Kh, Vh
+    # rows outside T_a are untouched by the attention block
+    mask = torch.ones(N, dtype=torch.bool, device=dev())
+    mask[ia.long()] = False
+    assert torch.equal(Xmid[mask], X0[mask])
+
+    # ---- FFN block from the GPU's post-attention residual: LTP scores and T_f in full, update on sampled rows
+    if mf < N:
+        B = O.rmsnorm(xm, ones, shape.rms_eps)
+        _, Sf_o = O.ltp_score(B, S_o, W, O.round_bf16)
+        del B
+        swaps_f = check_index_set(jf_h, Sf_o, mf)
+    else:
+        swaps_f = 0
+        assert np.array_equal(jf_h, np.arange(N))
+    smp_f = jf_h[_sample(mf, n_rows, 12)]
+    check_output(host(Xd[torch.from_numpy(smp_f).to(dev())]), O.ffn_block_rows(xm, W, shape, smp_f, mode="bf16"), "bf16")
+    # Eq. 2: rows outside T_f keep the post-attention value, rows outside both sets keep the input
+    mask_f = torch.ones(N, dtype=torch.bool, device=dev())
+    mask_f[jf.long()] = False
+    assert torch.equal(Xd[mask_f], Xmid[mask_f])
+    lib.close()
+    return swaps_a + swaps_f, S, X0
+
+
+def test_config2_layer_sampled_rows():
+    """BASELINE config 2: one 8B-shaped layer, 8192 tokens, attention keep 0.5, FFN keep 0.4."""
+    _run_layer_case("cfg2", 8192, 4096, math.ceil(0.4 * 8192), 256)
+
+
+def test_bench_stage0_layer_sampled_rows_and_prune():
+    """The benchmark's first-stage launch shape: 32768 candidates, 16384 attention rows, 13108 FFN rows; then the
+    stage-end prune to 24576 candidates (Eq. 16) on the layer's own PAP score."""
+    from paper_2601_13155_b200 import binding
+    N, n_next = 32768, 24576
+    _, S, X0 = _run_layer_case("cfg3", N, 16384, math.ceil(0.4 * N), 256)
+    shape = replace(synth.LLAMA8B, n_layers=1)
+    lib = binding.Spts(shape, max_seq=N)
+    ar = torch.arange(N, dtype=torch.int32, device=dev())
+    Xo = torch.empty(n_next, shape.hidden, dtype=torch.bfloat16, device=dev())
+    po, oo, io = (torch.empty(n_next, dtype=torch.int32, device=dev()) for _ in range(3))
+    lib.msdp_compact(X0, ar * 2 + 3, ar, S, n_next, Xo, po, oo, io)
+    assert lib.device_status() == 0
+    T = O.topk_select(S.cpu().numpy(), n_next, True)          # bit-exact given the same fp32 scores
+    assert np.array_equal(io.cpu().numpy(), T)
+    Tt = torch.from_numpy(T).to(dev())
+    assert torch.equal(Xo, X0[Tt]) and torch.equal(oo.long(), Tt) and torch.equal(po.long(), Tt * 2 + 3)
+    lib.close()
+
+
+def test_bench_last_stage_dense_ragged_layer():
+    """The benchmark's last-stage shape: 11469 candidates (not a multiple of any tile), budgets clipped to the
+    candidate count, so both blocks run densely without probing."""
+    _run_layer_case("cfg3", 11469, 11469, 11469, 256)

@@ -181,6 +181,45 @@ def test_attention_matches_torch_sdpa():
     assert np.allclose(O.causal_gqa_attention(Q, K, V), want, atol=1e-12)
 
 
+def test_attention_rows_match_torch_sdpa_and_full_routine():
+    rng = np.random.default_rng(16)
+    m, H, Hkv, d = 41, 4, 2, 16
+    Q, K, V = rng.standard_normal((m, H, d)), rng.standard_normal((m, Hkv, d)), rng.standard_normal((m, Hkv, d))
+    rows = np.array([0, 1, 7, 8, 22, 40])
+    t = lambda a: torch.from_numpy(a).permute(1, 0, 2)[None]
+    want = torch.nn.functional.scaled_dot_product_attention(t(Q), t(K), t(V), is_causal=True, enable_gqa=True)
+    want = want[0].permute(1, 0, 2).reshape(m, H * d).numpy()
+    got = O.causal_gqa_attention_rows(Q[rows], rows, K, V)
+    assert np.allclose(got, want[rows], atol=1e-12)
+    assert np.allclose(got, O.causal_gqa_attention(Q, K, V)[rows], atol=1e-12)
+
+
+@pytest.mark.parametrize("mode", ["exact", "bf16"])
+def test_sampled_block_rows_equal_the_whole_layer(mode):
+    """The row-sampled evaluation used at full size reproduces the rows of the whole-layer
+    oracle (which is pinned against the HF decoder layer and Eq. 2)."""
+    W = _layer()
+    N, ma, mf = 48, 20, 17
+    X, pos = _x(N), np.arange(N) * 3 + 2
+    r = O.layer_prefill_skip(X, pos, W, SH, ma, mf, mode=mode)
+    rz = O.layer_prefill_skip(X, pos, dict(W, w_down=np.zeros_like(W["w_down"])), SH, ma, N, mode=mode)
+    sample = np.array([0, 1, 5, 19])
+    got, Kh, Vh = O.attention_block_rows(X, pos, W, SH, r["idx_attn"], r["K_all"], sample, mode=mode)
+
+    def same(a, b):
+        # BLAS sums in a different order for a different row count: equal up to fp64 rounding; in
+        # bf16 mode a value sitting on a rounding boundary may land one bf16 step away
+        d = np.abs(a - b)
+        if mode == "exact":
+            return d.max() < 1e-11
+        return (d < 1e-11).mean() > 0.99 and np.all(d <= np.abs(b) * 2.0 ** -7 + 1e-11)
+
+    assert same(got, rz["X"][r["idx_attn"][sample]])
+    assert same(Kh, r["K"]) and same(Vh, r["V"])
+    rows = r["idx_ffn"][[0, 3, 16]]
+    assert same(O.ffn_block_rows(rz["X"], W, SH, rows, mode=mode), r["X"][rows])
+
+
 # ------------------------------------------------------------------ dense layer vs HF
 def _hf_config(shape):
     from transformers import LlamaConfig
