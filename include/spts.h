@@ -192,6 +192,27 @@ spts_status spts_ltp_score(spts_ctx* ctx, const spts_layer_weights* w, const voi
 spts_status spts_topk_select(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags,
                              int32_t* idx_out);
 
+/* The same selection for callers that cannot allocate device memory (the paper has no counterpart:
+ * this exists for hosts whose device memory is planned and frozen before inference starts, or that are
+ * only ever handed input and output buffers -- they can neither allocate the workspace spts_create()
+ * needs nor let a library allocate behind their back).  It needs no context and no workspace: its
+ * scratch is a fixed array of SPTS_TOPK_STATIC_SCRATCH_BYTES inside the library, resident on every GPU
+ * that loads the library until the process exits.  Same result as spts_topk_select (same ordering rule,
+ * ascending output, SPTS_FORCE_LAST); NaN scores rank last but are not reported, there being no context
+ * to hold a status word.  Work is enqueued on `cuda_stream` (a cudaStream_t, may be 0) of the current
+ * device and the call does not synchronise.
+ *   - 1 <= k <= N <= SPTS_TOPK_STATIC_MAX_N, else SPTS_ERR_INVALID_ARG / SPTS_ERR_SHAPE before any launch.
+ *   - The first call on each device looks up the array's device address (a synchronous runtime query,
+ *     made with that device current); make that first call before any stream capture begins.
+ *   - All calls on one device share the array.  Each call clears the counters it needs, so calls that
+ *     are ordered on the GPU (same stream, or dependent streams) are fine; calls that may overlap on
+ *     the GPU race on the scratch and give undefined index lists.
+ *   - It calls no cudaMalloc / cudaFree or other allocating routine. */
+#define SPTS_TOPK_STATIC_MAX_N 8388608
+#define SPTS_TOPK_STATIC_SCRATCH_BYTES 36928
+spts_status spts_topk_select_static(const float* scores, int N, int k, uint32_t flags, int32_t* idx_out,
+                                    void* cuda_stream);
+
 /* One decoder layer of Algorithm 1 in the prefill phase, in place on X [N, D]:
  *   S_mha (Eq. 4) -> T_a = TopK(S_mha, m_attn) -> Q, V projected for the rows in T_a, K rows
  *   reused -> cache <- (K^, V^, pos[T_a]) -> causal GQA attention among the active rows ->

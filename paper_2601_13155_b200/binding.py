@@ -59,7 +59,8 @@ class ModelWeightsC(C.Structure):
 EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_option",
            "spts_last_device_status", "spts_launch_count", "spts_fold_norm_gain", "spts_pap_score",
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
-           "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end")
+           "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
+           "spts_topk_select_static")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -85,6 +86,7 @@ def load_library() -> C.CDLL:
     lib.spts_pap_score.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, vp, vp]
     lib.spts_ltp_score.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, vp, vp]
     lib.spts_topk_select.argtypes = [vp, vp, i32, i32, u32, vp]
+    lib.spts_topk_select_static.argtypes = [vp, i32, i32, u32, vp, vp]
     lib.spts_layer_prefill_skip.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, i32, i32, u32,
                                             C.POINTER(KvLayerC), vp, vp, vp]
     lib.spts_msdp_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, vp, vp, vp, vp]
@@ -117,6 +119,29 @@ def to_device(a: np.ndarray, dtype: str, device="cuda:0") -> torch.Tensor:
     """Uploads a float32 array (already rounded to the storage type) as a device tensor."""
     t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(device)
     return t.to(torch_dtype(dtype)).contiguous()
+
+
+TOPK_STATIC_MAX_N = 8388608
+_static_lib = None
+
+
+def topk_select_static(scores: torch.Tensor, k: int, flags: int = 0, idx_out: Optional[torch.Tensor] = None,
+                       stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """spts_topk_select_static: top-k without a context or a workspace, for callers that cannot allocate
+    device memory (the scratch is a fixed array inside the library).  The index buffer is the caller's:
+    pass `idx_out` [k] int32 to keep this call itself free of allocations."""
+    global _static_lib
+    if _static_lib is None:
+        _static_lib = load_library()
+    N = scores.shape[0]
+    if idx_out is None:
+        idx_out = torch.empty(max(k, 1), dtype=torch.int32, device=scores.device)
+    st = stream if stream is not None else torch.cuda.current_stream(scores.device)
+    with torch.cuda.device(scores.device):
+        code = _static_lib.spts_topk_select_static(_ptr(scores), N, k, flags, _ptr(idx_out), C.c_void_p(st.cuda_stream))
+    if code != 0:
+        raise SptsError(code, "spts_topk_select_static")
+    return idx_out
 
 
 class LayerWeights:

@@ -3,6 +3,8 @@
 //
 // Selection rule: score descending, then index ascending; -0.0 == +0.0; NaN ranks with -inf;
 // with SPTS_FORCE_LAST the last element ranks first.  Output indices are ascending.
+#include <mutex>
+
 #include "spts_common.cuh"
 
 namespace spts {
@@ -297,3 +299,65 @@ spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* 
 }
 
 }  // namespace spts
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free top-k (declared in spts.h as spts_topk_select_static)
+//
+// Every other call of the library works out of a workspace the caller allocated.  Some hosts cannot
+// allocate at all: an inference server whose device memory was planned and frozen at start-up, a
+// plugin that only ever receives input and output buffers from its framework, a real-time loop that
+// must not touch the allocator.  For them the radix-select scratch lives in this file-scope device
+// array, which every GPU that loads the library holds from load to exit.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) uint32_t spts_static_topk_scratch[spts::TOPK_SCRATCH_WORDS];
+static_assert(sizeof(uint32_t) * spts::TOPK_SCRATCH_WORDS == SPTS_TOPK_STATIC_SCRATCH_BYTES, "scratch size as documented");
+static_assert((long)spts::TOPK_MAX_CTAS * spts::TOPK_CHUNK == SPTS_TOPK_STATIC_MAX_N, "size limit as documented");
+
+namespace spts {
+namespace {
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mu;
+uint32_t* g_static_ptr[STATIC_MAX_DEVICES];   // device address of the array, per device ordinal
+
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address each device gave it is looked up once per device, with that device current.
+spts_status static_scratch_address(uint32_t** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return SPTS_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, spts_static_topk_scratch) != cudaSuccess || p == nullptr) return SPTS_ERR_CUDA;
+    g_static_ptr[dev] = static_cast<uint32_t*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return SPTS_OK;
+}
+
+}  // namespace
+}  // namespace spts
+
+extern "C" spts_status spts_topk_select_static(const float* scores, int N, int k, uint32_t flags, int32_t* idx_out,
+                                               void* cuda_stream) {
+  using namespace spts;
+  if (scores == nullptr || idx_out == nullptr || N < 1 || k < 1 || k > N) return SPTS_ERR_INVALID_ARG;
+  if (N > SPTS_TOPK_STATIC_MAX_N) return SPTS_ERR_SHAPE;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (k == N) {   // the identity list needs no scratch
+    iota_kernel<<<ceil_div(N, 256), 256, 0, st>>>(idx_out, N);
+    return cudaGetLastError() == cudaSuccess ? SPTS_OK : SPTS_ERR_CUDA;
+  }
+  uint32_t* scratch = nullptr;
+  spts_status s = static_scratch_address(&scratch);
+  if (s != SPTS_OK) return s;
+  const int nb = ceil_div(N, TOPK_CHUNK);
+  const int fl = (flags & SPTS_FORCE_LAST) ? 1 : 0;
+  // the array keeps the previous call's contents: histograms, prefix and counters must start at zero
+  if (cudaMemsetAsync(scratch, 0, (4 * 256 + 16) * sizeof(uint32_t), st) != cudaSuccess) return SPTS_ERR_CUDA;
+  for (int pass = 0; pass < 4; ++pass)
+    topk_hist_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, pass, fl, scratch, nullptr);
+  topk_count_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, fl, scratch);
+  topk_emit_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, fl, scratch, idx_out);
+  return cudaGetLastError() == cudaSuccess ? SPTS_OK : SPTS_ERR_CUDA;
+}
