@@ -2,17 +2,23 @@
 // Index lists are ascending, so causality among the selected tokens is a lower triangle in the
 // compact row order.
 //
-// One CTA = 128 queries of one head.  grid = (H, ceil(m/128)); heads of one GQA group are
-// neighbours so they share K/V tiles through L2, and the longest (last) query tiles start first.
-//   warp 0      TMA producer: Q tile once, then K_j [128 keys x 128] and V^T_j [128 x 128 keys]
-//   warp 1      TMEM owner and single-thread MMA issuer:  S_j = Q K_j^T  (two S buffers in TMEM),
-//               O += P_j V_j  (O accumulates in TMEM)
-//   warps 2-5   one query row per thread: S from TMEM, online softmax in the exp2 domain with a
-//               lazily updated running maximum (O is rescaled in TMEM only when the maximum grows
-//               by more than 2^8), P_j written as bf16 into the swizzled K-major operand layout
-//               in shared memory, final O / l written to global memory.
-// QK^T of block j+1 is issued before P_j V_j, so the tensor core works on S_{j+1} while the softmax
-// warps process S_j.
+// tc_attention_pair_kernel (used when the GQA group size H / Hkv is even): one CTA = 128 queries of
+// TWO query heads that share a KV head, so every K_j / V_j tile staged in shared memory feeds two
+// score tiles, and the tensor core always has the other tile's MMAs to run while one tile's
+// softmax is in progress.  grid = (H / 2, ceil(m / 128)), longest query tiles first.
+//   warp 0      TMA producer: both Q tiles once, then K_j [128 keys x 128] and V^T_j [128 x 128 keys]
+//   warp 1      TMEM owner and single-thread MMA issuer.  TMEM columns: S_0 | S_1 | O_0 | O_1
+//               (4 x 128 fp32 columns).  Per key block j and tile t:  O_t += P_t V_j  (A operand P_t
+//               read from TMEM, where it overwrites the first 64 columns of S_t), then
+//               S_t = Q_t K_{j+1}^T.
+//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1; one query row per thread: row
+//               maximum, p = 2^(s * log2(e)/sqrt(d) - max) with a lazily updated running maximum (O_t
+//               is rescaled in TMEM only when the maximum grows by more than 2^8), row sum, P_t
+//               written back to TMEM as packed bf16; at the end O_t / l goes to global memory.
+//
+// tc_attention_kernel (any group size): one CTA = 128 queries of one head, P_j staged through shared
+// memory; QK^T of block j+1 is issued before P_j V_j so the tensor core works on S_{j+1} while the
+// softmax warps process S_j.
 #include "spts_common.cuh"
 #include "tc_ptx.cuh"
 
@@ -300,6 +306,276 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// paired-head kernel
+// ---------------------------------------------------------------------------------------------
+constexpr int AP_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 softmax warps
+constexpr int AP_SMEM = 2 * TILE_BYTES /*Q_0, Q_1*/ + KV_STAGES * TILE_BYTES /*K*/ + KV_STAGES * TILE_BYTES /*V^T*/ +
+                        1024 + 256;
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+__global__ void __launch_bounds__(AP_THREADS, 1)
+tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                         const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sQ = base;                                  // two tiles
+  const uint32_t sK = sQ + 2 * TILE_BYTES;
+  const uint32_t sV = sK + KV_STAGES * TILE_BYTES;
+  const uint32_t bars = sV + KV_STAGES * TILE_BYTES;
+  const uint32_t q_full = bars;
+  const uint32_t k_full = bars + 8;          // [2 stages]
+  const uint32_t k_free = bars + 24;         // [2]
+  const uint32_t v_full = bars + 40;         // [2]
+  const uint32_t v_free = bars + 56;         // [2]
+  const uint32_t s_full = bars + 72;         // [2 tiles]  S_t of the next key block is complete
+  const uint32_t p_full = bars + 88;         // [2 tiles]  P_t written by its 128 softmax threads
+  const uint32_t o_full = bars + 104;        // [2 tiles]  last P_t V_j done
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + (bars - base) + 128);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int h0 = 2 * (int)blockIdx.x;                         // heads h0, h0 + 1 share a KV head
+  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;        // longest tiles first
+  const int kvh = h0 / (p.H / p.Hkv);
+  const int nblk = qt + 1;
+  const uint64_t t0 = globaltimer_ns();
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    mbar_init(q_full, 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(k_full + 8 * s, 1); mbar_init(k_free + 8 * s, 1);
+      mbar_init(v_full + 8 * s, 1); mbar_init(v_free + 8 * s, 1);
+      mbar_init(s_full + 8 * s, 1); mbar_init(p_full + 8 * s, 128); mbar_init(o_full + 8 * s, 1);
+    }
+    fence_mbar_init();
+    prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), AT_TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(q_full, 2 * TILE_BYTES);
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t) * TILE, qt * TILE);
+        tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t) * TILE + 64, qt * TILE);
+      }
+      bool ok = true;
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int s = j & 1;
+        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+        ok = mbar_wait(k_free + 8 * s, ph ^ 1, abort_flag, t0);
+        if (!ok) break;
+        mbar_expect_tx(k_full + 8 * s, TILE_BYTES);
+        tma_load_2d(sK + s * TILE_BYTES, &tmK, k_full + 8 * s, kvh * TILE, j * TILE);
+        tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, k_full + 8 * s, kvh * TILE + 64, j * TILE);
+        ok = mbar_wait(v_free + 8 * s, ph ^ 1, abort_flag, t0);
+        if (!ok) break;
+        mbar_expect_tx(v_full + 8 * s, TILE_BYTES);
+        tma_load_2d(sV + s * TILE_BYTES, &tmV, v_full + 8 * s, j * TILE, kvh * TILE);
+        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, v_full + 8 * s, j * TILE + 64, kvh * TILE);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(TILE, TILE);
+      // S_t = Q_t K_j^T
+      auto issue_qk = [&](int t, int j) {
+        const uint32_t kb = sK + (j & 1) * TILE_BYTES, qb = sQ + t * TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
+          mma_bf16(tmem_base + t * TILE, smem_desc_sw128(qb + off), smem_desc_sw128(kb + off), idesc, k > 0 ? 1u : 0u);
+        }
+      };
+      // O_t += P_t V_j, P_t read from the columns of S_t
+      auto issue_pv = [&](int t, int j) {
+        const uint32_t vb = sV + (j & 1) * TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
+          mma_bf16_tmem_a(tmem_base + 2 * TILE + t * TILE, tmem_base + t * TILE + k * 8, smem_desc_sw128(vb + off), idesc,
+                          (j > 0 || k > 0) ? 1u : 0u);
+        }
+      };
+      bool ok = mbar_wait(q_full, 0, abort_flag, t0);
+      if (ok) ok = mbar_wait(k_full, 0, abort_flag, t0);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        mma_commit(s_full);
+        issue_qk(1, 0);
+        mma_commit(s_full + 8);
+        mma_commit(k_free);
+      }
+      for (int j = 0; j < nblk && ok; ++j) {
+        const int sv = j & 1;
+        const bool more = j + 1 < nblk;
+        ok = mbar_wait(v_full + 8 * sv, (uint32_t)(j >> 1) & 1u, abort_flag, t0);
+        if (!ok) break;
+        if (more) {
+          ok = mbar_wait(k_full + 8 * ((j + 1) & 1), (uint32_t)((j + 1) >> 1) & 1u, abort_flag, t0);
+          if (!ok) break;
+        }
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          ok = mbar_wait(p_full + 8 * t, (uint32_t)j & 1u, abort_flag, t0);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(t, j);
+          if (more) {
+            issue_qk(t, j + 1);
+            mma_commit(s_full + 8 * t);       // also covers P_t V_j: O_t is quiescent when S_t arrives
+          } else {
+            mma_commit(o_full + 8 * t);
+          }
+        }
+        if (!ok) break;
+        mma_commit(v_free + 8 * sv);
+        if (more) mma_commit(k_free + 8 * ((j + 1) & 1));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax / rescale / epilogue
+    const int t = (warp - 2) >> 2;                     // tile (head h0 + t)
+    const int quarter = warp & 3;                      // TMEM lane quarter this warp may access
+    const int row = quarter * 32 + lane;
+    const int qi = qt * TILE + row;                    // compact query index
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const uint32_t tSt = tmem_base + t * TILE + lane_off;
+    const uint32_t tOt = tmem_base + 2 * TILE + t * TILE + lane_off;
+    const float sc = 0.08838834764831845f * 1.4426950408889634f;   // log2(e) / sqrt(128)
+    const float2 sc2 = make_float2(sc, sc);
+    float m_used = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nblk && ok; ++j) {
+      ok = mbar_wait(s_full + 8 * t, (uint32_t)j & 1u, abort_flag, t0);
+      if (!ok) break;
+      tc_fence_after();
+      const bool diag = (j == qt);
+      const int key0 = j * TILE;
+      // pass 1: row maximum of the raw scores
+      float bmax = -INFINITY;
+#pragma unroll 1
+      for (int c = 0; c < TILE; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(tSt + c, r);
+        tmem_ld_wait();
+        if (diag) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (key0 + c + i <= qi) bmax = fmaxf(bmax, __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) bmax = max3(bmax, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+        }
+      }
+      bmax *= sc;
+      float alpha = 1.0f;      // factor applied to O and l when the running maximum is replaced
+      if (bmax > m_used + RESCALE_THRESHOLD || m_used == -INFINITY) {
+        alpha = (m_used == -INFINITY) ? 0.0f : ex2(m_used - bmax);
+        m_used = bmax;
+      }
+      // S_t complete means P_t V_{j-1} has completed too, and P_t V_j cannot start before this thread's
+      // P arrives: O_t is safe to rescale here
+      if (j >= 1 && __any_sync(0xffffffffu, alpha != 1.0f)) {
+#pragma unroll 1
+        for (int c = 0; c < TILE; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tOt + c, r);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+          tmem_st32(tOt + c, r);
+        }
+      }
+      // pass 2: p = 2^(s * sc - m), row sum, bf16 pairs written over the first half of S_t
+      const float2 nm2 = make_float2(-m_used, -m_used);
+      float2 ps0 = make_float2(0.f, 0.f), ps1 = make_float2(0.f, 0.f);
+#pragma unroll 1
+      for (int c = 0; c < TILE; c += 32) {
+        uint32_t r[32], pk[16];
+        tmem_ld32(tSt + c, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          float2 x0 = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
+          float2 x1 = __ffma2_rn(make_float2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sc2, nm2);
+          if (diag) {
+            if (key0 + c + i > qi) x0.x = -INFINITY;
+            if (key0 + c + i + 1 > qi) x0.y = -INFINITY;
+            if (key0 + c + i + 2 > qi) x1.x = -INFINITY;
+            if (key0 + c + i + 3 > qi) x1.y = -INFINITY;
+          }
+          float2 e0 = make_float2(ex2(x0.x), ex2(x0.y));
+          float2 e1 = make_float2(ex2(x1.x), ex2(x1.y));
+          ps0 = __fadd2_rn(ps0, e0);
+          ps1 = __fadd2_rn(ps1, e1);
+          pk[i >> 1] = pack2(e0.x, e0.y);
+          pk[(i >> 1) + 1] = pack2(e1.x, e1.y);
+        }
+        tmem_st16(tSt + (c >> 1), pk);
+      }
+      l = l * alpha + ((ps0.x + ps0.y) + (ps1.x + ps1.y));
+      tmem_st_wait();
+      tc_fence_before();
+      mbar_arrive(p_full + 8 * t);
+    }
+    // ---- epilogue: O_t / l
+    if (ok) ok = mbar_wait(o_full + 8 * t, 0, abort_flag, t0);
+    if (ok) {
+      tc_fence_after();
+      const float inv = 1.0f / l;
+      bf16* orow = p.O + ((size_t)qi * p.H + (h0 + t)) * TILE;
+#pragma unroll 1
+      for (int c = 0; c < TILE; c += 32) {
+        uint32_t r[32];
+        tmem_ld32(tOt + c, r);
+        tmem_ld_wait();
+        if (qi < p.m) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint4 w;
+            w.x = pack2(__uint_as_float(r[g * 8 + 0]) * inv, __uint_as_float(r[g * 8 + 1]) * inv);
+            w.y = pack2(__uint_as_float(r[g * 8 + 2]) * inv, __uint_as_float(r[g * 8 + 3]) * inv);
+            w.z = pack2(__uint_as_float(r[g * 8 + 4]) * inv, __uint_as_float(r[g * 8 + 5]) * inv);
+            w.w = pack2(__uint_as_float(r[g * 8 + 6]) * inv, __uint_as_float(r[g * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c + g * 8) = w;
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) set_status(p.status, SPTS_ERR_TIMEOUT);
+    const uint64_t t1 = globaltimer_ns();
+    while (globaltimer_ns() - t1 < 200000ull) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, AT_TMEM_COLS);
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -322,6 +598,8 @@ spts_status tc_init(spts_ctx* ctx) {
   if (s != SPTS_OK) return s;
   if (cudaFuncSetAttribute(tc_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM) != cudaSuccess)
     return SPTS_ERR_CUDA;
+  if (cudaFuncSetAttribute(tc_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AP_SMEM) != cudaSuccess)
+    return SPTS_ERR_CUDA;
   return SPTS_OK;
 }
 
@@ -339,8 +617,13 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
   if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)m, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
   AttnParams p;
   p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.O = O; p.status = ctx->ws.status;
-  dim3 grid(d.n_q_heads, ceil_div(m, TILE));
-  tc_attention_kernel<<<grid, AT_THREADS, AT_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  if ((d.n_q_heads / d.n_kv_heads) % 2 == 0) {
+    dim3 grid(d.n_q_heads / 2, ceil_div(m, TILE));
+    tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  } else {
+    dim3 grid(d.n_q_heads, ceil_div(m, TILE));
+    tc_attention_kernel<<<grid, AT_THREADS, AT_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  }
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }
