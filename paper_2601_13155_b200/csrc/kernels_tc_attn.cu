@@ -313,6 +313,26 @@ constexpr int AP_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 softma
 constexpr int AP_SMEM = 2 * TILE_BYTES /*Q_0, Q_1*/ + KV_STAGES * TILE_BYTES /*K*/ + KV_STAGES * TILE_BYTES /*V^T*/ +
                         1024 + 256;
 
+constexpr int POLY_PAIRS = 2;                // of every 4 element pairs, how many take the polynomial 2^x
+
+// 2^x for x in [-126, 2^22) on the FMA pipe: x = n + f with n = round(x), |f| <= 1/2;
+// 2^f by a cubic (relative error 7.5e-5, far below the bf16 rounding of P), then n added to the
+// exponent field.  Arguments below -126 are clamped (their result is ~1e-38, i.e. zero in the sum).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  const float magic = 12582912.f;             // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 t = __fadd2_rn(x, make_float2(magic, magic));
+  const float2 n = __fadd2_rn(t, make_float2(-magic, -magic));
+  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
+  float2 q = __ffma2_rn(make_float2(0.0551714264f, 0.0551714264f), f, make_float2(0.242610544f, 0.242610544f));
+  q = __ffma2_rn(q, f, make_float2(0.693260968f, 0.693260968f));
+  q = __ffma2_rn(q, f, make_float2(0.999928117f, 0.999928117f));
+  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
+  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
+  return q;
+}
+
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -469,23 +489,24 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       tc_fence_after();
       const bool diag = (j == qt);
       const int key0 = j * TILE;
-      // pass 1: row maximum of the raw scores
-      float bmax = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < TILE; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(tSt + c, r);
-        tmem_ld_wait();
-        if (diag) {
+      // the whole score row into registers: four loads in flight, one wait
+      uint32_t r[TILE];
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (key0 + c + i <= qi) bmax = fmaxf(bmax, __uint_as_float(r[i]));
-        } else {
+      for (int c = 0; c < TILE; c += 32) tmem_ld32(tSt + c, r + c);
+      tmem_ld_wait();
+      if (diag) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) bmax = max3(bmax, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-        }
+        for (int i = 0; i < TILE; ++i)
+          if (key0 + i > qi) r[i] = 0xFF800000u;        // -inf: keys after the query
       }
-      bmax *= sc;
+      // row maximum of the raw scores (four independent chains)
+      float bm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int i = 0; i < TILE; i += 8) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) bm[u] = max3(bm[u], __uint_as_float(r[i + 2 * u]), __uint_as_float(r[i + 2 * u + 1]));
+      }
+      const float bmax = fmaxf(fmaxf(bm[0], bm[1]), fmaxf(bm[2], bm[3])) * sc;
       float alpha = 1.0f;      // factor applied to O and l when the running maximum is replaced
       if (bmax > m_used + RESCALE_THRESHOLD || m_used == -INFINITY) {
         alpha = (m_used == -INFINITY) ? 0.0f : ex2(m_used - bmax);
@@ -496,41 +517,42 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       if (j >= 1 && __any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll 1
         for (int c = 0; c < TILE; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(tOt + c, r);
+          uint32_t o[32];
+          tmem_ld32(tOt + c, o);
           tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-          tmem_st32(tOt + c, r);
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+          tmem_st32(tOt + c, o);
         }
       }
-      // pass 2: p = 2^(s * sc - m), row sum, bf16 pairs written over the first half of S_t
+      // p = 2^(s * sc - m), row sum, bf16 pairs written over the first half of S_t.  The exponential
+      // unit is the scarce resource (a quarter of a warp per clock), so outside the diagonal block
+      // POLY_PAIRS of every four element pairs are evaluated on the FMA pipe instead.
       const float2 nm2 = make_float2(-m_used, -m_used);
-      float2 ps0 = make_float2(0.f, 0.f), ps1 = make_float2(0.f, 0.f);
-#pragma unroll 1
-      for (int c = 0; c < TILE; c += 32) {
-        uint32_t r[32], pk[16];
-        tmem_ld32(tSt + c, r);
-        tmem_ld_wait();
+      float2 ps[4];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          float2 x0 = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
-          float2 x1 = __ffma2_rn(make_float2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sc2, nm2);
-          if (diag) {
-            if (key0 + c + i > qi) x0.x = -INFINITY;
-            if (key0 + c + i + 1 > qi) x0.y = -INFINITY;
-            if (key0 + c + i + 2 > qi) x1.x = -INFINITY;
-            if (key0 + c + i + 3 > qi) x1.y = -INFINITY;
-          }
-          float2 e0 = make_float2(ex2(x0.x), ex2(x0.y));
-          float2 e1 = make_float2(ex2(x1.x), ex2(x1.y));
-          ps0 = __fadd2_rn(ps0, e0);
-          ps1 = __fadd2_rn(ps1, e1);
-          pk[i >> 1] = pack2(e0.x, e0.y);
-          pk[(i >> 1) + 1] = pack2(e1.x, e1.y);
+      for (int u = 0; u < 4; ++u) ps[u] = make_float2(0.f, 0.f);
+      uint32_t pk[TILE / 2];
+      if (diag) {
+#pragma unroll
+        for (int i = 0; i < TILE; i += 2) {
+          float2 x = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
+          float2 e = make_float2(ex2(x.x), ex2(x.y));
+          ps[(i >> 1) & 3] = __fadd2_rn(ps[(i >> 1) & 3], e);
+          pk[i >> 1] = pack2(e.x, e.y);
         }
-        tmem_st16(tSt + (c >> 1), pk);
+      } else {
+#pragma unroll
+        for (int i = 0; i < TILE; i += 2) {
+          float2 x = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
+          float2 e = (((i >> 1) & 3) < POLY_PAIRS) ? exp2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
+          ps[(i >> 1) & 3] = __fadd2_rn(ps[(i >> 1) & 3], e);
+          pk[i >> 1] = pack2(e.x, e.y);
+        }
       }
+#pragma unroll
+      for (int c = 0; c < TILE / 2; c += 16) tmem_st16(tSt + c, pk + c);
+      const float2 ps0 = __fadd2_rn(ps[0], ps[1]), ps1 = __fadd2_rn(ps[2], ps[3]);
       l = l * alpha + ((ps0.x + ps0.y) + (ps1.x + ps1.y));
       tmem_st_wait();
       tc_fence_before();
