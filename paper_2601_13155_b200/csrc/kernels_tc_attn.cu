@@ -6,13 +6,14 @@
 // TWO query heads that share a KV head, so every K_j / V_j tile staged in shared memory feeds two
 // score tiles, and the tensor core always has the other tile's MMAs to run while one tile's
 // softmax is in progress.  grid = (H / 2, ceil(m / 128)), longest query tiles first.
-//   warp 0      TMA producer: both Q tiles once, then K_j [128 keys x 128] and V^T_j [128 x 128 keys]
+//   warp 0      TMA producer: both Q tiles and K_0 once, then per key block the pair (V^T_j, K_{j+1})
+//               [128 x 128 each] under one barrier
 //   warp 1      TMEM owner and single-thread MMA issuer.  TMEM columns: S_0 | S_1 | O_0 | O_1
 //               (4 x 128 fp32 columns).  Per key block j and tile t:  O_t += P_t V_j  (A operand P_t
-//               read from TMEM, where it overwrites the first 64 columns of S_t), then
-//               S_t = Q_t K_{j+1}^T.
-//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1; one query row per thread: row
-//               maximum, p = 2^(s * log2(e)/sqrt(d) - max) with a lazily updated running maximum (O_t
+//               read from TMEM, where it overwrites the first 64 columns of S_t; issued piece by
+//               piece as the softmax warps deliver it), then S_t = Q_t K_{j+1}^T.
+//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1; one query row per thread, the whole score
+//               row in registers: row maximum, p = 2^(s * log2(e)/sqrt(d) - max) with a lazily updated running maximum (O_t
 //               is rescaled in TMEM only when the maximum grows by more than 2^8), row sum, P_t
 //               written back to TMEM as packed bf16; at the end O_t / l goes to global memory.
 //
@@ -313,25 +314,7 @@ constexpr int AP_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 softma
 constexpr int AP_SMEM = 2 * TILE_BYTES /*Q_0, Q_1*/ + KV_STAGES * TILE_BYTES /*K*/ + KV_STAGES * TILE_BYTES /*V^T*/ +
                         1024 + 256;
 
-constexpr int POLY_PAIRS = 2;                // of every 4 element pairs, how many take the polynomial 2^x
-
-// 2^x for x in [-126, 2^22) on the FMA pipe: x = n + f with n = round(x), |f| <= 1/2;
-// 2^f by a cubic (relative error 7.5e-5, far below the bf16 rounding of P), then n added to the
-// exponent field.  Arguments below -126 are clamped (their result is ~1e-38, i.e. zero in the sum).
-__device__ __forceinline__ float2 exp2_poly2(float2 x) {
-  const float magic = 12582912.f;             // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-  x.x = fmaxf(x.x, -126.f);
-  x.y = fmaxf(x.y, -126.f);
-  const float2 t = __fadd2_rn(x, make_float2(magic, magic));
-  const float2 n = __fadd2_rn(t, make_float2(-magic, -magic));
-  const float2 f = __fadd2_rn(x, make_float2(-n.x, -n.y));
-  float2 q = __ffma2_rn(make_float2(0.0551714264f, 0.0551714264f), f, make_float2(0.242610544f, 0.242610544f));
-  q = __ffma2_rn(q, f, make_float2(0.693260968f, 0.693260968f));
-  q = __ffma2_rn(q, f, make_float2(0.999928117f, 0.999928117f));
-  q.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
-  q.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
-  return q;
-}
+constexpr int P_PARTS = 2;                   // pieces (64 keys each) in which a P tile is handed to the MMA warp
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
@@ -349,13 +332,13 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   const uint32_t sV = sK + KV_STAGES * TILE_BYTES;
   const uint32_t bars = sV + KV_STAGES * TILE_BYTES;
   const uint32_t q_full = bars;
-  const uint32_t k_full = bars + 8;          // [2 stages]
-  const uint32_t k_free = bars + 24;         // [2]
-  const uint32_t v_full = bars + 40;         // [2]
-  const uint32_t v_free = bars + 56;         // [2]
-  const uint32_t s_full = bars + 72;         // [2 tiles]  S_t of the next key block is complete
-  const uint32_t p_full = bars + 88;         // [2 tiles]  P_t written by its 128 softmax threads
-  const uint32_t o_full = bars + 104;        // [2 tiles]  last P_t V_j done
+  // K and V travel in pairs: stage j & 1 holds V_j and K_{j+1}, the two tiles key block j's MMAs
+  // (P_t V_j, then Q_t K_{j+1}^T) read, so one wait and one release per block serve both
+  const uint32_t kv_full = bars + 8;         // [2 stages]
+  const uint32_t kv_free = bars + 24;        // [2]
+  const uint32_t s_full = bars + 40;         // [2 tiles]  S_t of the next key block is complete
+  const uint32_t o_full = bars + 56;         // [2 tiles]  last P_t V_j done
+  const uint32_t p_full = bars + 72;         // [2 tiles][P_PARTS]  a piece of P_t written by its 128 softmax threads
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + (bars - base) + 128);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -371,9 +354,9 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     *abort_flag = 0;
     mbar_init(q_full, 1);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(k_full + 8 * s, 1); mbar_init(k_free + 8 * s, 1);
-      mbar_init(v_full + 8 * s, 1); mbar_init(v_free + 8 * s, 1);
-      mbar_init(s_full + 8 * s, 1); mbar_init(p_full + 8 * s, 128); mbar_init(o_full + 8 * s, 1);
+      mbar_init(kv_full + 8 * s, 1); mbar_init(kv_free + 8 * s, 1);
+      mbar_init(s_full + 8 * s, 1); mbar_init(o_full + 8 * s, 1);
+      for (int part = 0; part < P_PARTS; ++part) mbar_init(p_full + 8 * (P_PARTS * s + part), 128);
     }
     fence_mbar_init();
     prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
@@ -389,26 +372,29 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
 
   if (warp == 0) {
     if (lane == 0) {
-      mbar_expect_tx(q_full, 2 * TILE_BYTES);
+      mbar_expect_tx(q_full, 3 * TILE_BYTES);               // both Q tiles and K_0 (K_j sits in slot (j + 1) & 1)
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
         tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t) * TILE, qt * TILE);
         tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t) * TILE + 64, qt * TILE);
       }
+      tma_load_2d(sK + TILE_BYTES, &tmK, q_full, kvh * TILE, 0);
+      tma_load_2d(sK + TILE_BYTES + SLAB_BYTES, &tmK, q_full, kvh * TILE + 64, 0);
       bool ok = true;
       for (int j = 0; j < nblk && ok; ++j) {
         const int s = j & 1;
-        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-        ok = mbar_wait(k_free + 8 * s, ph ^ 1, abort_flag, t0);
+        const bool more = j + 1 < nblk;
+        // stage 1 starts occupied (its K slot holds K_0) and is first released after Q_t K_0^T, so its
+        // releases run one ahead of stage 0's
+        ok = mbar_wait(kv_free + 8 * s, ((uint32_t)(j >> 1) & 1u) ^ (uint32_t)(s ^ 1), abort_flag, t0);
         if (!ok) break;
-        mbar_expect_tx(k_full + 8 * s, TILE_BYTES);
-        tma_load_2d(sK + s * TILE_BYTES, &tmK, k_full + 8 * s, kvh * TILE, j * TILE);
-        tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, k_full + 8 * s, kvh * TILE + 64, j * TILE);
-        ok = mbar_wait(v_free + 8 * s, ph ^ 1, abort_flag, t0);
-        if (!ok) break;
-        mbar_expect_tx(v_full + 8 * s, TILE_BYTES);
-        tma_load_2d(sV + s * TILE_BYTES, &tmV, v_full + 8 * s, j * TILE, kvh * TILE);
-        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, v_full + 8 * s, j * TILE + 64, kvh * TILE);
+        mbar_expect_tx(kv_full + 8 * s, more ? 2 * TILE_BYTES : TILE_BYTES);
+        tma_load_2d(sV + s * TILE_BYTES, &tmV, kv_full + 8 * s, j * TILE, kvh * TILE);
+        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, kv_full + 8 * s, j * TILE + 64, kvh * TILE);
+        if (more) {
+          tma_load_2d(sK + s * TILE_BYTES, &tmK, kv_full + 8 * s, kvh * TILE, (j + 1) * TILE);
+          tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, kv_full + 8 * s, kvh * TILE + 64, (j + 1) * TILE);
+        }
       }
     }
   } else if (warp == 1) {
@@ -416,48 +402,50 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       constexpr uint32_t idesc = idesc_bf16(TILE, TILE);
       // S_t = Q_t K_j^T
       auto issue_qk = [&](int t, int j) {
-        const uint32_t kb = sK + (j & 1) * TILE_BYTES, qb = sQ + t * TILE_BYTES;
+        const uint32_t kb = sK + ((j + 1) & 1) * TILE_BYTES, qb = sQ + t * TILE_BYTES;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
           mma_bf16(tmem_base + t * TILE, smem_desc_sw128(qb + off), smem_desc_sw128(kb + off), idesc, k > 0 ? 1u : 0u);
         }
       };
-      // O_t += P_t V_j, P_t read from the columns of S_t
-      auto issue_pv = [&](int t, int j) {
+      // O_t += P_t V_j for the keys of piece `part`, P_t read from the columns of S_t
+      auto issue_pv = [&](int t, int j, int part) {
         const uint32_t vb = sV + (j & 1) * TILE_BYTES;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
+        for (int kk = 0; kk < 8 / P_PARTS; ++kk) {
+          const int k = part * (8 / P_PARTS) + kk;
           const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
           mma_bf16_tmem_a(tmem_base + 2 * TILE + t * TILE, tmem_base + t * TILE + k * 8, smem_desc_sw128(vb + off), idesc,
                           (j > 0 || k > 0) ? 1u : 0u);
         }
       };
       bool ok = mbar_wait(q_full, 0, abort_flag, t0);
-      if (ok) ok = mbar_wait(k_full, 0, abort_flag, t0);
       if (ok) {
         tc_fence_after();
         issue_qk(0, 0);
         mma_commit(s_full);
         issue_qk(1, 0);
         mma_commit(s_full + 8);
-        mma_commit(k_free);
+        mma_commit(kv_free + 8);             // K_0's slot may be refilled (with K_2) once these are done
       }
       for (int j = 0; j < nblk && ok; ++j) {
         const int sv = j & 1;
         const bool more = j + 1 < nblk;
-        ok = mbar_wait(v_full + 8 * sv, (uint32_t)(j >> 1) & 1u, abort_flag, t0);
+        ok = mbar_wait(kv_full + 8 * sv, (uint32_t)(j >> 1) & 1u, abort_flag, t0);
         if (!ok) break;
-        if (more) {
-          ok = mbar_wait(k_full + 8 * ((j + 1) & 1), (uint32_t)((j + 1) >> 1) & 1u, abort_flag, t0);
-          if (!ok) break;
-        }
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          ok = mbar_wait(p_full + 8 * t, (uint32_t)j & 1u, abort_flag, t0);
+          // P_t arrives in P_PARTS pieces (one barrier each), so the first MMAs of P_t V_j run while
+          // the softmax warps are still computing the exponentials of the later keys
+#pragma unroll
+          for (int part = 0; part < P_PARTS; ++part) {
+            ok = mbar_wait(p_full + 8 * (P_PARTS * t + part), (uint32_t)j & 1u, abort_flag, t0);
+            if (!ok) break;
+            tc_fence_after();
+            issue_pv(t, j, part);
+          }
           if (!ok) break;
-          tc_fence_after();
-          issue_pv(t, j);
           if (more) {
             issue_qk(t, j + 1);
             mma_commit(s_full + 8 * t);       // also covers P_t V_j: O_t is quiescent when S_t arrives
@@ -466,8 +454,7 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           }
         }
         if (!ok) break;
-        mma_commit(v_free + 8 * sv);
-        if (more) mma_commit(k_free + 8 * ((j + 1) & 1));
+        mma_commit(kv_free + 8 * sv);
       }
     }
   } else {
@@ -525,38 +512,32 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
           tmem_st32(tOt + c, o);
         }
       }
-      // p = 2^(s * sc - m), row sum, bf16 pairs written over the first half of S_t.  The exponential
-      // unit is the scarce resource (a quarter of a warp per clock), so outside the diagonal block
-      // POLY_PAIRS of every four element pairs are evaluated on the FMA pipe instead.
+      // p = 2^(s * sc - m), row sum, bf16 pairs written over the first half of S_t, handed over in
+      // P_PARTS pieces.  The first piece's wait::st also covers the O_t rescale stores above.
       const float2 nm2 = make_float2(-m_used, -m_used);
       float2 ps[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) ps[u] = make_float2(0.f, 0.f);
-      uint32_t pk[TILE / 2];
-      if (diag) {
 #pragma unroll
-        for (int i = 0; i < TILE; i += 2) {
-          float2 x = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
-          float2 e = make_float2(ex2(x.x), ex2(x.y));
+      for (int part = 0; part < P_PARTS; ++part) {
+        constexpr int PE = TILE / P_PARTS;             // elements per piece
+        uint32_t pk[PE / 2];
+#pragma unroll
+        for (int i = 0; i < PE; i += 2) {
+          const int e0 = part * PE + i;
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[e0]), __uint_as_float(r[e0 + 1])), sc2, nm2);
+          const float2 e = make_float2(ex2(x.x), ex2(x.y));
           ps[(i >> 1) & 3] = __fadd2_rn(ps[(i >> 1) & 3], e);
           pk[i >> 1] = pack2(e.x, e.y);
         }
-      } else {
 #pragma unroll
-        for (int i = 0; i < TILE; i += 2) {
-          float2 x = __ffma2_rn(make_float2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2);
-          float2 e = (((i >> 1) & 3) < POLY_PAIRS) ? exp2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
-          ps[(i >> 1) & 3] = __fadd2_rn(ps[(i >> 1) & 3], e);
-          pk[i >> 1] = pack2(e.x, e.y);
-        }
+        for (int c = 0; c < PE / 2; c += 16) tmem_st16(tSt + part * (PE / 2) + c, pk + c);
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(p_full + 8 * (P_PARTS * t + part));
       }
-#pragma unroll
-      for (int c = 0; c < TILE / 2; c += 16) tmem_st16(tSt + c, pk + c);
       const float2 ps0 = __fadd2_rn(ps[0], ps[1]), ps1 = __fadd2_rn(ps[2], ps[3]);
       l = l * alpha + ((ps0.x + ps0.y) + (ps1.x + ps1.y));
-      tmem_st_wait();
-      tc_fence_before();
-      mbar_arrive(p_full + 8 * t);
     }
     // ---- epilogue: O_t / l
     if (ok) ok = mbar_wait(o_full + 8 * t, 0, abort_flag, t0);
