@@ -4,14 +4,17 @@
 One step = one whole prefill of the 32-layer LLaMA-3.1-8B-shaped model (random-init weights,
 synthetic hidden states with heavy tokens) through Algorithm 1: per layer PAP score, top-k,
 reduced attention, LTP score, top-k, reduced FFN; stage-end pruning; first-token head.
-The default workload is BASELINE config 3 (32768-token prompt, four MSDP stages).
+The default workload is BASELINE config 3 (32768-token prompt, four MSDP stages); its line also
+carries `ctx_128k`, the same measurement on config 4 (131072 tokens, one timed step).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2|cfg5] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `value` = prompt tokens / second over all replicas with inputs
 resident in HBM; `e2e` = the same through host buffers (pinned H2D of the prompt's hidden states,
 D2H of the first token) every step; `dense` = the same code with skipping disabled.
-More than one GPU = independent replicas (the path has no inter-GPU exchange).
+`--workload cfg5` instead times whole requests (prefill + greedy decoding against the compressed
+caches) over a keep-ratio sweep.  More than one GPU = independent replicas (the path has no
+inter-GPU exchange).
 """
 from __future__ import annotations
 
@@ -35,7 +38,9 @@ def parse():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="spts", choices=["spts", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--no-128k", action="store_true", help="skip the 131072-token measurement added to the cfg3 line")
+    ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="also print a per-operation table to stderr")
@@ -124,7 +129,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2601_13155_b200 import synth
-    w = synth.workload(args.workload)
+    w = synth.workload("cfg3" if args.workload == "cfg5" else args.workload)
     vals = []
     for i in range(args.warmup + args.steps):
         tps, cores, desc, dt = oracle_sample(w)
@@ -168,7 +173,139 @@ def main():
         build.build()
     rep.barrier()
 
-    w = synth.workload(args.workload)
+    if args.workload == "cfg5":
+        line = generation_line(args, rep, dev)
+    else:
+        line = prefill_line(args, rep, dev, args.workload, args.steps, max(args.warmup, 3), 2, True)
+        if args.workload == "cfg3" and not args.no_128k and not args.layers:
+            # the same measurement at the longest context (BASELINE config 4), kernels already warm
+            torch.cuda.empty_cache()
+            sub = prefill_line(args, rep, dev, "cfg4", 1, 1, 0, False)
+            if rank == 0:
+                line["ctx_128k"] = {k: sub[k] for k in ("value", "unit", "ms_per_step", "ttft_ms", "steps", "warmup", "config",
+                                                        "dense", "roofline", "algorithmic_tflop_per_step",
+                                                        "achieved_tflops_whole_step", "breakdown_ms", "gpu_launches")}
+    if rank == 0:
+        print(json.dumps(line))
+    rep.close()
+
+
+def generation_line(args, rep, dev):
+    """BASELINE config 5: a 32768-token prompt is prefilled (Algorithm 1), then `--decode-steps` tokens are decoded
+    greedily against the per-layer compressed caches; repeated for keep ratios 1.0 / 0.7 / 0.5 / 0.3 (attention
+    and FFN budgets = ceil(keep * prompt), MSDP stages as in config 3) and once with skipping disabled.
+    value = generated + prompt tokens per second of the whole request at keep 0.5."""
+    import torch
+    from paper_2601_13155_b200 import binding, schedule, synth
+    rank, world = rep.rank, rep.world
+    w = synth.workload("cfg3")
+    shape = w.shape
+    L, N, T = shape.n_layers, w.n_tokens, args.decode_steps
+    layers = []
+    for l in range(L):
+        t = synth.device_layer_weights(shape, w.seed, l, dev)
+        lw = binding.LayerWeights.__new__(binding.LayerWeights)
+        lw.t = t
+        lw.c = binding.LayerWeightsC(**{n: t[n].data_ptr() for n in binding.WEIGHT_NAMES})
+        layers.append(lw)
+    hw = synth.device_head_weights(shape, w.seed, dev)
+    model = binding.Model(layers, hw["lm_head"], hw["embed"])
+    X0, _ = synth.device_hidden_states(w, dev)
+    lib = binding.Spts(shape, max_seq=N, device=dev)
+    cache = binding.KvCache(shape, L, N + T, dev)
+    X, Xa = torch.empty_like(X0), torch.empty_like(X0)
+    ar = torch.arange(N, dtype=torch.int32, device=dev)
+    pos, orig, pa, oa = ar.clone(), ar.clone(), ar.clone(), ar.clone()
+    tok = torch.zeros(1, dtype=torch.int32, device=dev)
+    logits = torch.empty(shape.vocab, dtype=torch.float32, device=dev)
+
+    def request(plan, steps):
+        """One request; returns (prefill ms, decode ms, first-step logits, generated tokens, cached token-layers)."""
+        cache.reset()
+        X.copy_(X0)
+        pos.copy_(ar)
+        orig.copy_(ar)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        rep.barrier()
+        ev[0].record()
+        lib.prefill(model, plan, X, pos, orig, Xa, pa, oa, cache, token_out=tok)
+        ev[1].record()
+        t_in = int(tok.item())                      # greedy decoding reads every token back
+        kv = sum(cache.length(l) for l in range(L))
+        toks, first = [t_in], None
+        for i in range(steps):
+            lib.decode_step(model, cache, N + i, token_in=t_in, logits_out=logits if i == 0 else None, token_out=tok)
+            if i == 0:
+                first = logits.clone()
+            t_in = int(tok.item())
+            toks.append(t_in)
+        ev[2].record()
+        rep.barrier()
+        return ev[0].elapsed_time(ev[1]), ev[1].elapsed_time(ev[2]), first, toks, kv
+
+    def plan_for(keep):
+        return schedule.workload_plan(w, keep_attn=keep, keep_ffn=keep)
+
+    request(plan_for(0.5), 8)                        # warm-up
+    request(plan_for(0.5), 8)
+    request(schedule.workload_plan(w, dense=True), 8)
+    lib.profile_begin(14)
+    pd, dd, lg_d, tk_d, kv_d = request(schedule.workload_plan(w, dense=True), T)
+    prof_d = lib.profile_end()
+    sweep = {}
+    for keep in (1.0, 0.7, 0.5, 0.3):
+        lib.profile_begin(14)
+        pm, dm, lg, tk, kv = request(plan_for(keep), T)
+        prof = lib.profile_end()["decode"]
+        dev_l2 = float((lg - lg_d).norm() / lg_d.norm())
+        match = float(sum(a == b for a, b in zip(tk, tk_d)) / len(tk))
+        sweep[str(keep)] = {"ttft_ms": pm, "decode_ms_per_token": dm / T, "request_ms": pm + dm,
+                            "tokens_per_s": (N + T) * world / ((pm + dm) * 1e-3),
+                            "decode_tokens_per_s": T * world / (dm * 1e-3),
+                            "decode_kernel_gbs": prof["bytes"] / max(prof["ms"], 1e-9) / 1e6,
+                            "kv_token_layers": kv, "kv_vs_dense": kv / kv_d,
+                            "first_logits_rel_l2_vs_dense": dev_l2, "token_match_vs_dense": match,
+                            "speedup_vs_dense": (pd + dd) / (pm + dm)}
+    status = lib.device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+    peaks = {}
+    pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk_path):
+        peaks = json.load(open(pk_path))
+    peak = peaks.get("hbm_gbs", 6650.0)
+    dk = prof_d["decode"]
+    ach = dk["bytes"] / max(dk["ms"], 1e-9) / 1e6
+    mid = sweep["0.5"]
+    line = None
+    if rank == 0:
+        line = {"metric": "e2e_generation_tokens_per_s", "value": mid["tokens_per_s"], "unit": "tokens/s", "n_gpus": world,
+                "steps": 1, "warmup": 3, "ms_per_step": mid["request_ms"], "ttft_ms": mid["ttft_ms"],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": f"cfg5: {L}-layer LLaMA-3.1-8B shape, prompt {N} prefilled with SPTS (keep 0.5, MSDP "
+                                       f"stages of cfg3), then {T} greedy decode steps, vocab {shape.vocab}",
+                           "global_batch": world, "seq_len": N, "parallelism": f"replicas x{world}",
+                           "l2": "15 GB of weights streamed per decode step"},
+                "dense": {"ttft_ms": pd, "decode_ms_per_token": dd / T, "request_ms": pd + dd,
+                          "tokens_per_s": (N + T) * world / ((pd + dd) * 1e-3), "kv_token_layers": kv_d},
+                "keep_sweep": sweep,
+                "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                             "traffic": None, "kernel": "decode step (all layers, dense arm)", "launches": dk["calls"],
+                             "ms_per_launch": dk["ms"] / dk["calls"],
+                             "peak_source": "measured (copy)" if peaks else "fallback"},
+                "gpu_launches": int(lib.launch_count())}
+    lib.close()
+    return line
+
+
+def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
+    """Times `steps` whole prefills of workload `wname` (after `warmup`), the same through host buffers, and the
+    dense arm; returns the JSON line as a dict (rank 0) or None."""
+    import torch
+    from paper_2601_13155_b200 import binding, schedule, synth
+    rank, world = rep.rank, rep.world
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = synth.workload(wname)
     shape = w.shape
     if args.layers:
         from dataclasses import replace
@@ -229,7 +366,7 @@ def main():
         prof = lib.profile_end() if profile_op else {}
         return rep.max_over_ranks(ms), lib.launch_count() - l0, prof
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         step(plan)
     status = lib.device_status()
     if status != 0:
@@ -244,20 +381,20 @@ def main():
 
     clocks = ClockSampler(local)
     clocks.start()
-    ms, launches, prof = timed(plan, args.steps, profile_op=dom_id)
+    ms, launches, prof = timed(plan, steps, profile_op=dom_id)
     clk = clocks.stop()
-    ms_step = ms / args.steps
+    ms_step = ms / steps
     value = N * world / (ms_step * 1e-3)
 
-    ms_e2e, _, _ = timed(plan, args.steps, from_host=True)
-    e2e = N * world / (ms_e2e / args.steps * 1e-3)
+    ms_e2e, _, _ = timed(plan, steps, from_host=True)
+    e2e = N * world / (ms_e2e / steps * 1e-3)
 
     dense = None
     if not args.no_dense:
-        for _ in range(2):
+        for _ in range(dense_warmup):
             step(plan_dense)
-        ms_d, _, _ = timed(plan_dense, max(1, args.steps))
-        ms_d /= max(1, args.steps)
+        ms_d, _, _ = timed(plan_dense, max(1, steps))
+        ms_d /= max(1, steps)
         dense = {"value": N * world / (ms_d * 1e-3), "unit": "tokens/s", "ms_per_step": ms_d,
                  "ttft_ms": ms_d, "speedup_spts_vs_dense": ms_d / ms_step}
     status = lib.device_status()
@@ -286,11 +423,11 @@ def main():
                 "peak_source": "measured (copy)" if peaks else "fallback"}
 
     total_flops = sum(v["flops"] for v in table.values())
+    line = None
     if rank == 0:
-        tps_cpu, cores, desc, _ = oracle_sample(w)
         line = {
-            "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ttft_ms": ms_step, "higher_is_better": True,
+            "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms_step, "ttft_ms": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": {"workload": f"{w.name}: {L}-layer LLaMA-3.1-8B shape, prompt {N}, MSDP stages at layers "
@@ -299,11 +436,10 @@ def main():
                        "global_batch": world, "seq_len": N, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (14 GB of weights streamed per step)"},
             "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": int(X0_host.numel() * X0_host.element_size()),
-                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / args.steps},
+                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / steps},
             "gpu_launches": int(launches),
             "clocks": clk,
             "roofline": roof,
-            "cpu_baseline": {"value": tps_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc},
             "dense": dense,
             "algorithmic_tflop_per_step": total_flops / 1e12,
             "achieved_tflops_whole_step": total_flops / 1e12 / (ms_step * 1e-3),
@@ -314,8 +450,12 @@ def main():
                 tf = v["flops"] / max(v["ms"], 1e-9) / 1e9
                 gb = v["bytes"] / max(v["ms"], 1e-9) / 1e6
                 sys.stderr.write(f"{k:12s} {v['ms']:9.3f} ms  {v['calls']:4d} calls  {tf:8.1f} TFLOP/s  {gb:8.1f} GB/s\n")
-        print(json.dumps(line))
-    rep.close()
+        if with_cpu:
+            tps_cpu, cores, desc, _ = oracle_sample(w)
+            line["cpu_baseline"] = {"value": tps_cpu, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": desc}
+    lib.close()
+    del lib, cache, model, layers, hw, X, Xa, X0, X0_host
+    return line
 
 
 if __name__ == "__main__":
