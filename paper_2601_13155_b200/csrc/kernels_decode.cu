@@ -1,7 +1,17 @@
 // Decode step (Algorithm 1 outside the prefill phase): one new token runs every layer densely
-// against that layer's compressed KV cache plus itself.  Batch-1 decode streams every weight
-// once, so all kernels here are HBM-bound matrix-vector products with 16-byte loads; the
-// residual vector lives in fp32 scratch and is rounded through the storage type at the same
+// against that layer's compressed KV cache plus itself.  Batch-1 decode streams every weight and
+// every cached key / value once, so everything here is HBM-bound; the kernels are built to keep
+// many 16-byte loads in flight per thread:
+//
+//   gemv core    one CTA = 8 weight rows (16 for the gate / up pair); its 8 warps split K, every
+//                lane issues the loads of all rows of a K-chunk together, partial dots meet in
+//                shared memory.  RMSNorm is an fp32 scale computed from the same pass over x.
+//   epilogues    q / k / v projection with rotary embedding and the cache append fused in;
+//                SwiGLU of the gate / up pair; residual update (O and down projections).
+//   attention    one CTA = one KV head x one slice of the cache, serving the whole GQA group of
+//                query heads at once (each cached row is read once), online softmax, then a
+//                combine kernel over the slices.
+// The residual vector lives in fp32 scratch and is rounded through the storage type at the same
 // points as the prefill path.
 #include "spts_common.cuh"
 
@@ -15,11 +25,11 @@ template <> struct DV<bf16> { static constexpr int N = 8; };
 
 template <typename T> __device__ __forceinline__ void ld16(const T* p, float* out);
 template <> __device__ __forceinline__ void ld16<float>(const float* p, float* out) {
-  float4 v = *reinterpret_cast<const float4*>(p);
+  float4 v = __ldg(reinterpret_cast<const float4*>(p));
   out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
 }
 template <> __device__ __forceinline__ void ld16<bf16>(const bf16* p, float* out) {
-  uint4 v = *reinterpret_cast<const uint4*>(p);
+  uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
   const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -41,70 +51,162 @@ __global__ void vec_store_kernel(const float* __restrict__ x, int D, T* __restri
   if (i < D) out[i] = from_f32<T>(x[i]);
 }
 
-// out[j] (op)= scale * sum_k xin[k] W[j, k], with scale = rstd(xin) when NORM.
-// RESID: out[j] = round(out[j] + dot).  One warp per output row; xin staged in shared memory.
-template <typename T, bool NORM, bool RESID>
-__global__ void __launch_bounds__(256)
-gemv_kernel(const T* __restrict__ W, int rows, int K, const float* __restrict__ xin, float eps,
-            float* __restrict__ out) {
+constexpr int GV_THREADS = 256;   // 8 warps
+constexpr int GV_WARPS = 8;
+
+// dots[r] = sum_k x[k] * row_r[k] for R rows given by pointer, and sumsq = sum_k x[k]^2.
+// Results are valid in shared memory (dots_out[0..R), *ss_out) for all threads after the call.
+template <typename T, int R>
+__device__ __forceinline__ void gemv_rows(const T* (&rowp)[R], int K, const float* __restrict__ x,
+                                          float* dots_out, float* ss_out) {
   constexpr int V = DV<T>::N;
-  extern __shared__ float xs[];
-  __shared__ float red[8];
-  __shared__ float rs_sh;
-  const int tid = threadIdx.x;
+  __shared__ float red[GV_WARPS][R + 1];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float acc[R];
+#pragma unroll
+  for (int r = 0; r < R; ++r) acc[r] = 0.f;
   float ss = 0.f;
-  for (int c = tid; c < K; c += blockDim.x) { float v = xin[c]; xs[c] = v; ss = fmaf(v, v, ss); }
-  if (NORM) {
-    ss = warp_sum(ss);
-    if ((tid & 31) == 0) red[tid >> 5] = ss;
-    __syncthreads();
-    if (tid == 0) {
-      float v = 0.f;
-      for (int w = 0; w < 8; ++w) v += red[w];
-      rs_sh = 1.0f / sqrtf(v / (float)K + eps);
+  for (int c = (warp * 32 + lane) * V; c < K; c += GV_THREADS * V) {
+    float w[R][V];
+#pragma unroll
+    for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c, w[r]);      // R independent 16-byte loads in flight
+    float xv[V];
+#pragma unroll
+    for (int e = 0; e < V; e += 4) {
+      float4 t = __ldg(reinterpret_cast<const float4*>(x + c + e));
+      xv[e] = t.x; xv[e + 1] = t.y; xv[e + 2] = t.z; xv[e + 3] = t.w;
+    }
+#pragma unroll
+    for (int e = 0; e < V; ++e) {
+      ss = fmaf(xv[e], xv[e], ss);
+#pragma unroll
+      for (int r = 0; r < R; ++r) acc[r] = fmaf(xv[e], w[r][e], acc[r]);
     }
   }
-  __syncthreads();
-  const int row = blockIdx.x * 8 + (tid >> 5);
-  if (row >= rows) return;
-  const int lane = tid & 31;
-  const T* w = W + (size_t)row * K;
-  float a = 0.f;
-  for (int c = lane * V; c < K; c += 32 * V) {
-    float u[V];
-    ld16<T>(w + c, u);
 #pragma unroll
-    for (int e = 0; e < V; ++e) a = fmaf(xs[c + e], u[e], a);
-  }
-  a = warp_sum(a);
+  for (int r = 0; r < R; ++r) acc[r] = warp_sum(acc[r]);
+  ss = warp_sum(ss);
   if (lane == 0) {
-    if (NORM) a *= rs_sh;
-    if (RESID) out[row] = round_through<T>(out[row] + a);
-    else out[row] = a;
+#pragma unroll
+    for (int r = 0; r < R; ++r) red[warp][r] = acc[r];
+    red[warp][R] = ss;
+  }
+  __syncthreads();
+  if (threadIdx.x <= R) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < GV_WARPS; ++w) s += red[w][threadIdx.x];
+    if (threadIdx.x < R) dots_out[threadIdx.x] = s;
+    else *ss_out = s;
+  }
+  __syncthreads();
+}
+
+// out[j] = round(out[j] + x . W[j, :])   (O and down projections: residual update, Eq. 2 with all rows)
+template <typename T>
+__global__ void __launch_bounds__(GV_THREADS)
+gemv_resid_kernel(const T* __restrict__ W, int rows, int K, const float* __restrict__ x, float* __restrict__ out) {
+  __shared__ float dots[8];
+  __shared__ float ss;
+  const int r0 = blockIdx.x * 8;
+  const T* rowp[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) rowp[r] = W + (size_t)min(r0 + r, rows - 1) * K;
+  gemv_rows<T, 8>(rowp, K, x, dots, &ss);
+  if (threadIdx.x < 8 && r0 + threadIdx.x < rows) {
+    const int j = r0 + threadIdx.x;
+    out[j] = round_through<T>(out[j] + dots[threadIdx.x]);
   }
 }
 
-// RoPE on q and k of the new token, rounding through the storage type; append k, v, pos to the cache.
+// hm[j] = round(silu(rs * x . Wg[j, :]) * (rs * x . Wu[j, :])),  rs = 1 / sqrt(mean(x^2) + eps)   (Eq. 6)
 template <typename T>
-__global__ void dec_rope_store_kernel(float* __restrict__ q32, const float* __restrict__ k32,
-                                      const float* __restrict__ v32, int H, int Hkv, int d, int pos,
-                                      double theta, T* __restrict__ kc, T* __restrict__ vc,
-                                      int32_t* __restrict__ pc, int slot) {
-  int half = d >> 1;
-  int t = blockIdx.x * blockDim.x + threadIdx.x;
-  int nq = H * half, nk = Hkv * half;
-  if (t < nq + nk) {
-    bool isq = t < nq;
-    int u = isq ? t : t - nq;
-    int h = u / half, i = u - h * half;
-    double inv = exp2(-(double)(2 * i) / (double)d * log2(theta));
-    double s, c;
-    sincos((double)pos * inv, &s, &c);
-    float cf = (float)c, sf = (float)s;
-    const float* src = isq ? q32 : k32;
-    float a = src[h * d + i], b = src[h * d + i + half];
-    float r1 = a * cf - b * sf, r2 = b * cf + a * sf;
-    if (isq) {
+__global__ void __launch_bounds__(GV_THREADS)
+gemv_swiglu_kernel(const T* __restrict__ Wg, const T* __restrict__ Wu, int rows, int K, const float* __restrict__ x,
+                   float eps, float* __restrict__ hm) {
+  __shared__ float dots[16];
+  __shared__ float ss;
+  const int r0 = blockIdx.x * 8;
+  const T* rowp[16];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const size_t off = (size_t)min(r0 + r, rows - 1) * K;
+    rowp[r] = Wg + off;
+    rowp[8 + r] = Wu + off;
+  }
+  gemv_rows<T, 16>(rowp, K, x, dots, &ss);
+  if (threadIdx.x < 8 && r0 + threadIdx.x < rows) {
+    const float rs = 1.0f / sqrtf(ss / (float)K + eps);
+    const float g = dots[threadIdx.x] * rs, u = dots[8 + threadIdx.x] * rs;
+    hm[r0 + threadIdx.x] = round_through<T>(g / (1.0f + expf(-g)) * u);
+  }
+}
+
+// logits[j] = rs * x . W[j, :]   (first-token head)
+template <typename T>
+__global__ void __launch_bounds__(GV_THREADS)
+gemv_norm_kernel(const T* __restrict__ W, int rows, int K, const float* __restrict__ x, float eps,
+                 float* __restrict__ out) {
+  __shared__ float dots[8];
+  __shared__ float ss;
+  const int r0 = blockIdx.x * 8;
+  const T* rowp[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) rowp[r] = W + (size_t)min(r0 + r, rows - 1) * K;
+  gemv_rows<T, 8>(rowp, K, x, dots, &ss);
+  if (threadIdx.x < 8 && r0 + threadIdx.x < rows)
+    out[r0 + threadIdx.x] = dots[threadIdx.x] * (1.0f / sqrtf(ss / (float)K + eps));
+}
+
+// q, k, v projections of the new token with RMSNorm scale, rotary embedding (q, k) and the cache
+// append fused in.  Blocks [0, nq) serve q, [nq, nq + nk) k -- eight rows each: four rotary pairs
+// (i, i + d/2) of one head -- and the rest v, eight consecutive rows.
+template <typename T>
+__global__ void __launch_bounds__(GV_THREADS)
+dec_qkv_kernel(const T* __restrict__ wq, const T* __restrict__ wk, const T* __restrict__ wv, int H, int Hkv, int d,
+               int K, const float* __restrict__ x, float eps, int pos, double theta, float* __restrict__ q32,
+               T* __restrict__ kc, T* __restrict__ vc, int32_t* __restrict__ pc, int slot) {
+  __shared__ float dots[8];
+  __shared__ float ss;
+  const int half = d >> 1;
+  const int per_head = half / 4;                     // blocks per head for q and k
+  const int nq = H * per_head, nk = Hkv * per_head;
+  const int b = blockIdx.x;
+  const T* rowp[8];
+  int kind, h = 0, i0 = 0, v0 = 0;                   // kind 0 q, 1 k, 2 v
+  if (b < nq + nk) {
+    kind = b < nq ? 0 : 1;
+    const int bb = kind == 0 ? b : b - nq;
+    h = bb / per_head;
+    i0 = (bb - h * per_head) * 4;
+    const T* w = kind == 0 ? wq : wk;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      rowp[r] = w + (size_t)(h * d + i0 + r) * K;
+      rowp[4 + r] = w + (size_t)(h * d + half + i0 + r) * K;
+    }
+  } else {
+    kind = 2;
+    v0 = (b - nq - nk) * 8;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) rowp[r] = wv + (size_t)min(v0 + r, Hkv * d - 1) * K;
+  }
+  gemv_rows<T, 8>(rowp, K, x, dots, &ss);
+  const float rs = 1.0f / sqrtf(ss / (float)K + eps);
+  const int t = threadIdx.x;
+  if (kind == 2) {
+    if (t < 8 && v0 + t < Hkv * d) vc[(size_t)slot * Hkv * d + v0 + t] = from_f32<T>(dots[t] * rs);
+    return;
+  }
+  if (t < 4) {
+    const int i = i0 + t;
+    const double inv = exp2(-(double)(2 * i) / (double)d * log2(theta));
+    double sn, cs;
+    sincos((double)pos * inv, &sn, &cs);
+    const float cf = (float)cs, sf = (float)sn;
+    const float a = dots[t] * rs, bb2 = dots[4 + t] * rs;
+    const float r1 = a * cf - bb2 * sf, r2 = bb2 * cf + a * sf;
+    if (kind == 0) {
       q32[h * d + i] = round_through<T>(r1);
       q32[h * d + i + half] = round_through<T>(r2);
     } else {
@@ -112,62 +214,93 @@ __global__ void dec_rope_store_kernel(float* __restrict__ q32, const float* __re
       kc[((size_t)slot * Hkv + h) * d + i + half] = from_f32<T>(r2);
     }
   }
-  if (t < Hkv * d) vc[(size_t)slot * Hkv * d + t] = from_f32<T>(v32[t]);
-  if (t == 0) pc[slot] = pos;
+  if (b == 0 && t == 32) pc[slot] = pos;
 }
 
-// Split-KV attention of one query: block (h, s) handles keys [s*len/ns, (s+1)*len/ns).
-// part[(h*ns + s)] = (max, sum, o[d]); 4 warps, each strides over keys; lane owns d/32 dims.
-template <typename T, int DPL>
+// Split-KV attention of the new token.  Block (x, s): query heads [x * G, x * G + G) -- all of
+// them read KV head (x * G) / group -- over cached rows [s * len / ns, (s + 1) * len / ns).
+// A cached row is D * sizeof(T) bytes = LPK lanes x 16 bytes, so a warp takes 32 / LPK rows per
+// step and two steps are in flight.  part[(h * ns + s)] = (max, sum, o[D]) per query head.
+template <typename T, int D, int G>
 __global__ void __launch_bounds__(128)
-dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc, const T* __restrict__ vc,
-                        int len, int H, int Hkv, int nsplit, float* __restrict__ part) {
-  constexpr int d = DPL * 32;
-  __shared__ float sm_m[4], sm_l[4], sm_o[4][d];
-  const int h = blockIdx.x, s = blockIdx.y;
-  const int kvh = h / (H / Hkv);
+dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc, const T* __restrict__ vc, int len,
+                        int H, int Hkv, int nsplit, float* __restrict__ part) {
+  constexpr int V = DV<T>::N;              // elements per 16-byte chunk
+  constexpr int LPK = D / V;               // lanes per cached row
+  constexpr int KPW = 32 / LPK;            // rows per warp step
+  constexpr int NP = 4 * KPW;              // partial states per block
+  __shared__ float sm_m[NP][G], sm_l[NP][G];
+  __shared__ float sm_o[NP][G][D];
+  const int hb = blockIdx.x * G, s = blockIdx.y;
+  const int kvh = hb / (H / Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPK, li = lane % LPK;       // which row of the step, which chunk of the row
   const int j0 = (int)((long)len * s / nsplit), j1 = (int)((long)len * (s + 1) / nsplit);
-  const float scale = rsqrtf((float)d);
-  float qv[DPL];
+  const float scale = rsqrtf((float)D);
+  float q[G][V], o[G][V], m[G], l[G];
 #pragma unroll
-  for (int c = 0; c < DPL; ++c) qv[c] = q32[h * d + c * 32 + lane] * scale;
-  float m = -INFINITY, l = 0.f, o[DPL];
+  for (int g = 0; g < G; ++g) {
+    m[g] = -INFINITY; l[g] = 0.f;
 #pragma unroll
-  for (int c = 0; c < DPL; ++c) o[c] = 0.f;
-  for (int j = j0 + warp; j < j1; j += 4) {
-    const T* kr = kc + ((size_t)j * Hkv + kvh) * d;
-    const T* vr = vc + ((size_t)j * Hkv + kvh) * d;
-    float dot = 0.f;
-#pragma unroll
-    for (int c = 0; c < DPL; ++c) dot = fmaf(qv[c], to_f32(kr[c * 32 + lane]), dot);
-    dot = warp_sum(dot);
-    float mn = fmaxf(m, dot);
-    float corr = expf(m - mn), p = expf(dot - mn);
-    l = l * corr + p;
-#pragma unroll
-    for (int c = 0; c < DPL; ++c) o[c] = fmaf(p, to_f32(vr[c * 32 + lane]), o[c] * corr);
-    m = mn;
+    for (int e = 0; e < V; ++e) { q[g][e] = q32[(hb + g) * D + li * V + e] * scale; o[g][e] = 0.f; }
   }
-  if (lane == 0) { sm_m[warp] = m; sm_l[warp] = l; }
+  const size_t rstride = (size_t)Hkv * D;
+  const T* kbase = kc + (size_t)kvh * D + li * V;
+  const T* vbase = vc + (size_t)kvh * D + li * V;
+  constexpr int STEP = 4 * KPW;                      // rows per block step
+  // the trip count is the same for every lane of a warp (the shuffles below need all of them)
+  for (int jw = j0 + warp * KPW; jw < j1; jw += 2 * STEP) {
+    const int ja = jw + sub, jb = ja + STEP;
+    const bool hasa = ja < j1, hasb = jb < j1;
+    float ka[V], va[V], kb[V], vb[V];
+    ld16<T>(kbase + (size_t)(hasa ? ja : j0) * rstride, ka);
+    ld16<T>(vbase + (size_t)(hasa ? ja : j0) * rstride, va);
+    ld16<T>(kbase + (size_t)(hasb ? jb : j0) * rstride, kb);
+    ld16<T>(vbase + (size_t)(hasb ? jb : j0) * rstride, vb);
 #pragma unroll
-  for (int c = 0; c < DPL; ++c) sm_o[warp][c * 32 + lane] = o[c];
-  __syncthreads();
-  if (warp == 0) {
-    float M = fmaxf(fmaxf(sm_m[0], sm_m[1]), fmaxf(sm_m[2], sm_m[3]));
-    float L = 0.f, acc[DPL];
+    for (int g = 0; g < G; ++g) {
+      float da = 0.f, db = 0.f;
 #pragma unroll
-    for (int c = 0; c < DPL; ++c) acc[c] = 0.f;
-    for (int w = 0; w < 4; ++w) {
-      float f = sm_m[w] == -INFINITY ? 0.f : expf(sm_m[w] - M);
-      L += sm_l[w] * f;
+      for (int e = 0; e < V; ++e) { da = fmaf(q[g][e], ka[e], da); db = fmaf(q[g][e], kb[e], db); }
 #pragma unroll
-      for (int c = 0; c < DPL; ++c) acc[c] = fmaf(sm_o[w][c * 32 + lane], f, acc[c]);
+      for (int off = LPK / 2; off > 0; off >>= 1) {
+        da += __shfl_xor_sync(0xffffffffu, da, off);
+        db += __shfl_xor_sync(0xffffffffu, db, off);
+      }
+      if (hasa) {                                      // hasb implies hasa
+        if (!hasb) db = -INFINITY;
+        const float mn = fmaxf(m[g], fmaxf(da, db));
+        const float corr = expf(m[g] - mn), pa = expf(da - mn), pb = expf(db - mn);
+        l[g] = l[g] * corr + pa + pb;
+#pragma unroll
+        for (int e = 0; e < V; ++e) o[g][e] = fmaf(pa, va[e], fmaf(pb, vb[e], o[g][e] * corr));
+        m[g] = mn;
+      }
     }
-    float* p = part + ((size_t)h * nsplit + s) * (d + 2);
-    if (lane == 0) { p[0] = M; p[1] = L; }
+  }
+  const int pi = warp * KPW + sub;
 #pragma unroll
-    for (int c = 0; c < DPL; ++c) p[2 + c * 32 + lane] = acc[c];
+  for (int g = 0; g < G; ++g) {
+    if (li == 0) { sm_m[pi][g] = m[g]; sm_l[pi][g] = l[g]; }
+#pragma unroll
+    for (int e = 0; e < V; ++e) sm_o[pi][g][li * V + e] = o[g][e];
+  }
+  __syncthreads();
+  for (int t = threadIdx.x; t < G * D; t += 128) {
+    const int g = t / D, c = t - g * D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) M = fmaxf(M, sm_m[p][g]);
+    float L = 0.f, acc = 0.f;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+      const float f = sm_m[p][g] == -INFINITY ? 0.f : expf(sm_m[p][g] - M);
+      L += sm_l[p][g] * f;
+      acc = fmaf(sm_o[p][g][c], f, acc);
+    }
+    float* pp = part + ((size_t)(hb + g) * nsplit + s) * (D + 2);
+    if (c == 0) { pp[0] = M; pp[1] = L; }
+    pp[2 + c] = acc;
   }
 }
 
@@ -187,17 +320,29 @@ __global__ void dec_attn_combine_kernel(const float* __restrict__ part, int nspl
   att32[h * d + t] = round_through<T>(acc / L);
 }
 
-template <typename T>
-__global__ void dec_swiglu_kernel(const float* __restrict__ g, const float* __restrict__ u, int n,
-                                  float* __restrict__ out) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) {
-    float a = g[i];
-    out[i] = round_through<T>(a / (1.0f + expf(-a)) * u[i]);
-  }
-}
-
 constexpr int DEC_MAX_SPLIT = 64;
+#define TRY_DEC(...) do { spts_status s__ = (__VA_ARGS__); if (s__ != SPTS_OK) return s__; } while (0)
+
+template <typename T, int D>
+spts_status launch_attn_partial(spts_ctx* ctx, const float* q32, const spts_kv_layer* cache, int len, int nsplit,
+                                float* part) {
+  const auto& d = ctx->desc;
+  const int H = d.n_q_heads, Hkv = d.n_kv_heads, group = H / Hkv;
+  cudaStream_t st = ctx->stream;
+  const T* kc = (const T*)cache->k;
+  const T* vc = (const T*)cache->v;
+  // all query heads of a GQA group in one block when the group size is 2, 4 or 8; else one head per block
+  if (group % 8 == 0)
+    dec_attn_partial_kernel<T, D, 8><<<dim3(H / 8, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+  else if (group % 4 == 0)
+    dec_attn_partial_kernel<T, D, 4><<<dim3(H / 4, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+  else if (group % 2 == 0)
+    dec_attn_partial_kernel<T, D, 2><<<dim3(H / 2, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+  else
+    dec_attn_partial_kernel<T, D, 1><<<dim3(H, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
 
 template <typename T>
 spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_layer* cache, float* x32,
@@ -207,47 +352,30 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
   const int D = d.hidden, H = d.n_q_heads, Hkv = d.n_kv_heads, hd = d.head_dim, Dff = d.ffn_dim;
   float* base = (float*)ctx->ws.dec;
   float* q32 = base + D;                     // [H*hd]
-  float* k32 = q32 + H * hd;                 // [Hkv*hd]
-  float* v32 = k32 + Hkv * hd;               // [Hkv*hd]
-  float* att32 = v32 + Hkv * hd;             // [H*hd]
-  float* g32 = att32 + H * hd;               // [Dff]
-  float* u32 = g32 + Dff;                    // [Dff]
-  float* hm32 = u32 + Dff;                   // [Dff]
+  float* att32 = q32 + H * hd;               // [H*hd]
+  float* hm32 = att32 + H * hd;              // [Dff]
   float* part = hm32 + Dff;                  // [H, DEC_MAX_SPLIT, hd + 2]
   if (cache->len + 1 > cache->capacity) return SPTS_ERR_WORKSPACE;
-  const size_t smD = (size_t)D * 4;
-  gemv_kernel<T, true, false><<<ceil_div(H * hd, 8), 256, smD, st>>>((const T*)w->wq, H * hd, D, x32, d.rms_eps, q32);
-  SPTS_CUDA_OK(ctx);
-  gemv_kernel<T, true, false><<<ceil_div(Hkv * hd, 8), 256, smD, st>>>((const T*)w->wk, Hkv * hd, D, x32, d.rms_eps, k32);
-  SPTS_CUDA_OK(ctx);
-  gemv_kernel<T, true, false><<<ceil_div(Hkv * hd, 8), 256, smD, st>>>((const T*)w->wv, Hkv * hd, D, x32, d.rms_eps, v32);
-  SPTS_CUDA_OK(ctx);
   const int slot = cache->len;
-  int nthr = max(H * hd / 2 + Hkv * hd / 2, Hkv * hd);
-  dec_rope_store_kernel<T><<<ceil_div(nthr, 256), 256, 0, st>>>(q32, k32, v32, H, Hkv, hd, pos, (double)d.rope_theta,
-                                                              (T*)cache->k, (T*)cache->v, cache->pos, slot);
+  const int per_head = hd / 8;
+  const int qkv_blocks = (H + Hkv) * per_head + ceil_div(Hkv * hd, 8);
+  dec_qkv_kernel<T><<<qkv_blocks, GV_THREADS, 0, st>>>((const T*)w->wq, (const T*)w->wk, (const T*)w->wv, H, Hkv, hd, D,
+                                                        x32, d.rms_eps, pos, (double)d.rope_theta, q32, (T*)cache->k,
+                                                        (T*)cache->v, cache->pos, slot);
   SPTS_CUDA_OK(ctx);
   cache->len = slot + 1;
   const int len = cache->len;
-  int nsplit = min(DEC_MAX_SPLIT, max(1, len / 256));
-  dim3 grid(H, nsplit);
-  if (hd == 128) dec_attn_partial_kernel<T, 4><<<grid, 128, 0, st>>>(q32, (const T*)cache->k, (const T*)cache->v, len, H, Hkv, nsplit, part);
-  else dec_attn_partial_kernel<T, 2><<<grid, 128, 0, st>>>(q32, (const T*)cache->k, (const T*)cache->v, len, H, Hkv, nsplit, part);
-  SPTS_CUDA_OK(ctx);
+  const int nsplit = min(DEC_MAX_SPLIT, max(1, len / 128));
+  if (hd == 128) TRY_DEC(launch_attn_partial<T, 128>(ctx, q32, cache, len, nsplit, part));
+  else TRY_DEC(launch_attn_partial<T, 64>(ctx, q32, cache, len, nsplit, part));
   dec_attn_combine_kernel<T><<<H, hd, 0, st>>>(part, nsplit, hd, att32);
   SPTS_CUDA_OK(ctx);
-  gemv_kernel<T, false, true><<<ceil_div(D, 8), 256, (size_t)H * hd * 4, st>>>((const T*)w->wo, D, H * hd, att32, 0.f, x32);
+  gemv_resid_kernel<T><<<ceil_div(D, 8), GV_THREADS, 0, st>>>((const T*)w->wo, D, H * hd, att32, x32);
   SPTS_CUDA_OK(ctx);
-  gemv_kernel<T, true, false><<<ceil_div(Dff, 8), 256, smD, st>>>((const T*)w->w_gate, Dff, D, x32, d.rms_eps, g32);
+  gemv_swiglu_kernel<T><<<ceil_div(Dff, 8), GV_THREADS, 0, st>>>((const T*)w->w_gate, (const T*)w->w_up, Dff, D, x32,
+                                                                  d.rms_eps, hm32);
   SPTS_CUDA_OK(ctx);
-  gemv_kernel<T, true, false><<<ceil_div(Dff, 8), 256, smD, st>>>((const T*)w->w_up, Dff, D, x32, d.rms_eps, u32);
-  SPTS_CUDA_OK(ctx);
-  dec_swiglu_kernel<T><<<ceil_div(Dff, 256), 256, 0, st>>>(g32, u32, Dff, hm32);
-  SPTS_CUDA_OK(ctx);
-  if ((size_t)Dff * 4 > 48 * 1024) {
-    cudaFuncSetAttribute(gemv_kernel<T, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Dff * 4);
-  }
-  gemv_kernel<T, false, true><<<ceil_div(D, 8), 256, (size_t)Dff * 4, st>>>((const T*)w->w_down, D, Dff, hm32, 0.f, x32);
+  gemv_resid_kernel<T><<<ceil_div(D, 8), GV_THREADS, 0, st>>>((const T*)w->w_down, D, Dff, hm32, x32);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }
@@ -255,8 +383,8 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
 }  // namespace
 
 size_t decode_scratch_floats(const spts_model_desc& d) {
-  return (size_t)d.hidden + 2 * (size_t)d.n_q_heads * d.head_dim + 2 * (size_t)d.n_kv_heads * d.head_dim +
-         3 * (size_t)d.ffn_dim + (size_t)d.n_q_heads * DEC_MAX_SPLIT * (d.head_dim + 2) + 64;
+  return (size_t)d.hidden + 2 * (size_t)d.n_q_heads * d.head_dim + (size_t)d.ffn_dim +
+         (size_t)d.n_q_heads * DEC_MAX_SPLIT * (d.head_dim + 2) + 64;
 }
 
 spts_status launch_decode_load(spts_ctx* ctx, const void* x) {
@@ -281,6 +409,19 @@ spts_status launch_decode_layer(spts_ctx* ctx, const spts_layer_weights* w, spts
   float* x32 = (float*)ctx->ws.dec;
   if (ctx->desc.dtype == SPTS_BF16) return decode_layer_t<bf16>(ctx, w, cache, x32, pos);
   return decode_layer_t<float>(ctx, w, cache, x32, pos);
+}
+
+// logits = rstd(x) * lm_head x for one hidden row held in fp32 (x32) -- shared with the first-token head
+spts_status launch_head_logits(spts_ctx* ctx, const float* x32, const void* lm_head, float* logits) {
+  const auto& d = ctx->desc;
+  if (d.dtype == SPTS_BF16)
+    gemv_norm_kernel<bf16><<<ceil_div(d.vocab, 8), GV_THREADS, 0, ctx->stream>>>((const bf16*)lm_head, d.vocab, d.hidden,
+                                                                                 x32, d.rms_eps, logits);
+  else
+    gemv_norm_kernel<float><<<ceil_div(d.vocab, 8), GV_THREADS, 0, ctx->stream>>>((const float*)lm_head, d.vocab,
+                                                                                  d.hidden, x32, d.rms_eps, logits);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
 }
 
 }  // namespace spts

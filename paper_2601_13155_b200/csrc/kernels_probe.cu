@@ -169,41 +169,6 @@ __global__ void pad_proxy_kernel(const T* __restrict__ vg, const T* __restrict__
   out[total + t] = c < r ? zero : vu[row * r + (c - r)];
 }
 
-// logits[v] = rstd(x) * x . lm_head[v, :]; one warp per vocabulary row
-template <typename T>
-__global__ void head_logits_kernel(const T* __restrict__ x, const T* __restrict__ lm, int D, int V_,
-                                   float eps, float* __restrict__ logits) {
-  constexpr int V = Vec16<T>::N;
-  extern __shared__ float xs[];
-  __shared__ float red[32];
-  __shared__ float rs_sh;
-  int tid = threadIdx.x;
-  float ss = 0.f;
-  for (int c = tid; c < D; c += blockDim.x) { float v = to_f32(x[c]); xs[c] = v; ss = fmaf(v, v, ss); }
-  ss = warp_sum(ss);
-  if ((tid & 31) == 0) red[tid >> 5] = ss;
-  __syncthreads();
-  if (tid < 32) {
-    float v = tid < (blockDim.x >> 5) ? red[tid] : 0.f;
-    v = warp_sum(v);
-    if (tid == 0) rs_sh = 1.0f / sqrtf(v / (float)D + eps);
-  }
-  __syncthreads();
-  int row = blockIdx.x * (blockDim.x >> 5) + (tid >> 5);
-  if (row >= V_) return;
-  int lane = tid & 31;
-  const T* w = lm + (size_t)row * D;
-  float a = 0.f;
-  for (int c = lane * V; c < D; c += 32 * V) {
-    float u[V];
-    load16<T>(w + c, u);
-#pragma unroll
-    for (int e = 0; e < V; ++e) a = fmaf(xs[c + e], u[e], a);
-  }
-  a = warp_sum(a);
-  if (lane == 0) logits[row] = a * rs_sh;
-}
-
 // argmax with the lowest index on ties (single block)
 __global__ void __launch_bounds__(1024)
 argmax_kernel(const float* __restrict__ logits, int n, int32_t* __restrict__ out) {
@@ -315,18 +280,14 @@ spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void
 
 spts_status launch_head(spts_ctx* ctx, const void* x_row, const void* lm_head, float* logits,
                         int32_t* token_out) {
-  const auto& d = ctx->desc;
-  const int wpb = 8;
-  size_t sm = (size_t)d.hidden * sizeof(float);
-  if (d.dtype == SPTS_BF16)
-    head_logits_kernel<bf16><<<ceil_div(d.vocab, wpb), wpb * 32, sm, ctx->stream>>>(
-        (const bf16*)x_row, (const bf16*)lm_head, d.hidden, d.vocab, d.rms_eps, logits);
-  else
-    head_logits_kernel<float><<<ceil_div(d.vocab, wpb), wpb * 32, sm, ctx->stream>>>(
-        (const float*)x_row, (const float*)lm_head, d.hidden, d.vocab, d.rms_eps, logits);
-  SPTS_CUDA_OK(ctx);
+  // the row is widened into the fp32 vector scratch that the decode kernels use, then the same
+  // weight-streaming matrix-vector kernel computes rstd(x) * lm_head x
+  spts_status s = launch_decode_load(ctx, x_row);
+  if (s != SPTS_OK) return s;
+  s = launch_head_logits(ctx, (const float*)ctx->ws.dec, lm_head, logits);
+  if (s != SPTS_OK) return s;
   if (token_out != nullptr) {
-    argmax_kernel<<<1, 1024, 0, ctx->stream>>>(logits, d.vocab, token_out);
+    argmax_kernel<<<1, 1024, 0, ctx->stream>>>(logits, ctx->desc.vocab, token_out);
     SPTS_CUDA_OK(ctx);
   }
   return SPTS_OK;

@@ -149,6 +149,7 @@ spts_status launch_decode_load(spts_ctx* ctx, const void* x);     // x [D] -> fp
 spts_status launch_decode_store(spts_ctx* ctx, void* x);          // fp32 residual scratch -> x [D]
 spts_status launch_decode_layer(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_layer* cache,
                                 int32_t pos);
+spts_status launch_head_logits(spts_ctx* ctx, const float* x32, const void* lm_head, float* logits);
 
 // ---- kernels_tc_gemm.cu / kernels_tc_attn.cu : tcgen05 path (bf16)
 enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4 };
