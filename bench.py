@@ -38,7 +38,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="spts", choices=["spts", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5", "paper"])
     ap.add_argument("--no-128k", action="store_true", help="skip the 131072-token measurement added to the cfg3 line")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
@@ -129,7 +129,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2601_13155_b200 import synth
-    w = synth.workload("cfg3" if args.workload == "cfg5" else args.workload)
+    w = synth.workload("cfg3" if args.workload in ("cfg5", "paper") else args.workload)
     vals = []
     for i in range(args.warmup + args.steps):
         tps, cores, desc, dt = oracle_sample(w)
@@ -175,6 +175,8 @@ def main():
 
     if args.workload == "cfg5":
         line = generation_line(args, rep, dev)
+    elif args.workload == "paper":
+        line = paper_protocol_line(args, rep, dev)
     else:
         line = prefill_line(args, rep, dev, args.workload, args.steps, max(args.warmup, 3), 2, True)
         if args.workload == "cfg3" and not args.no_128k and not args.layers:
@@ -293,6 +295,83 @@ def generation_line(args, rep, dev):
                              "traffic": None, "kernel": "decode step (all layers, dense arm)", "launches": dk["calls"],
                              "ms_per_launch": dk["ms"] / dk["calls"],
                              "peak_source": "measured (copy)" if peaks else "fallback"},
+                "gpu_launches": int(lib.launch_count())}
+    lib.close()
+    return line
+
+
+def paper_protocol_line(args, rep, dev):
+    """The paper's efficiency protocol on this code: LLaMA schedule of Section 4.1 (dense layers 0-9, stage ends after
+    13 / 18 / 23 / 28, budgets 9 / 7 / 4 / 2 Ki), prompt lengths 8K-32K, TTFT of dense, PAP only, PAP + LTP and full SPTS
+    (the rows of its component ablation, Table 2).  value = prompt tokens / s of full SPTS at 32K."""
+    import torch
+    from paper_2601_13155_b200 import binding, schedule, synth
+    rank, world = rep.rank, rep.world
+    w = synth.workload("cfg3")
+    shape = w.shape
+    L, Nmax = shape.n_layers, w.n_tokens
+    layers = []
+    for l in range(L):
+        t = synth.device_layer_weights(shape, w.seed, l, dev)
+        lw = binding.LayerWeights.__new__(binding.LayerWeights)
+        lw.t = t
+        lw.c = binding.LayerWeightsC(**{n: t[n].data_ptr() for n in binding.WEIGHT_NAMES})
+        layers.append(lw)
+    hw = synth.device_head_weights(shape, w.seed, dev)
+    model = binding.Model(layers, hw["lm_head"], hw["embed"])
+    X0, _ = synth.device_hidden_states(w, dev)
+    lib = binding.Spts(shape, max_seq=Nmax, device=dev)
+    cache = binding.KvCache(shape, L, Nmax, dev)
+    X, Xa = torch.empty_like(X0), torch.empty_like(X0)
+    ar = torch.arange(Nmax, dtype=torch.int32, device=dev)
+    pos, orig, pa, oa = ar.clone(), ar.clone(), ar.clone(), ar.clone()
+    tok = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def ttft(plan, n, steps):
+        def one():
+            X[:n].copy_(X0[:n])
+            pos[:n].copy_(ar[:n])
+            orig[:n].copy_(ar[:n])
+            lib.prefill(model, plan, X, pos, orig, Xa, pa, oa, cache, token_out=tok, n_tokens=n)
+        one()
+        rep.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            one()
+        e1.record()
+        rep.barrier()
+        return rep.max_over_ranks(e0.elapsed_time(e1)) / steps
+
+    table = {}
+    for n in (8192, 16384, 24576, 32768):
+        plans = {"dense": [(n, n, 0)] * L,
+                 "pap": schedule.paper_llama_plan(n, ltp=False, msdp=False),
+                 "pap_ltp": schedule.paper_llama_plan(n, msdp=False),
+                 "spts": schedule.paper_llama_plan(n)}
+        ms = {k: ttft(p, n, max(1, args.steps)) for k, p in plans.items()}
+        kv = schedule.kv_token_layers(plans["spts"])
+        table[str(n)] = {"ttft_ms": ms, "speedup_vs_dense": {k: ms["dense"] / v for k, v in ms.items() if k != "dense"},
+                         "kv_saving_pct": 100.0 * (1 - kv / (L * n))}
+    if lib.device_status() != 0:
+        raise RuntimeError("device status")
+    line = None
+    if rank == 0:
+        full = table["32768"]
+        line = {"metric": "prefill_tokens_per_s", "value": 32768 * world / (full["ttft_ms"]["spts"] * 1e-3), "unit": "tokens/s",
+                "n_gpus": world, "steps": max(1, args.steps), "warmup": 1, "ms_per_step": full["ttft_ms"]["spts"],
+                "ttft_ms": full["ttft_ms"]["spts"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": "paper protocol: 32-layer LLaMA-3.1-8B shape, the paper's LLaMA schedule (skip from layer "
+                                       "10, stage ends 13/18/23/28, budgets 9/7/4/2 Ki, prune to budget - 1 Ki), prompts 8K-32K",
+                           "global_batch": world, "seq_len": 32768, "parallelism": f"replicas x{world}",
+                           "l2": "inputs larger than L2 (14 GB of weights streamed per step)"},
+                "lengths": table,
+                "paper_context": {"ttft_speedup_a800": {"pap": [1.08, 1.24, 1.35, 1.44], "pap_ltp": [1.26, 1.70, 1.98, 2.15],
+                                                         "spts": [1.35, 1.91, 2.26, 2.46]},
+                                  "kv_saving_pct": [29.7, 48.4, 55.2, 58.6],
+                                  "note": "Table 2 / Table 3 of the paper: one A800 80 GB, trained LLaMA-3.1-8B-Instruct, LongBench "
+                                          "prompts, HF Transformers + FlashAttention-2; context only"},
                 "gpu_launches": int(lib.launch_count())}
     lib.close()
     return line

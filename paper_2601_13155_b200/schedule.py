@@ -44,3 +44,35 @@ def workload_plan(w, keep_attn=None, keep_ffn=None, dense: bool = False):
 
 def cache_capacities(plan, extra: int = 0):
     return [p[0] + extra for p in plan]
+
+
+def paper_llama_plan(n_prompt: int, n_layers: int = 32, ltp: bool = True, msdp: bool = True):
+    """The paper's LLaMA-3.1-8B setting (Section 4.1): layers 0-9 dense, skipping from layer 10, stage ends after
+    layers 13 / 18 / 23 / 28 with active budgets of 9 / 7 / 4 / 2 Ki tokens, each stage end pruning the candidates
+    to its budget minus 1 Ki; the layers after the last boundary keep the last budget (0-indexed layers; the
+    reading that reproduces the KV-cache sizes of Table 3).
+    ltp=False leaves the FFN dense (the "PAP only" row of the paper's component ablation, Table 2);
+    msdp=False keeps every token a candidate in every layer (budgets unchanged, no pruning)."""
+    ki = 1024
+    budgets = (9 * ki, 7 * ki, 4 * ki, 2 * ki)
+    ends = (13, 18, 23, 28)
+    cur = n_prompt
+    out = []
+    for l in range(n_layers):
+        if l < 10:
+            out.append((cur, cur, 0))
+            continue
+        s = next((i for i, e in enumerate(ends) if l <= e), len(ends) - 1)
+        m = min(cur, budgets[s])
+        nxt = 0
+        if msdp and l in ends:
+            nxt = min(cur, budgets[ends.index(l)] - ki)
+        out.append((m, m if ltp else cur, nxt if nxt < cur else 0))
+        if nxt and nxt < cur:
+            cur = nxt
+    return out
+
+
+def kv_token_layers(plan) -> int:
+    """Cached (token, layer) pairs after prefill: every layer caches its m_attn active rows."""
+    return sum(p[0] for p in plan)

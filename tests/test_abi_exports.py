@@ -69,3 +69,28 @@ def test_product_schedule_matches_budget_rule():
     op = O.msdp_schedule(32, w.n_tokens, w.stage_first_layer, w.stage_tokens,
                          math.ceil(w.keep_attn * w.n_tokens), math.ceil(w.keep_ffn * w.n_tokens))
     assert [(p["m_attn"], p["m_ffn"], p["prune_to"] or 0) for p in op] == plan
+
+
+def test_paper_llama_plan_matches_oracle_and_table3():
+    """The product's statement of the paper's LLaMA schedule agrees with the oracle's independent one and
+    reproduces the KV-cache sizes the paper prints (Table 3: 2.81 / 4.13 / 5.38 / 6.63 with PAP against
+    4 / 8 / 12 / 16 without, i.e. savings of 29.7 / 48.4 / 55.2 / 58.6 %)."""
+    from paper_2601_13155_b200 import schedule
+    from oracle import spts_oracle as O
+    printed = {8192: (2.81, 29.7), 16384: (4.13, 48.4), 24576: (5.38, 55.2), 32768: (6.63, 58.6)}
+    for n, (size, saving) in printed.items():
+        plan = schedule.paper_llama_plan(n)
+        cur, want = n, []
+        for q in O.paper_llama_schedule(n):
+            pr = q["prune_to"] if q["prune_to"] is not None and q["prune_to"] < cur else 0
+            want.append((q["m_attn"], q["m_ffn"], pr))
+            cur = pr or cur
+        assert plan == want
+        kv = schedule.kv_token_layers(plan)
+        assert f"{kv / 1024 / 64 + 1e-9:.2f}" == f"{size:.2f}"
+        assert abs(100 * (1 - kv / (32 * n)) - saving) < 0.06
+    # ablation switches: FFN dense without LTP; no pruning without MSDP
+    p = schedule.paper_llama_plan(32768, ltp=False)
+    assert p[20] == (4096, 6144, 0)                                  # 6144 candidates left after two prunes
+    p = schedule.paper_llama_plan(32768, msdp=False)
+    assert all(c == 0 for _, _, c in p) and p[31] == (2048, 2048, 0) and p[12] == (9216, 9216, 0)
