@@ -30,7 +30,7 @@ constexpr int BM = 128;
 constexpr int BK = 64;                        // 64 bf16 = one 128-byte swizzle row
 constexpr int A_STAGE_BYTES = BM * BK * 2;    // 16 KiB
 constexpr int GEMM_THREADS = 192;
-constexpr int GROUP_M = 8;
+constexpr double RASTER_L2_BYTES = 48e6;       // how much of the grouped operand is allowed to sit in L2
 
 template <int BN> struct Cfg {
   static constexpr int B_STAGE_BYTES = BN * BK * 2;
@@ -52,15 +52,24 @@ struct TcParams {
   float* csq; int csq_parts;
   int* status;
   int num_m, num_n;
+  int raster_group;             // tiles of the grouped dimension whose operand stays in L2 (8 or 16)
+  int raster_n;                 // 0: groups of row tiles sweep all column tiles; 1: groups of column tiles sweep all rows
 };
 
-__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int& mb, int& nb) {
-  const int per_group = GROUP_M * num_n;
+// Tile order.  The CTAs in flight at one time work on `group` tiles of one dimension times as many
+// tiles of the other as fit, so the grouped operand stays in L2 while the other streams past it; which
+// dimension is grouped is chosen by the launcher from the two operands' sizes.
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int raster_n, int group, int& mb, int& nb) {
+  const int na = raster_n ? num_n : num_m;      // grouped dimension
+  const int nbo = raster_n ? num_m : num_n;     // swept dimension
+  const int per_group = group * nbo;
   const int g = t / per_group;
   const int rem = t - g * per_group;
-  const int gm = min(GROUP_M, num_m - g * GROUP_M);
-  mb = g * GROUP_M + rem % gm;
-  nb = rem / gm;
+  const int gs = min(group, na - g * group);
+  const int a = g * group + rem % gs;
+  const int b = rem / gs;
+  mb = raster_n ? b : a;
+  nb = raster_n ? a : b;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -154,7 +163,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         int mb, nb;
-        tile_coords(t, p.num_m, p.num_n, mb, nb);
+        tile_coords(t, p.num_m, p.num_n, p.raster_n, p.raster_group, mb, nb);
         const int m0 = mb * BM, n0 = nb * NT;
         for (int kb = 0; kb < kblocks; ++kb) {
           ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1, abort_flag, t0);
@@ -181,7 +190,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
       int mb, nb;
-      tile_coords(t, p.num_m, p.num_n, mb, nb);
+      tile_coords(t, p.num_m, p.num_n, p.raster_n, p.raster_group, mb, nb);
       const int m0 = mb * BM;
       const bf16* rowp[8];
       uint32_t soff[8];
@@ -260,7 +269,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
       int mb, nb;
-      tile_coords(t, p.num_m, p.num_n, mb, nb);
+      tile_coords(t, p.num_m, p.num_n, p.raster_n, p.raster_group, mb, nb);
       const int grow = mb * BM + row_in_tile;
       const int n0 = nb * NT;
       const bool row_ok = grow < p.M;
@@ -453,7 +462,21 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
   p.num_m = ceil_div(a.M, BM);
   p.num_n = ceil_div(a.Nout, NT);
-  if (EPI == TC_SUMSQ && p.num_n > a.csq_parts) return SPTS_ERR_WORKSPACE;
+  {
+    // DRAM traffic of the candidate tile orders: the grouped operand is read once per group (it must fit in
+    // L2 beside the streams), the other operand once per pass over the groups
+    const double a_bytes = 2.0 * a.M * a.K, w_bytes = 2.0 * a.Nout * a.K * (EPI == TC_SWIGLU ? 2.0 : 1.0);
+    double best = -1.0;
+    for (int rn = 0; rn < 2; ++rn) {
+      for (int grp = 8; grp <= 16; grp += 8) {
+        const int tiles = rn ? p.num_n : p.num_m;
+        const double band = (rn ? w_bytes / p.num_n : a_bytes / p.num_m) * grp;
+        if (grp > 8 && band > RASTER_L2_BYTES) continue;
+        const double cost = (double)ceil_div(tiles, grp) * (rn ? a_bytes : w_bytes) + (rn ? w_bytes : a_bytes);
+        if (best < 0.0 || cost < best) { best = cost; p.raster_n = rn; p.raster_group = grp; }
+      }
+    }
+  }
   CUtensorMap tmA, tmB, tmB2;
   if (!make_map(ctx, &tmA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, (uint64_t)a.lda, (uint32_t)BM)) return SPTS_ERR_CUDA;
   if (!make_map(ctx, &tmB, a.W, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
