@@ -620,7 +620,7 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
   if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)m, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
   AttnParams p;
   p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.O = O; p.status = ctx->ws.status;
-  if ((d.n_q_heads / d.n_kv_heads) % 2 == 0) {
+  if ((d.n_q_heads / d.n_kv_heads) % 2 == 0 && !ctx->attn_one_tile) {
     dim3 grid(d.n_q_heads / 2, ceil_div(m, TILE));
     tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
   } else {

@@ -248,6 +248,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->launches = 0;
   ctx->sm_count = prop.multiProcessorCount;
   ctx->encode_tiled = nullptr;
+  ctx->attn_one_tile = false;
   ctx->prof = new (std::nothrow) Profiler;
   carve(*desc, max_seq, workspace, &ctx->ws);
   ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
@@ -306,6 +307,10 @@ spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
     if (ctx->desc.dtype == SPTS_FP32 || !tc_shape_ok(ctx->desc)) return value ? SPTS_OK : SPTS_ERR_UNSUPPORTED;
     if (!value && ctx->encode_tiled == nullptr) TRY(tc_init(ctx));
     ctx->reference_kernels = value != 0;
+    return SPTS_OK;
+  }
+  if (option == SPTS_ATTENTION_ONE_TILE) {
+    ctx->attn_one_tile = value != 0;
     return SPTS_OK;
   }
   return SPTS_ERR_INVALID_ARG;

@@ -85,6 +85,7 @@ struct spts_ctx {
   cudaStream_t stream;
   spts::Workspace ws;
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
+  bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
   int64_t launches;
   int sm_count;
   void* encode_tiled;       // cuTensorMapEncodeTiled entry point (tensor-core mode)

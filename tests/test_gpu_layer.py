@@ -182,3 +182,35 @@ def test_prefill_and_decode_match_oracle(dtype, ref):
         assert int(tok.item()) == int(np.argmax(host(lgd)))
     assert lib.device_status() == 0
     lib.close()
+
+
+def test_attention_kernels_agree_under_large_score_jumps():
+    """The two tensor-core attention kernels (two heads per CTA with P in tensor memory; one tile per CTA with P
+    through shared memory) keep their running maximum lazily: O is rescaled only when the maximum grows by more
+    than 2^8.  Here W_q and W_k are scaled so that logits spread over ~45 octaves, which makes rows jump by tens
+    of octaves between key blocks, and the two kernels must agree on identical Q^, K^, V^.  (At this scale the
+    bf16 rounding of Q^ and K^ alone moves probabilities by tens of percent, so the oracle is not the yardstick
+    for this case; the oracle comparisons above cover the ordinary range.)"""
+    from paper_2601_13155_b200 import binding
+    shape = SMALL_BF16
+    N = 1024 + 77
+    W = synth.layer_weights(shape, 31, 0, std=0.05)
+    W["wq"] = synth.quantize(W["wq"] * 5.0, "bf16")
+    W["wk"] = synth.quantize(W["wk"] * 5.0, "bf16")
+    W["w_down"] = np.zeros_like(W["w_down"])          # expose the attention block alone
+    X, _ = synth.hidden_states(shape, N, 31, heavy=16)
+    Wd = binding.LayerWeights(W, "bf16")
+    pos = i32(np.arange(N))
+    outs = []
+    for one_tile in (False, True):
+        lib = _mk(shape, 2048, False)
+        lib.set_attention_one_tile(one_tile)
+        Xd = up(X, "bf16")
+        lib.layer_prefill_skip(Wd, Xd, pos, N, N, binding.KvCache(shape, 1, N))
+        assert lib.device_status() == 0
+        outs.append(host(Xd))
+        lib.close()
+    assert np.isfinite(outs[0]).all()
+    delta = outs[0] - host(up(X, "bf16"))
+    assert np.abs(delta).max() > 0.1                    # the attention block did something
+    check_output(outs[0], outs[1], "bf16")              # same rule as against the oracle
