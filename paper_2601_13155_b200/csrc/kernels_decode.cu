@@ -304,23 +304,54 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
   }
 }
 
+constexpr int DEC_MAX_SPLIT = 64;
+
+// Combines the slices of one query head: thread s < nsplit first takes slice s's (max, sum) so that the global
+// maximum and the weights exp(max_s - M) come from one parallel step; then thread t sums dimension t over the
+// slices with the loads of eight slices in flight.  blockDim = d >= nsplit.
 template <typename T>
-__global__ void dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d,
-                                        float* __restrict__ att32) {
-  const int h = blockIdx.x, t = threadIdx.x;   // blockDim = d
-  float M = -INFINITY;
-  for (int s = 0; s < nsplit; ++s) M = fmaxf(M, part[((size_t)h * nsplit + s) * (d + 2)]);
-  float L = 0.f, acc = 0.f;
-  for (int s = 0; s < nsplit; ++s) {
-    const float* p = part + ((size_t)h * nsplit + s) * (d + 2);
-    float f = p[0] == -INFINITY ? 0.f : expf(p[0] - M);
-    L += p[1] * f;
-    acc = fmaf(p[2 + t], f, acc);
+__global__ void __launch_bounds__(128)
+dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float* __restrict__ att32) {
+  __shared__ float f[DEC_MAX_SPLIT];
+  __shared__ float red[4];
+  __shared__ float Msh, Lsh;
+  const int h = blockIdx.x, t = threadIdx.x, nw = blockDim.x >> 5;
+  const float* ph = part + (size_t)h * nsplit * (d + 2);
+  const float m = t < nsplit ? ph[(size_t)t * (d + 2)] : -INFINITY;
+  float v = warp_max(m);
+  if ((t & 31) == 0) red[t >> 5] = v;
+  __syncthreads();
+  if (t == 0) {
+    float M = red[0];
+    for (int w = 1; w < nw; ++w) M = fmaxf(M, red[w]);
+    Msh = M;
   }
-  att32[h * d + t] = round_through<T>(acc / L);
+  __syncthreads();
+  const float fs = m == -INFINITY ? 0.f : expf(m - Msh);
+  if (t < nsplit) f[t] = fs;
+  v = warp_sum(t < nsplit ? ph[(size_t)t * (d + 2) + 1] * fs : 0.f);
+  __syncthreads();                       // red[] has been read by thread 0
+  if ((t & 31) == 0) red[t >> 5] = v;
+  __syncthreads();
+  if (t == 0) {
+    float L = 0.f;
+    for (int w = 0; w < nw; ++w) L += red[w];
+    Lsh = L;
+  }
+  __syncthreads();
+  float acc = 0.f;
+  int s0 = 0;
+  for (; s0 + 8 <= nsplit; s0 += 8) {
+    float x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = ph[(size_t)(s0 + u) * (d + 2) + 2 + t];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc = fmaf(x[u], f[s0 + u], acc);
+  }
+  for (; s0 < nsplit; ++s0) acc = fmaf(ph[(size_t)s0 * (d + 2) + 2 + t], f[s0], acc);
+  att32[h * d + t] = round_through<T>(acc / Lsh);
 }
 
-constexpr int DEC_MAX_SPLIT = 64;
 #define TRY_DEC(...) do { spts_status s__ = (__VA_ARGS__); if (s__ != SPTS_OK) return s__; } while (0)
 
 template <typename T, int D>

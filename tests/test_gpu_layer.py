@@ -214,3 +214,20 @@ def test_attention_kernels_agree_under_large_score_jumps():
     delta = outs[0] - host(up(X, "bf16"))
     assert np.abs(delta).max() > 0.1                    # the attention block did something
     check_output(outs[0], outs[1], "bf16")              # same rule as against the oracle
+
+
+@pytest.mark.parametrize("N,ma,mf", [(1, 1, 1), (2, 1, 2), (3, 2, 1), (17, 5, 17), (129, 128, 1), (257, 129, 130)])
+@pytest.mark.parametrize("ref", [True, False])
+def test_tiny_and_ragged_sequences(N, ma, mf, ref):
+    """Degenerate sizes on the bf16 kernels (tensor-core and plain): a single token, budgets of one row, sizes one
+    past a tile edge.  Same block-wise comparison with the oracle as the larger cases."""
+    from paper_2601_13155_b200 import binding
+    shape = SMALL_BF16
+    lib = _mk(shape, 512, ref)
+    W, X, Wd = _layer_case(shape, N, 77 + N, min(N, 3))
+    Wmid = binding.LayerWeights(zero_down(W), shape.dtype)
+    pos = (np.arange(N) * 3 + 1).astype(np.int32)
+    Xd = up(X, shape.dtype)
+    cache = binding.KvCache(shape, 1, N)
+    check_layer_blocks(lib, shape, W, Wd, Wmid, Xd, i32(pos), ma, mf, cache)
+    lib.close()
