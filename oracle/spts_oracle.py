@@ -370,6 +370,59 @@ def proxy_macs_per_projection(D, d_low, r):
 
 
 # ----------------------------------------------------------------------------
+# offline construction of the low-rank proxy FFN (Section 3.3: saliency, channel
+# importance, channel selection, rank-r factorisation)
+# ----------------------------------------------------------------------------
+def proxy_saliency(Xc, W, shape):
+    """z(x) = |silu(x W_gate) * (x W_up)| for every calibration token (rows of Xc are the hidden
+    states preceding the FFN block; they are normalised like the FFN's input).  [n_cal, Dff]."""
+    B = rmsnorm(np.asarray(Xc, F64), np.ones(Xc.shape[1]), shape.rms_eps)
+    return np.abs(silu(B @ np.asarray(W["w_gate"], F64).T) * (B @ np.asarray(W["w_up"], F64).T))
+
+
+def proxy_channel_importance(z, rho):
+    """I_j = mean of the top rho-fraction of channel j's saliency values over the calibration set;
+    the count is max(1, floor(rho * |G|))."""
+    n = z.shape[0]
+    k = max(1, int(math.floor(rho * n)))
+    top = -np.sort(-np.asarray(z, F64), axis=0)[:k]
+    return top.mean(axis=0)
+
+
+def proxy_select_channels(importance, d_low):
+    """C = TopK(I, D_low), ascending channel indices, ties to the lower index."""
+    return topk_select(importance, d_low, force_last=False)
+
+
+def proxy_factor(Wp, r):
+    """Rank-r factorisation W' ~ U V of a [D, D_low] matrix by truncated SVD: U [D, r] has orthonormal
+    columns, V = diag(sigma_r) V_r^T [r, D_low].  Returns (U, V, all singular values)."""
+    Uf, sg, Vt = np.linalg.svd(np.asarray(Wp, F64), full_matrices=False)
+    return Uf[:, :r], sg[:r, None] * Vt[:r], sg
+
+
+def proxy_build(Xc, W, shape, rho=0.2, channels=None):
+    """The whole construction for one layer.  Returns the importance vector, the selected channels and the six
+    factors in the library's storage layout: ug/uu [r, D] = U^T, vg/vu [D_low, r] = V^T, vd [r, D_low] = V_down,
+    ud [D, r] = U_down, plus the singular values of the three reduced matrices."""
+    z = proxy_saliency(Xc, W, shape)
+    imp = proxy_channel_importance(z, rho)
+    C = proxy_select_channels(imp, shape.ltp_dlow) if channels is None else np.asarray(channels)
+    r = shape.ltp_rank
+    out = {"importance": imp, "channels": C, "sigma": {}}
+    # the paper writes the projections as [D, Dff] matrices; w_gate / w_up are stored [Dff, D], w_down [D, Dff]
+    for name, Wp in (("g", np.asarray(W["w_gate"], F64)[C].T), ("u", np.asarray(W["w_up"], F64)[C].T),
+                     ("d", np.asarray(W["w_down"], F64)[:, C])):
+        U, V, sg = proxy_factor(Wp, r)
+        out["sigma"][name] = sg
+        if name == "d":
+            out["vd"], out["ud"] = V, U
+        else:
+            out["u" + name], out["v" + name] = U.T, V.T
+    return out
+
+
+# ----------------------------------------------------------------------------
 # whole prefill (Algorithm 1) and decode
 # ----------------------------------------------------------------------------
 def model_prefill(X, layers, shape, plan, mode="exact", force_last=True):

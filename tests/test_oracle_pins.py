@@ -455,3 +455,64 @@ def test_bf16_mode_rounds_only_at_storage_points():
     rel = np.abs(r["X"] - e["X"]).max() / np.sqrt(np.mean(e["X"] ** 2))
     assert 0 < rel < 0.1
     assert np.array_equal(r["S_mha"], e["S_mha"])     # PAP scores come from unrounded K
+
+
+# ------------------------------------------------------------------ proxy construction (Section 3.3)
+def test_channel_importance_bruteforce_and_limits():
+    rng = np.random.default_rng(40)
+    z = rng.random((37, 11))
+    for rho in (0.05, 0.2, 0.5, 1.0):
+        k = max(1, int(rho * 37))
+        want = [np.mean(sorted(z[:, j], reverse=True)[:k]) for j in range(11)]
+        assert np.allclose(O.proxy_channel_importance(z, rho), want, rtol=1e-14)
+    assert np.allclose(O.proxy_channel_importance(z, 1.0), z.mean(axis=0))          # all samples: the plain mean
+    assert np.allclose(O.proxy_channel_importance(z, 1e-9), z.max(axis=0))          # at least one sample: the max
+    imp = np.array([0.5, 2.0, 2.0, 0.1, 3.0])
+    assert O.proxy_select_channels(imp, 3).tolist() == [1, 2, 4]
+    assert O.proxy_select_channels(imp, 2).tolist() == [1, 4]                        # tie: lower index
+
+
+def test_saliency_is_the_ffn_intermediate_magnitude():
+    W = _layer()
+    X = _x(9)
+    z = O.proxy_saliency(X, W, SH)
+    B = torch.nn.functional.rms_norm(torch.from_numpy(X), (SH.hidden,), None, SH.rms_eps)
+    g = torch.nn.functional.silu(B @ torch.from_numpy(W["w_gate"].astype(np.float64)).T)
+    u = B @ torch.from_numpy(W["w_up"].astype(np.float64)).T
+    assert np.allclose(z, (g * u).abs().numpy(), rtol=1e-12, atol=1e-15)
+
+
+def test_rank_r_factor_obeys_eckart_young():
+    rng = np.random.default_rng(41)
+    Wp = rng.standard_normal((40, 24))
+    for r in (1, 5, 24):
+        U, V, sg = O.proxy_factor(Wp, r)
+        assert U.shape == (40, r) and V.shape == (r, 24)
+        assert np.allclose(U.T @ U, np.eye(r), atol=1e-12)                            # orthonormal columns
+        err = np.linalg.norm(Wp - U @ V) ** 2
+        assert np.isclose(err, np.sum(sg[r:] ** 2), rtol=1e-10, atol=1e-18)          # optimal rank-r error
+    lowrank = rng.standard_normal((40, 3)) @ rng.standard_normal((3, 24))
+    U, V, _ = O.proxy_factor(lowrank, 3)
+    assert np.allclose(U @ V, lowrank, atol=1e-12)                                     # r = rank: exact
+
+
+def test_proxy_build_layout_and_full_rank_limit():
+    W = _layer()
+    Xc = _x(50, seed=12)
+    full = replace(SH, ltp_dlow=SH.ffn_dim, ltp_rank=min(SH.hidden, SH.ffn_dim))
+    P = O.proxy_build(Xc, W, full, rho=0.2)
+    assert P["channels"].tolist() == list(range(SH.ffn_dim))
+    Wp = {**{k: np.asarray(v, np.float64) for k, v in W.items()}, **{k: P[k] for k in ("ug", "vg", "uu", "vu", "vd", "ud")}}
+    B = O.rmsnorm(_x(7, seed=13), np.ones(SH.hidden), SH.rms_eps)
+    want = O.ffn(B, Wp["w_gate"], Wp["w_up"], Wp["w_down"])
+    assert np.allclose(O.ltp_proxy(B, Wp), want, atol=1e-10)                           # all channels, full rank: f = F_FFN
+    small = replace(SH, ltp_dlow=16, ltp_rank=4)
+    P = O.proxy_build(Xc, W, small, rho=0.2)
+    assert P["ug"].shape == (4, SH.hidden) and P["vg"].shape == (16, 4)
+    assert P["vd"].shape == (4, 16) and P["ud"].shape == (SH.hidden, 4)
+    C = P["channels"]
+    assert len(C) == 16 and np.all(np.diff(C) > 0)
+    # the kept channels are the ones with the largest importance
+    assert P["importance"][C].min() >= np.delete(P["importance"], C).max()
+    g = np.asarray(W["w_gate"], np.float64)[C].T
+    assert np.isclose(np.linalg.norm(g - P["ug"].T @ P["vg"].T) ** 2, np.sum(P["sigma"]["g"][4:] ** 2), rtol=1e-10)
