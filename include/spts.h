@@ -238,6 +238,23 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
                               uint32_t flags, void* X_out, int32_t* pos_out, int32_t* orig_out,
                               int32_t* idx_out);
 
+/* Offline construction of the low-rank proxy FFN of one layer (Section 3.3, "Low-rank Proxy FFN"):
+ *   z(x) = |silu(x W_gate) * (x W_up)| for every calibration token x (rows of calib [n_cal, D], the hidden states
+ *   preceding the FFN block, storage type; they are RMS-normalised like the FFN's input);
+ *   I_j = mean of the max(1, floor(rho * n_cal)) largest z(x)[j] over the calibration tokens;
+ *   C = TopK(I, D_low) (ascending, ties to the lower channel);  W' = W[:, C] for W_gate, W_up, W_down;
+ *   W' ~ U V by truncated SVD of rank r (U has orthonormal columns, V carries the singular values).
+ * Outputs, in the layouts spts_layer_weights expects (storage type): ug, uu [r, D]; vg, vu [D_low, r];
+ * vd [r, D_low]; ud [D, r].  Optional: importance_out [Dff] fp32, channels_out [D_low] int32,
+ * sigma_out [3, D_low] fp32 (singular values of the reduced gate, up, down matrices, descending).
+ * `scratch` is caller-owned device memory of spts_proxy_scratch_bytes(desc, n_cal) bytes, 256-byte aligned.
+ * Needs ltp_dlow <= ffn_dim, ltp_dlow even, ltp_rank <= min(ltp_dlow, hidden); 0 < rho <= 1.
+ * Runs off the inference path (a few hundred small launches per matrix); asynchronous like every other call. */
+size_t spts_proxy_scratch_bytes(const spts_model_desc* desc, int n_cal);
+spts_status spts_proxy_build(spts_ctx* ctx, const spts_layer_weights* w, const void* calib, int n_cal, double rho,
+                             void* scratch, size_t scratch_bytes, float* importance_out, int32_t* channels_out,
+                             void* ug, void* vg, void* uu, void* vu, void* vd, void* ud, float* sigma_out);
+
 /* End of prefill (the output of Algorithm 1 feeds next-token prediction): RMSNorm of one
  * hidden row x [D], logits = lm_head x (fp32 [vocab], optional), token = argmax (lowest index). */
 spts_status spts_first_token(spts_ctx* ctx, const void* x_row, const void* lm_head,

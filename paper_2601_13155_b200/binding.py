@@ -61,7 +61,7 @@ EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_opti
            "spts_last_device_status", "spts_launch_count", "spts_fold_norm_gain", "spts_pap_score",
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
            "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
-           "spts_topk_select_static")
+           "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -88,6 +88,10 @@ def load_library() -> C.CDLL:
     lib.spts_ltp_score.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, vp, vp]
     lib.spts_topk_select.argtypes = [vp, vp, i32, i32, u32, vp]
     lib.spts_topk_select_static.argtypes = [vp, i32, i32, u32, vp, vp]
+    lib.spts_proxy_scratch_bytes.restype = C.c_size_t
+    lib.spts_proxy_scratch_bytes.argtypes = [C.POINTER(ModelDesc), i32]
+    lib.spts_proxy_build.argtypes = [vp, C.POINTER(LayerWeightsC), vp, i32, C.c_double, vp, C.c_size_t, vp, vp,
+                                     vp, vp, vp, vp, vp, vp, vp]
     lib.spts_layer_prefill_skip.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, i32, i32, u32,
                                             C.POINTER(KvLayerC), vp, vp, vp]
     lib.spts_msdp_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, vp, vp, vp, vp]
@@ -100,7 +104,7 @@ def load_library() -> C.CDLL:
     lib.spts_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64), C.POINTER(C.c_double),
                                      C.POINTER(C.c_double)]
     for n in EXPORTS:
-        if n not in ("spts_workspace_bytes", "spts_destroy", "spts_launch_count"):
+        if n not in ("spts_workspace_bytes", "spts_destroy", "spts_launch_count", "spts_proxy_scratch_bytes"):
             getattr(lib, n).restype = C.c_int
     return lib
 
@@ -282,6 +286,33 @@ class Spts:
         self._check(self.lib.spts_msdp_compact(self.h, _ptr(X_in), _ptr(pos_in), _ptr(orig_in), _ptr(S_mha), N,
                                                n_next, flags, _ptr(X_out), _ptr(pos_out), _ptr(orig_out),
                                                _ptr(idx_out)), "spts_msdp_compact")
+
+    def proxy_build(self, w: LayerWeights, calib, rho: float = 0.2, want_sigma: bool = False):
+        """spts_proxy_build: returns {"importance", "channels", "ug", "vg", "uu", "vu", "vd", "ud"[, "sigma"]} as
+        device tensors (the factors in the storage type and the layouts LayerWeights uses)."""
+        s = self.shape
+        n_cal = calib.shape[0]
+        nbytes = self.lib.spts_proxy_scratch_bytes(C.byref(self.desc), n_cal)
+        if nbytes == 0:
+            raise SptsError(2, "spts_proxy_scratch_bytes")
+        scratch = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        dt, dv = self.dtype, self.device
+        out = {"importance": torch.empty(s.ffn_dim, dtype=torch.float32, device=dv),
+               "channels": torch.empty(s.ltp_dlow, dtype=torch.int32, device=dv),
+               "ug": torch.empty(s.ltp_rank, s.hidden, dtype=dt, device=dv),
+               "vg": torch.empty(s.ltp_dlow, s.ltp_rank, dtype=dt, device=dv),
+               "uu": torch.empty(s.ltp_rank, s.hidden, dtype=dt, device=dv),
+               "vu": torch.empty(s.ltp_dlow, s.ltp_rank, dtype=dt, device=dv),
+               "vd": torch.empty(s.ltp_rank, s.ltp_dlow, dtype=dt, device=dv),
+               "ud": torch.empty(s.hidden, s.ltp_rank, dtype=dt, device=dv)}
+        if want_sigma:
+            out["sigma"] = torch.empty(3, s.ltp_dlow, dtype=torch.float32, device=dv)
+        self._check(self.lib.spts_proxy_build(self.h, C.byref(w.c), _ptr(calib), n_cal, float(rho), _ptr(scratch), nbytes,
+                                              _ptr(out["importance"]), _ptr(out["channels"]), _ptr(out["ug"]),
+                                              _ptr(out["vg"]), _ptr(out["uu"]), _ptr(out["vu"]), _ptr(out["vd"]),
+                                              _ptr(out["ud"]), _ptr(out.get("sigma"))), "spts_proxy_build")
+        self.stream.synchronize()                                  # scratch is released on return
+        return out
 
     def first_token(self, x_row, lm_head, logits_out=None, token_out=None):
         self._check(self.lib.spts_first_token(self.h, _ptr(x_row), _ptr(lm_head), _ptr(logits_out), _ptr(token_out)),

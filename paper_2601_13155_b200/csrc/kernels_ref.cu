@@ -135,7 +135,8 @@ ref_gemm_kernel(RefGemmArgs a, const float2* __restrict__ cs, float* __restrict_
       } else if (EPI == REF_SWIGLU) {
         float u = acc2[i][j] * rs;
         float g = v / (1.0f + expf(-v));
-        out[(size_t)gi2 * a.ldo + gj2] = from_f32<T>(g * u);
+        if (a.sal_t != nullptr) a.sal_t[(size_t)gj2 * a.ld_sal + gi2] = fabsf(g * u);
+        else out[(size_t)gi2 * a.ldo + gj2] = from_f32<T>(g * u);
       } else if (EPI == REF_RESID) {
         long dst = a.dst_idx ? (long)a.dst_idx[gi2] : (long)gi2;
         size_t o = (size_t)dst * a.ldo + gj2;

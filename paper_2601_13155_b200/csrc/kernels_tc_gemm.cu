@@ -50,6 +50,7 @@ struct TcParams {
   const float2* cs;             // rotary table [rows, 64]
   const float* q; float* logits; int ld_logits; int group;
   float* csq; int csq_parts;
+  float* sal_t; int ld_sal;     // TC_SWIGLU: write |silu(g) u| as fp32 [column, row] instead of the bf16 tile
   int* status;
   int num_m, num_n;
   int raster_group;             // tiles of the grouped dimension whose operand stays in L2 (8 or 16)
@@ -364,7 +365,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               float a = __uint_as_float(g[i]) * rs, b = __uint_as_float(u[i]) * rs;
               v[i] = a / (1.0f + expf(-a)) * b;
             }
-            store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
+            if (p.sal_t != nullptr) {
+              // saliency of the proxy construction: |silu(g) * u| in fp32, one row per channel (transposed)
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n0 + c + i < p.Nout) p.sal_t[(size_t)(n0 + c + i) * p.ld_sal + grow] = fabsf(v[i]);
+            } else {
+              store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
+            }
           }
         }
       } else if (EPI == TC_RESID) {
@@ -460,6 +468,7 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   p.rowscale = a.rowscale; p.out = a.out; p.ldo = a.ldo; p.out_t = a.out_t; p.ldt = a.ldt;
   p.cs = ctx->ws.rope_cs; p.q = a.q; p.logits = a.logits; p.ld_logits = a.ld_logits; p.group = a.group;
   p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
+  p.sal_t = a.sal_t; p.ld_sal = a.ld_sal;
   p.num_m = ceil_div(a.M, BM);
   p.num_n = ceil_div(a.Nout, NT);
   {
@@ -534,6 +543,7 @@ spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a) {
   if (ctx->encode_tiled == nullptr) return SPTS_ERR_UNSUPPORTED;
   if ((a.K % 8) || (a.lda % 8) || (reinterpret_cast<uintptr_t>(a.A) & 15) || (reinterpret_cast<uintptr_t>(a.W) & 15))
     return SPTS_ERR_SHAPE;
+  if (a.out == nullptr && epi != TC_SUMSQ && !(epi == TC_SWIGLU && a.sal_t != nullptr)) return SPTS_ERR_INVALID_ARG;
   if (a.out != nullptr && ((a.ldo % 8) || (reinterpret_cast<uintptr_t>(a.out) & 15))) return SPTS_ERR_SHAPE;
   if (a.Nout % 8) return SPTS_ERR_SHAPE;
   const bool narrow = a.Nout <= 128;       // a 128-wide tile wastes less on the skinny proxy factors

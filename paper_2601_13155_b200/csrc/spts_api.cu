@@ -2,6 +2,7 @@
 // schedule of Algorithm 1.  Everything here is host code that enqueues kernels on the context's
 // stream; no call synchronises except spts_last_device_status().
 #include <new>
+#include <cmath>
 #include <cstring>
 #include <vector>
 
@@ -94,6 +95,7 @@ struct Gemm {
   void* out_t; int ldt;
   const float* q; float* logits; int ld_logits;
   float* csq;
+  float* sal_t; int ld_sal;
 };
 
 spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
@@ -106,7 +108,7 @@ spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
     a.W = (const bf16*)g.W; a.W2 = (const bf16*)g.W2; a.M = g.M; a.Nout = g.Nout; a.K = g.K;
     a.rowscale = g.rowscale; a.out = (bf16*)g.out; a.ldo = g.ldo; a.out_t = (bf16*)g.out_t; a.ldt = g.ldt;
     a.q = g.q; a.logits = g.logits; a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads;
-    a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts;
+    a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts; a.sal_t = g.sal_t; a.ld_sal = g.ld_sal;
     return launch_tc_gemm(ctx, epi, a);
   }
   RefGemmArgs a;
@@ -115,6 +117,7 @@ spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
   a.M = g.M; a.Nout = g.Nout; a.K = g.K; a.rowscale = g.rowscale; a.out = g.out; a.ldo = g.ldo;
   a.out_t = g.out_t; a.ldt = g.ldt; a.head_dim = d.head_dim; a.q = g.q; a.logits = g.logits;
   a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads; a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts;
+  a.sal_t = g.sal_t; a.ld_sal = g.ld_sal;
   return launch_ref_gemm(ctx, epi, a);
 }
 
@@ -458,6 +461,75 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
   TRY(launch_gather_rows(ctx, X_in, idx, n_next, (int)(ctx->desc.hidden * elt_size(ctx->desc)), X_out));
   TRY(launch_gather_i32(ctx, pos_in, idx, n_next, pos_out));
   TRY(launch_gather_i32(ctx, orig_in, idx, n_next, orig_out));
+  return SPTS_OK;
+}
+
+namespace {
+constexpr int PROXY_SWEEPS = 14;
+struct ProxyScratch {
+  float* rstd; float* zt; int ld; float* importance; int32_t* channels; float* A; float* V; float* sigma;
+  int32_t* order; unsigned int* offdiag;
+};
+size_t carve_proxy(const spts_model_desc& d, int n_cal, void* base, ProxyScratch* out) {
+  Carver c{reinterpret_cast<char*>(base), 0};
+  ProxyScratch p;
+  p.ld = (int)align_up((size_t)n_cal, 32);
+  p.rstd = c.take<float>((size_t)n_cal);
+  p.zt = c.take<float>((size_t)d.ffn_dim * p.ld);
+  p.importance = c.take<float>((size_t)d.ffn_dim);
+  p.channels = c.take<int32_t>((size_t)d.ltp_dlow);
+  p.A = c.take<float>((size_t)d.ltp_dlow * d.hidden);
+  p.V = c.take<float>((size_t)d.ltp_dlow * d.ltp_dlow);
+  p.sigma = c.take<float>((size_t)d.ltp_dlow);
+  p.order = c.take<int32_t>((size_t)d.ltp_dlow);
+  p.offdiag = c.take<unsigned int>(64);
+  if (out) *out = p;
+  return align_up(c.off, 256);
+}
+}  // namespace
+
+size_t spts_proxy_scratch_bytes(const spts_model_desc* desc, int n_cal) {
+  if (desc == nullptr || n_cal < 1 || !shape_ok(*desc)) return 0;
+  return carve_proxy(*desc, n_cal, nullptr, nullptr);
+}
+
+spts_status spts_proxy_build(spts_ctx* ctx, const spts_layer_weights* w, const void* calib, int n_cal, double rho,
+                             void* scratch, size_t scratch_bytes, float* importance_out, int32_t* channels_out,
+                             void* ug, void* vg, void* uu, void* vu, void* vd, void* ud, float* sigma_out) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || calib == nullptr || scratch == nullptr || ug == nullptr || vg == nullptr || uu == nullptr ||
+      vu == nullptr || vd == nullptr || ud == nullptr || w->w_gate == nullptr || w->w_up == nullptr ||
+      w->w_down == nullptr)
+    return SPTS_ERR_INVALID_ARG;
+  const auto& d = ctx->desc;
+  if (n_cal < 1 || !(rho > 0.0) || rho > 1.0) return SPTS_ERR_INVALID_ARG;
+  if (d.ltp_dlow > d.ffn_dim || d.ltp_dlow % 2 != 0 || d.ltp_rank > d.ltp_dlow || d.ltp_rank > d.hidden) return SPTS_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(scratch) & 255) != 0 || !aligned16(calib)) return SPTS_ERR_INVALID_ARG;
+  if (carve_proxy(d, n_cal, nullptr, nullptr) > scratch_bytes) return SPTS_ERR_WORKSPACE;
+  ProxyScratch ps;
+  carve_proxy(d, n_cal, scratch, &ps);
+  float* imp = importance_out ? importance_out : ps.importance;
+  int32_t* ch = channels_out ? channels_out : ps.channels;
+  // saliency z(x) = |silu(x W_gate) * (x W_up)| of every calibration token, one row per channel
+  TRY(launch_rstd(ctx, calib, n_cal, ps.rstd));
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = calib; g.lda = d.hidden; g.a_rows = n_cal; g.W = w->w_gate; g.W2 = w->w_up; g.M = n_cal; g.Nout = d.ffn_dim;
+  g.K = d.hidden; g.rowscale = ps.rstd; g.sal_t = ps.zt; g.ld_sal = ps.ld;
+  TRY(run_gemm(ctx, REF_SWIGLU, g));
+  // channel importance: mean of the top rho-fraction per channel, then the D_low most important channels
+  int k = (int)floor(rho * (double)n_cal);
+  if (k < 1) k = 1;
+  TRY(launch_proxy_importance(ctx, ps.zt, ps.ld, n_cal, k, d.ffn_dim, imp));
+  TRY(launch_topk(ctx, imp, d.ffn_dim, d.ltp_dlow, 0u, ch, ctx->ws.topk_scratch));
+  // W' = W[:, C] ~ U V for the three projections
+  const int n = d.ltp_dlow;
+  TRY(launch_proxy_factor(ctx, w->w_gate, ch, 0, PROXY_SWEEPS, ps.A, ps.V, ps.sigma, ps.order, ps.offdiag, d.ltp_rank,
+                          ug, vg, sigma_out ? sigma_out : nullptr));
+  TRY(launch_proxy_factor(ctx, w->w_up, ch, 0, PROXY_SWEEPS, ps.A, ps.V, ps.sigma, ps.order, ps.offdiag + 16, d.ltp_rank,
+                          uu, vu, sigma_out ? sigma_out + n : nullptr));
+  TRY(launch_proxy_factor(ctx, w->w_down, ch, 1, PROXY_SWEEPS, ps.A, ps.V, ps.sigma, ps.order, ps.offdiag + 32, d.ltp_rank,
+                          ud, vd, sigma_out ? sigma_out + 2 * n : nullptr));
   return SPTS_OK;
 }
 

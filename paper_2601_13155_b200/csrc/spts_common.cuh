@@ -139,6 +139,7 @@ struct RefGemmArgs {
   int head_dim;                      // REF_ROPE: rotary table rows are indexed like A rows
   const float* q; float* logits; int ld_logits; int group;   // REF_ROPE + PAP: q [H, d], logits [H, ld]
   float* csq; int csq_parts;         // REF_SUMSQ
+  float* sal_t; int ld_sal;          // REF_SWIGLU: write |silu(g) u| as fp32 [column, row] instead of `out`
 };
 spts_status launch_ref_gemm(spts_ctx* ctx, int epi, const RefGemmArgs& a);
 spts_status launch_ref_attention(spts_ctx* ctx, const void* Q, const void* K, const void* V, int m,
@@ -151,6 +152,13 @@ spts_status launch_decode_store(spts_ctx* ctx, void* x);          // fp32 residu
 spts_status launch_decode_layer(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_layer* cache,
                                 int32_t pos);
 spts_status launch_head_logits(spts_ctx* ctx, const float* x32, const void* lm_head, float* logits);
+
+// ---- kernels_proxy.cu : offline proxy-FFN construction
+spts_status launch_proxy_importance(spts_ctx* ctx, const float* zt, int ld, int n_cal, int k, int n_channels,
+                                    float* importance);
+spts_status launch_proxy_factor(spts_ctx* ctx, const void* W, const int32_t* channels, int down, int sweeps,
+                                float* A, float* V, float* sigma, int32_t* order, unsigned int* offdiag, int r,
+                                void* u_out, void* v_out, float* sigma_sorted);
 
 // ---- kernels_tc_gemm.cu / kernels_tc_attn.cu : tcgen05 path (bf16)
 enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4 };
@@ -165,6 +173,7 @@ struct TcGemmArgs {
   bf16* out_t; int ldt;
   const float* q; float* logits; int ld_logits; int group;
   float* csq; int csq_parts;
+  float* sal_t; int ld_sal;             // TC_SWIGLU: saliency output (proxy construction)
 };
 spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
 spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,
