@@ -2,6 +2,7 @@
 
   python -m paper_2601_13155_b200.profile_case [--tokens 8192] [--dense] [--iters 1]
   python -m paper_2601_13155_b200.profile_case --decode 6 [--layers 4] [--cached 16384]
+  python -m paper_2601_13155_b200.profile_case --proxy 8192        (proxy-FFN construction on 8192 calibration tokens)
 """
 from __future__ import annotations
 
@@ -23,9 +24,12 @@ def main():
     ap.add_argument("--decode", type=int, default=0, help="run this many decode steps instead of a prefill layer")
     ap.add_argument("--layers", type=int, default=4, help="layers of the decode case")
     ap.add_argument("--cached", type=int, default=16384, help="cached tokens per layer of the decode case")
+    ap.add_argument("--proxy", type=int, default=0, help="build one layer's proxy FFN from this many calibration tokens")
     a = ap.parse_args()
     if a.decode:
         return decode_case(a)
+    if a.proxy:
+        return proxy_case(a)
     w = synth.workload("cfg2")
     shape = replace(w.shape, n_layers=1)
     dev = "cuda:0"
@@ -49,6 +53,32 @@ def main():
     for k, v in sorted(tab.items(), key=lambda kv: -kv[1]["ms"]):
         print(f"{k:12s} {v['ms'] / a.iters:8.3f} ms  {v['flops'] / max(v['ms'], 1e-9) / 1e9:8.1f} TFLOP/s  "
               f"{v['bytes'] / max(v['ms'], 1e-9) / 1e6:8.1f} GB/s")
+    print("device status", st)
+    if st != 0:
+        raise SystemExit(1)
+
+
+def proxy_case(a):
+    """spts_proxy_build of one 8B-shaped layer, timed with CUDA events after one warm-up build."""
+    w = synth.workload("cfg2")
+    shape = replace(w.shape, n_layers=1)
+    dev = "cuda:0"
+    t = synth.device_layer_weights(shape, w.seed, 0, dev)
+    lw = binding.LayerWeights.__new__(binding.LayerWeights)
+    lw.t = t
+    lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    Xc, _ = synth.device_hidden_states(w, dev, n_tokens=a.proxy)
+    lib = binding.Spts(shape, max_seq=1024)
+    lib.proxy_build(lw, Xc, rho=0.2)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = lib.launch_count()
+    e0.record()
+    lib.proxy_build(lw, Xc, rho=0.2)
+    e1.record()
+    torch.cuda.synchronize()
+    st = lib.device_status()
+    print(f"proxy build: {e0.elapsed_time(e1):.1f} ms, {lib.launch_count() - l0} launches, {a.proxy} calibration tokens, "
+          f"(D_low, r) = ({shape.ltp_dlow}, {shape.ltp_rank})")
     print("device status", st)
     if st != 0:
         raise SystemExit(1)

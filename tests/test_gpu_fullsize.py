@@ -137,3 +137,34 @@ def test_bench_last_stage_dense_ragged_layer():
     """The benchmark's last-stage shape: 11469 candidates (not a multiple of any tile), budgets clipped to the
     candidate count, so both blocks run densely without probing."""
     _run_layer_case("cfg3", 11469, 11469, 11469, 256)
+
+
+def test_proxy_build_at_the_8b_layer_shape():
+    """spts_proxy_build at the LLaMA-3.1-8B layer shape ((D_low, r) = (512, 128), 14336 channels) on 2048 synthetic
+    calibration tokens: importance in full, channel set, singular values and the rank-r products."""
+    from paper_2601_13155_b200 import binding
+    shape = replace(synth.LLAMA8B, n_layers=1)
+    wt = synth.device_layer_weights(shape, 1002, 0, dev())
+    lw = binding.LayerWeights.__new__(binding.LayerWeights)
+    lw.t = wt
+    lw.c = binding.LayerWeightsC(**{k: wt[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    w = synth.workload("cfg2")
+    Xc, _ = synth.device_hidden_states(w, dev(), n_tokens=2048)
+    lib = binding.Spts(shape, max_seq=1024)
+    got = lib.proxy_build(lw, Xc, rho=0.2, want_sigma=True)
+    assert lib.device_status() == 0
+    W = {k: wt[k].float().cpu().numpy().astype(np.float64) for k in ("w_gate", "w_up", "w_down")}
+    imp = O.proxy_channel_importance(O.proxy_saliency(host(Xc), W, shape), 0.2)
+    assert np.abs(host(got["importance"]) - imp).max() <= 1e-4 * imp.max()
+    C = got["channels"].cpu().numpy().astype(np.int64)
+    check_index_set(C, imp, shape.ltp_dlow, force_last=False)
+    want = O.proxy_build(host(Xc), W, shape, rho=0.2, channels=C)
+    sg = host(got["sigma"])
+    for row, name in ((0, "g"), (1, "u"), (2, "d")):
+        s_o = want["sigma"][name]
+        assert np.abs(sg[row] - s_o).max() <= 2e-4 * s_o[0], name
+    prod_g = host(got["ug"]).T @ host(got["vg"]).T
+    assert np.linalg.norm(prod_g - want["ug"].T @ want["vg"].T) <= 1e-2 * np.linalg.norm(W["w_gate"][C])
+    prod_d = host(got["ud"]) @ host(got["vd"])
+    assert np.linalg.norm(prod_d - want["ud"] @ want["vd"]) <= 1e-2 * np.linalg.norm(W["w_down"][:, C])
+    lib.close()
