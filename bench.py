@@ -46,9 +46,10 @@ def parse():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="spts", choices=["spts", "reference"])
-    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5", "paper"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5", "paper", "qwen2", "qwen3"])
     ap.add_argument("--no-128k", action="store_true", help="skip the 131072-token measurement added to the cfg3 line")
     ap.add_argument("--decode-steps", type=int, default=256)
+    ap.add_argument("--model", default="llama", choices=["llama", "qwen"], help="model family of --workload paper")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (debug)")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--breakdown", action="store_true", help="also print a per-operation table to stderr")
@@ -315,7 +316,7 @@ def paper_protocol_line(args, rep, dev):
     import torch
     from paper_2601_13155_b200 import binding, schedule, synth
     rank, world = rep.rank, rep.world
-    w = synth.workload("cfg3")
+    w = synth.workload("cfg3" if args.model == "llama" else "qwen3")
     shape = w.shape
     L, Nmax = shape.n_layers, w.n_tokens
     layers = []
@@ -354,9 +355,9 @@ def paper_protocol_line(args, rep, dev):
     table = {}
     for n in (8192, 16384, 24576, 32768):
         plans = {"dense": [(n, n, 0)] * L,
-                 "pap": schedule.paper_llama_plan(n, ltp=False, msdp=False),
-                 "pap_ltp": schedule.paper_llama_plan(n, msdp=False),
-                 "spts": schedule.paper_llama_plan(n)}
+                 "pap": schedule.paper_plan(args.model, n, ltp=False, msdp=False),
+                 "pap_ltp": schedule.paper_plan(args.model, n, msdp=False),
+                 "spts": schedule.paper_plan(args.model, n)}
         ms = {k: ttft(p, n, max(1, args.steps)) for k, p in plans.items()}
         kv = schedule.kv_token_layers(plans["spts"])
         table[str(n)] = {"ttft_ms": ms, "speedup_vs_dense": {k: ms["dense"] / v for k, v in ms.items() if k != "dense"},
@@ -370,16 +371,19 @@ def paper_protocol_line(args, rep, dev):
                 "n_gpus": world, "steps": max(1, args.steps), "warmup": 1, "ms_per_step": full["ttft_ms"]["spts"],
                 "ttft_ms": full["ttft_ms"]["spts"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": "paper protocol: 32-layer LLaMA-3.1-8B shape, the paper's LLaMA schedule (skip from layer "
-                                       "10, stage ends 13/18/23/28, budgets 9/7/4/2 Ki, prune to budget - 1 Ki), prompts 8K-32K",
+                "config": {"workload": f"paper protocol: {L}-layer {'LLaMA-3.1-8B' if args.model == 'llama' else 'Qwen-2.5-7B'} shape, "
+                                       f"the paper's schedule for it {schedule.PAPER_SCHEDULES[args.model]} (layers, first skip "
+                                       "layer, stage ends, budgets Ki, Ki pruned below the budget), prompts 8K-32K",
                            "global_batch": world, "seq_len": 32768, "parallelism": f"replicas x{world}",
                            "l2": "inputs larger than L2 (14 GB of weights streamed per step)"},
                 "lengths": table,
-                "paper_context": {"ttft_speedup_a800": {"pap": [1.08, 1.24, 1.35, 1.44], "pap_ltp": [1.26, 1.70, 1.98, 2.15],
-                                                         "spts": [1.35, 1.91, 2.26, 2.46]},
-                                  "kv_saving_pct": [29.7, 48.4, 55.2, 58.6],
-                                  "note": "Table 2 / Table 3 of the paper: one A800 80 GB, trained LLaMA-3.1-8B-Instruct, LongBench "
-                                          "prompts, HF Transformers + FlashAttention-2; context only"},
+                "paper_context": ({"ttft_speedup_a800": {"pap": [1.08, 1.24, 1.35, 1.44], "pap_ltp": [1.26, 1.70, 1.98, 2.15],
+                                                          "spts": [1.35, 1.91, 2.26, 2.46]},
+                                   "kv_saving_pct": [29.7, 48.4, 55.2, 58.6],
+                                   "note": "Table 2 / Table 3 of the paper: one A800 80 GB, trained LLaMA-3.1-8B-Instruct, LongBench "
+                                           "prompts, HF Transformers + FlashAttention-2; context only"} if args.model == "llama" else
+                                  {"note": "the paper gives no per-length TTFT table for Qwen-2.5-7B (average ratio 1.36x at its "
+                                           "accuracy operating point, Table 1, A800); context only"}),
                 "gpu_launches": int(lib.launch_count())}
     lib.close()
     return line
@@ -522,7 +526,7 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
             "warmup": warmup, "ms_per_step": ms_step, "ttft_ms": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
             "data": "synthetic",
-            "config": {"workload": f"{w.name}: {L}-layer LLaMA-3.1-8B shape, prompt {N}, MSDP stages at layers "
+            "config": {"workload": f"{w.name}: {L}-layer {'Qwen-2.5-7B' if shape.hidden == 3584 else 'LLaMA-3.1-8B'} shape, prompt {N}, MSDP stages at layers "
                                    f"{list(w.stage_first_layer)} with {list(w.stage_tokens)} candidates, keep "
                                    f"{w.keep_attn}/{w.keep_ffn}, LTP (D_low, r) = ({shape.ltp_dlow}, {shape.ltp_rank})",
                        "global_batch": world, "seq_len": N, "parallelism": f"replicas x{world}",

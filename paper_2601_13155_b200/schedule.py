@@ -46,31 +46,46 @@ def cache_capacities(plan, extra: int = 0):
     return [p[0] + extra for p in plan]
 
 
-def paper_llama_plan(n_prompt: int, n_layers: int = 32, ltp: bool = True, msdp: bool = True):
-    """The paper's LLaMA-3.1-8B setting (Section 4.1): layers 0-9 dense, skipping from layer 10, stage ends after
-    layers 13 / 18 / 23 / 28 with active budgets of 9 / 7 / 4 / 2 Ki tokens, each stage end pruning the candidates
-    to its budget minus 1 Ki; the layers after the last boundary keep the last budget (0-indexed layers; the
-    reading that reproduces the KV-cache sizes of Table 3).
+PAPER_SCHEDULES = {
+    # model: (layers, first skip layer, stage-end layers, active budgets in Ki tokens, Ki tokens pruned below the budget)
+    "llama": (32, 10, (13, 18, 23, 28), (9, 7, 4, 2), 1),
+    "qwen": (28, 9, (12, 16, 20, 24), (13, 10, 7, 4), 2),
+    "openpangu": (26, 11, (13, 16, 19, 22), (13, 10, 7, 4), 2),
+}
+
+
+def paper_plan(model: str, n_prompt: int, ltp: bool = True, msdp: bool = True):
+    """The schedules of the paper's implementation details (Section 4.1), 0-indexed layers: dense layers before the
+    first skip layer, then four stages ending at the given layers with fixed active budgets; each stage end prunes
+    the candidates to its budget minus the stated number of Ki tokens; the layers after the last boundary keep the
+    last budget (the reading that reproduces the KV-cache sizes of Table 3 for LLaMA).
     ltp=False leaves the FFN dense (the "PAP only" row of the paper's component ablation, Table 2);
     msdp=False keeps every token a candidate in every layer (budgets unchanged, no pruning)."""
+    n_layers, skip_from, ends, budgets_ki, prune_ki = PAPER_SCHEDULES[model]
     ki = 1024
-    budgets = (9 * ki, 7 * ki, 4 * ki, 2 * ki)
-    ends = (13, 18, 23, 28)
+    budgets = tuple(b * ki for b in budgets_ki)
     cur = n_prompt
     out = []
     for l in range(n_layers):
-        if l < 10:
+        if l < skip_from:
             out.append((cur, cur, 0))
             continue
         s = next((i for i, e in enumerate(ends) if l <= e), len(ends) - 1)
         m = min(cur, budgets[s])
         nxt = 0
         if msdp and l in ends:
-            nxt = min(cur, budgets[ends.index(l)] - ki)
+            nxt = min(cur, budgets[ends.index(l)] - prune_ki * ki)
         out.append((m, m if ltp else cur, nxt if nxt < cur else 0))
         if nxt and nxt < cur:
             cur = nxt
     return out
+
+
+def paper_llama_plan(n_prompt: int, n_layers: int = 32, ltp: bool = True, msdp: bool = True):
+    """paper_plan("llama", ...): skipping from layer 10, stage ends after layers 13 / 18 / 23 / 28, budgets
+    9 / 7 / 4 / 2 Ki, candidates pruned to budget - 1 Ki."""
+    assert n_layers == 32
+    return paper_plan("llama", n_prompt, ltp=ltp, msdp=msdp)
 
 
 def kv_token_layers(plan) -> int:

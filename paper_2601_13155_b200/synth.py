@@ -47,6 +47,11 @@ TINY = ModelShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, ffn_dim=68
                   ltp_dlow=128, ltp_rank=16, n_layers=1, vocab=512, dtype="fp32")
 LLAMA8B = ModelShape(hidden=4096, n_q_heads=32, n_kv_heads=8, head_dim=128, ffn_dim=14336,
                      ltp_dlow=512, ltp_rank=128, n_layers=32, vocab=128256, dtype="bf16")
+# the second model family the paper evaluates (Qwen-2.5-7B): 28 query / 4 KV heads (an odd GQA group of 7),
+# dimensions from the public model card, (D_low, r) from the paper's implementation details
+QWEN7B = ModelShape(hidden=3584, n_q_heads=28, n_kv_heads=4, head_dim=128, ffn_dim=18944,
+                    ltp_dlow=1024, ltp_rank=256, n_layers=28, vocab=152064, rms_eps=1e-6,
+                    rope_theta=1000000.0, dtype="bf16")
 
 
 def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
@@ -156,6 +161,13 @@ def workload(name: str) -> Workload:
     if name == "cfg3":
         n = 32768
         return Workload("cfg3", LLAMA8B, n, 1003, 328, 1, (0, 8, 16, 24),
+                        (n, round(0.75 * n), round(0.5 * n), round(0.35 * n)), 0.5, 0.4)
+    if name == "qwen2":        # one Qwen-2.5-7B-shaped layer, sized like config 2
+        s = replace(QWEN7B, n_layers=1)
+        return Workload("qwen2", s, 8192, 1012, 82, 1, (0,), (8192,), 0.5, 0.4)
+    if name == "qwen3":        # the 28-layer Qwen-shaped model on a 32768-token prompt, staged like config 3
+        n = 32768
+        return Workload("qwen3", QWEN7B, n, 1013, 328, 1, (0, 7, 14, 21),
                         (n, round(0.75 * n), round(0.5 * n), round(0.35 * n)), 0.5, 0.4)
     if name == "cfg4":
         n = 131072

@@ -113,6 +113,13 @@ def test_config2_layer_sampled_rows():
     _run_layer_case("cfg2", 8192, 4096, math.ceil(0.4 * 8192), 256)
 
 
+def test_qwen_shaped_layer_sampled_rows():
+    """One Qwen-2.5-7B-shaped layer (hidden 3584, 28 query / 4 KV heads -- an odd GQA group of 7 --, FFN 18944,
+    (D_low, r) = (1024, 256)), 8192 tokens: the paper's second model family, and tile counts that differ from the
+    8B shape's."""
+    _run_layer_case("qwen2", 8192, 4096, math.ceil(0.4 * 8192), 128)
+
+
 def test_bench_stage0_layer_sampled_rows_and_prune():
     """The benchmark's first-stage launch shape: 32768 candidates, 16384 attention rows, 13108 FFN rows; then the
     stage-end prune to 24576 candidates (Eq. 16) on the layer's own PAP score."""

@@ -18,6 +18,11 @@ SMALL_BF16 = replace(synth.LLAMA8B, hidden=512, n_q_heads=8, n_kv_heads=2, head_
                      ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
 
 
+# an odd GQA group (3 query heads per KV head): takes the one-tile attention kernel and the per-head decode attention
+ODD_GROUP_BF16 = replace(synth.LLAMA8B, hidden=384, n_q_heads=6, n_kv_heads=2, head_dim=128, ffn_dim=768,
+                         ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
+
+
 def _mk(shape, max_seq, reference=None):
     from paper_2601_13155_b200 import binding
     lib = binding.Spts(shape, max_seq=max_seq)
@@ -43,6 +48,7 @@ def _modes():
         pytest.param(SMALL_BF16, 777, 300, 211, False, id="small8b-bf16-tensorcore"),
         pytest.param(SMALL_BF16, 1024, 1024, 1024, False, id="small8b-bf16-tensorcore-dense"),
         pytest.param(SMALL_BF16, 640, 640, 200, False, id="small8b-bf16-tensorcore-attn-dense"),
+        pytest.param(ODD_GROUP_BF16, 515, 259, 130, False, id="oddgroup-bf16-tensorcore"),
     ]
 
 
@@ -105,7 +111,7 @@ def test_keep_all_equals_dense_and_is_deterministic(dtype, ref):
     lib.close()
 
 
-@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", True), ("bf16", False)])
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", True), ("bf16", False), ("bf16-oddgroup", False)])
 def test_prefill_and_decode_match_oracle(dtype, ref):
     """Algorithm 1 over four layers in two stages, then two decode steps.
 
@@ -114,7 +120,8 @@ def test_prefill_and_decode_match_oracle(dtype, ref):
     -- a boundary token swapped in an earlier layer -- would otherwise compound).  The single
     spts_prefill call must then reproduce the per-layer chain bit for bit."""
     from paper_2601_13155_b200 import binding
-    base = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    base = {"bf16": SMALL_BF16, "fp32": synth.TINY, "bf16-oddgroup": ODD_GROUP_BF16}[dtype]
+    dtype = base.dtype
     L = 4
     shape = replace(base, n_layers=L, vocab=1000)
     lib = _mk(shape, 1024, ref)
