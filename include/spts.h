@@ -57,8 +57,8 @@ enum { SPTS_BF16 = 0, SPTS_FP32 = 1 };
 enum {
   SPTS_FORCE_LAST = 1u,   /* the last candidate is always selected (it carries the output state) */
   SPTS_REFERENCE_KERNELS = 2u, /* spts_set_option: run the plain CUDA-core kernels also in bf16 mode */
-  SPTS_ATTENTION_ONE_TILE = 4u /* spts_set_option: tensor-core attention with one query tile per CTA (the variant
-                                  used for odd GQA group sizes) also where the two-head variant applies */
+  SPTS_ATTENTION_ONE_TILE = 4u /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
+                                  slower kernel kept as a cross-check of the two-tile kernel) */
 };
 
 typedef struct {

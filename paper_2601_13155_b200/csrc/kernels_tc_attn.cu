@@ -2,10 +2,12 @@
 // Index lists are ascending, so causality among the selected tokens is a lower triangle in the
 // compact row order.
 //
-// tc_attention_pair_kernel (used when the GQA group size H / Hkv is even): one CTA = 128 queries of
-// TWO query heads that share a KV head, so every K_j / V_j tile staged in shared memory feeds two
-// score tiles, and the tensor core always has the other tile's MMAs to run while one tile's
-// softmax is in progress.  grid = (H / 2, ceil(m / 128)), longest query tiles first.
+// tc_attention_pair_kernel: one CTA = two score tiles of 128 queries that read the same K / V: two
+// query heads that share a KV head (even GQA group, grid = (H / 2, ceil(m / 128))), or else two
+// consecutive query tiles of one head (grid = (H, ceil(m / 256)); the earlier tile then sits out the
+// last key block).  Every K_j / V_j tile staged in shared memory feeds two score tiles, and the
+// tensor core always has the other tile's MMAs to run while one tile's softmax is in progress.
+// Longest query tiles first.
 //   warp 0      TMA producer: both Q tiles and K_0 once, then per key block the pair (V^T_j, K_{j+1})
 //               [128 x 128 each] under one barrier
 //   warp 1      TMEM owner and single-thread MMA issuer.  TMEM columns: S_0 | S_1 | O_0 | O_1
@@ -17,9 +19,9 @@
 //               is rescaled in TMEM only when the maximum grows by more than 2^8), row sum, P_t
 //               written back to TMEM as packed bf16; at the end O_t / l goes to global memory.
 //
-// tc_attention_kernel (any group size): one CTA = 128 queries of one head, P_j staged through shared
-// memory; QK^T of block j+1 is issued before P_j V_j so the tensor core works on S_{j+1} while the
-// softmax warps process S_j.
+// tc_attention_kernel (kept as a cross-check, option SPTS_ATTENTION_ONE_TILE): one CTA = 128 queries of
+// one head, P_j staged through shared memory; QK^T of block j+1 is issued before P_j V_j so the tensor
+// core works on S_{j+1} while the softmax warps process S_j.
 #include "spts_common.cuh"
 #include "tc_ptx.cuh"
 
@@ -43,6 +45,7 @@ constexpr float RESCALE_THRESHOLD = 8.0f;    // log2 units
 
 struct AttnParams {
   int m, H, Hkv;
+  int pair_tiles;   // paired kernel: 0 = the CTA's two tiles are two heads of one KV head, 1 = two query tiles of one head
   bf16* O;          // [m, H*128]
   int* status;
 };
@@ -344,10 +347,15 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h0 = 2 * (int)blockIdx.x;                         // heads h0, h0 + 1 share a KV head
-  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;        // longest tiles first
+  // Tile t of the CTA is (head_t, query tile qt_t).  Even GQA groups: two heads that share a KV head, same query
+  // tile (both tiles see the same key blocks).  Otherwise: two consecutive query tiles of one head; tile 0 then has
+  // one key block fewer than tile 1 and sits out the last block.
+  const int yy = (int)gridDim.y - 1 - (int)blockIdx.y;        // longest tiles first
+  const int h0 = p.pair_tiles ? (int)blockIdx.x : 2 * (int)blockIdx.x;
+  const int qt0 = p.pair_tiles ? 2 * yy : yy;
+  const int dh = p.pair_tiles ? 0 : 1, dq = p.pair_tiles ? 1 : 0;   // head / query-tile step from tile 0 to tile 1
   const int kvh = h0 / (p.H / p.Hkv);
-  const int nblk = qt + 1;
+  const int nblk = qt0 + dq + 1;                               // key blocks of the longer tile
   const uint64_t t0 = globaltimer_ns();
 
   if (threadIdx.x == 0) {
@@ -375,8 +383,8 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       mbar_expect_tx(q_full, 3 * TILE_BYTES);               // both Q tiles and K_0 (K_j sits in slot (j + 1) & 1)
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
-        tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t) * TILE, qt * TILE);
-        tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t) * TILE + 64, qt * TILE);
+        tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE, (qt0 + t * dq) * TILE);
+        tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE + 64, (qt0 + t * dq) * TILE);
       }
       tma_load_2d(sK + TILE_BYTES, &tmK, q_full, kvh * TILE, 0);
       tma_load_2d(sK + TILE_BYTES + SLAB_BYTES, &tmK, q_full, kvh * TILE + 64, 0);
@@ -431,11 +439,13 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       }
       for (int j = 0; j < nblk && ok; ++j) {
         const int sv = j & 1;
-        const bool more = j + 1 < nblk;
         ok = mbar_wait(kv_full + 8 * sv, (uint32_t)(j >> 1) & 1u, abort_flag, t0);
         if (!ok) break;
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
+          const int nblk_t = qt0 + t * dq + 1;
+          if (j >= nblk_t) continue;                    // the shorter tile has no such key block
+          const bool more_t = j + 1 < nblk_t;
           // P_t arrives in P_PARTS pieces (one barrier each), so the first MMAs of P_t V_j run while
           // the softmax warps are still computing the exponentials of the later keys
 #pragma unroll
@@ -446,7 +456,7 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
             issue_pv(t, j, part);
           }
           if (!ok) break;
-          if (more) {
+          if (more_t) {
             issue_qk(t, j + 1);
             mma_commit(s_full + 8 * t);       // also covers P_t V_j: O_t is quiescent when S_t arrives
           } else {
@@ -459,7 +469,9 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     }
   } else {
     // ------------------------------------------------------------------ softmax / rescale / epilogue
-    const int t = (warp - 2) >> 2;                     // tile (head h0 + t)
+    const int t = (warp - 2) >> 2;                     // tile
+    const int qt = qt0 + t * dq, head = h0 + t * dh;
+    const int nblk_t = qt + 1;
     const int quarter = warp & 3;                      // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;
     const int qi = qt * TILE + row;                    // compact query index
@@ -470,7 +482,7 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     const float2 sc2 = make_float2(sc, sc);
     float m_used = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int j = 0; j < nblk && ok; ++j) {
+    for (int j = 0; j < nblk_t && ok; ++j) {
       ok = mbar_wait(s_full + 8 * t, (uint32_t)j & 1u, abort_flag, t0);
       if (!ok) break;
       tc_fence_after();
@@ -544,7 +556,7 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (ok) {
       tc_fence_after();
       const float inv = 1.0f / l;
-      bf16* orow = p.O + ((size_t)qi * p.H + (h0 + t)) * TILE;
+      bf16* orow = p.O + ((size_t)qi * p.H + head) * TILE;
 #pragma unroll 1
       for (int c = 0; c < TILE; c += 32) {
         uint32_t r[32];
@@ -619,9 +631,12 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
   if (!make_map(ctx, &tmK, K, (uint64_t)m, (uint64_t)KD, (uint64_t)KD)) return SPTS_ERR_CUDA;
   if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)m, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
   AttnParams p;
-  p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.O = O; p.status = ctx->ws.status;
-  if ((d.n_q_heads / d.n_kv_heads) % 2 == 0 && !ctx->attn_one_tile) {
-    dim3 grid(d.n_q_heads / 2, ceil_div(m, TILE));
+  p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.pair_tiles = 0; p.O = O; p.status = ctx->ws.status;
+  if (!ctx->attn_one_tile) {
+    // two score tiles per CTA: two heads of one KV head when the GQA group is even, else two query tiles of a head
+    p.pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 0 : 1;
+    dim3 grid(p.pair_tiles ? d.n_q_heads : d.n_q_heads / 2,
+              p.pair_tiles ? ceil_div(ceil_div(m, TILE), 2) : ceil_div(m, TILE));
     tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
   } else {
     dim3 grid(d.n_q_heads, ceil_div(m, TILE));
