@@ -195,7 +195,8 @@ def main():
             if rank == 0:
                 line["ctx_128k"] = {k: sub[k] for k in ("value", "unit", "ms_per_step", "ttft_ms", "steps", "warmup", "config",
                                                         "dense", "roofline", "algorithmic_tflop_per_step",
-                                                        "achieved_tflops_whole_step", "breakdown_ms", "gpu_launches")}
+                                                        "achieved_tflops_whole_step", "breakdown_ms", "per_operation",
+                                                        "gpu_launches")}
     if rank == 0:
         print(json.dumps(line))
     rep.close()
@@ -389,6 +390,26 @@ def paper_protocol_line(args, rep, dev):
     return line
 
 
+def per_operation(table, tensor_ops, peaks):
+    """Every operation of one instrumented prefill against the roofline that bounds it: algorithmic FLOPs (tensor-core
+    operations) or bytes (the rest) over the CUDA-event time summed over the layers, as a fraction of the measured peak
+    (sustained cuBLAS bf16 TFLOP/s, copy GB/s)."""
+    out = {}
+    tf_peak = peaks.get("bf16_tflops_sustained", 1400.0)
+    bw_peak = peaks.get("hbm_gbs", 6650.0)
+    for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"]):
+        sec = max(v["ms"], 1e-9) * 1e-3
+        if k in tensor_ops:
+            ach = v["flops"] / sec / 1e12
+            out[k] = {"ms": round(v["ms"], 3), "calls": v["calls"], "bound": "tensor", "achieved_tflops": round(ach, 1),
+                      "frac_of_measured_peak": round(ach / tf_peak, 3)}
+        else:
+            ach = v["bytes"] / sec / 1e9
+            out[k] = {"ms": round(v["ms"], 3), "calls": v["calls"], "bound": "hbm", "achieved_gbs": round(ach, 1),
+                      "frac_of_measured_peak": round(ach / bw_peak, 3)}
+    return out
+
+
 def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
     """Times `steps` whole prefills of workload `wname` (after `warmup`), the same through host buffers, and the
     dense arm; returns the JSON line as a dict (rank 0) or None."""
@@ -540,6 +561,7 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
             "algorithmic_tflop_per_step": total_flops / 1e12,
             "achieved_tflops_whole_step": total_flops / 1e12 / (ms_step * 1e-3),
             "breakdown_ms": {k: round(v["ms"], 3) for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"])},
+            "per_operation": per_operation(table, tensor_ops, peaks),
         }
         if args.breakdown:
             for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"]):
