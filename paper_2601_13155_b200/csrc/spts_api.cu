@@ -55,6 +55,7 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws) {
   w.q = c.take<float>(HD);
   w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
   w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
+  w.ugu = c.take<char>(2 * (size_t)d.ltp_rank * d.hidden * es);
   w.logits = c.take<float>((size_t)d.n_q_heads * Npad);
   w.head_stats = c.take<float>(2 * (size_t)d.n_q_heads);
   w.s_mha = c.take<float>(N);
@@ -169,7 +170,11 @@ spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   const int ld = (int)align_up((size_t)N, 128);
   const double es = (double)elt_size(d), Nd = (double)N, Dd = (double)d.hidden;
   OP(SPTS_OP_PREP, 0.0, Nd * Dd * es + 4.0 * Nd, launch_rstd(ctx, X, N, ws.rstd));
-  OP(SPTS_OP_PREP, 0.0, Nd * (4.0 + 4.0 * d.head_dim), launch_rope_table(ctx, pos, N, ws.rope_cs));
+  if (!(ctx->rope_trust && ctx->rope_pos == pos && ctx->rope_n == N)) {
+    OP(SPTS_OP_PREP, 0.0, Nd * (4.0 + 4.0 * d.head_dim), launch_rope_table(ctx, pos, N, ws.rope_cs));
+    ctx->rope_pos = pos;
+    ctx->rope_n = N;
+  }
   if (want_scores)
     OP(SPTS_OP_PREP, 2.0 * Dd * d.n_q_heads * d.head_dim, Dd * d.n_q_heads * d.head_dim * es,
        launch_q_last(ctx, X, ws.rope_cs, N, w->wq, ws.rstd, ws.q));
@@ -196,12 +201,15 @@ spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
                    Nd * d.hidden * (double)es + 3.0 * r * ((double)d.hidden + Dl) * (double)es + 8.0 * Nd);
   TRY(launch_pad_proxy(ctx, w->vg, w->vu, ws.vgu_pad));
   Gemm g;
-  // t1 = [x Ug | x Uu]  (two column blocks of one [N, 2r] matrix)
+  // t1 = [x Ug | x Uu]: the two first factors are stacked into one [2r, D] matrix so that the residual
+  // stream (the only large operand of the whole proxy) is read once
+  const size_t ubytes = (size_t)r * d.hidden * es;
+  if (cudaMemcpyAsync(ws.ugu, w->ug, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess ||
+      cudaMemcpyAsync((char*)ws.ugu + ubytes, w->uu, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+    return SPTS_ERR_CUDA;
   memset(&g, 0, sizeof(g));
-  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->ug; g.M = N; g.Nout = r; g.K = d.hidden;
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = ws.ugu; g.M = N; g.Nout = 2 * r; g.K = d.hidden;
   g.rowscale = ws.rstd; g.out = ws.t1; g.ldo = 2 * r;
-  TRY(run_gemm(ctx, REF_STORE, g));
-  g.W = w->uu; g.out = (char*)ws.t1 + (size_t)r * es;
   TRY(run_gemm(ctx, REF_STORE, g));
   // hlow = silu(t_g Vg) * (t_u Vu)
   memset(&g, 0, sizeof(g));
@@ -252,6 +260,9 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->sm_count = prop.multiProcessorCount;
   ctx->encode_tiled = nullptr;
   ctx->attn_one_tile = false;
+  ctx->rope_trust = false;
+  ctx->rope_pos = nullptr;
+  ctx->rope_n = 0;
   ctx->prof = new (std::nothrow) Profiler;
   carve(*desc, max_seq, workspace, &ctx->ws);
   ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
@@ -553,6 +564,13 @@ spts_status spts_prefill(spts_ctx* ctx, const spts_model_weights* mw, const spts
     return SPTS_ERR_INVALID_ARG;
   if (N < 1 || N > ctx->max_seq) return SPTS_ERR_SHAPE;
   const auto& d = ctx->desc;
+  // the caller's pos buffers are only written by this call's own compactions while it runs, so a rotary table
+  // stays valid until the buffers swap
+  struct RopeTrust {
+    spts_ctx* c;
+    explicit RopeTrust(spts_ctx* cc) : c(cc) { c->rope_trust = true; c->rope_pos = nullptr; }
+    ~RopeTrust() { c->rope_trust = false; c->rope_pos = nullptr; }
+  } rope_guard(ctx);
   void* xc = X; int32_t* pc = pos; int32_t* oc = orig;
   void* xa = X_alt; int32_t* pa = pos_alt; int32_t* oa = orig_alt;
   int cur = N, in_alt = 0;

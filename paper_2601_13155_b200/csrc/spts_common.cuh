@@ -52,6 +52,7 @@ struct Workspace {
   float* q;             // [H*d]
   float2* rope_cs;      // [Nmax, d/2] cos/sin of the rotary angles
   void* vgu_pad;        // [2, Dlow, 2r] zero-padded proxy factors (gate | up)
+  void* ugu;            // [2r, D] the proxy's first factors stacked (Ug^T over Uu^T): one GEMM reads x once
   float* logits;        // [H, Nmax]
   float* head_stats;    // [2*H] max and sum of exp per head
   float* s_mha;         // [Nmax]
@@ -86,6 +87,11 @@ struct spts_ctx {
   spts::Workspace ws;
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
   bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
+  // rotary table reuse inside spts_prefill: positions only change at a stage end, so the table computed for
+  // (pos pointer, N) stays valid for the following layers of the stage
+  bool rope_trust;
+  const int32_t* rope_pos;
+  int rope_n;
   int64_t launches;
   int sm_count;
   void* encode_tiled;       // cuTensorMapEncodeTiled entry point (tensor-core mode)
