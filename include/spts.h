@@ -57,6 +57,9 @@ enum { SPTS_BF16 = 0, SPTS_FP32 = 1 };
 enum {
   SPTS_FORCE_LAST = 1u,   /* the last candidate is always selected (it carries the output state) */
   SPTS_REFERENCE_KERNELS = 2u, /* spts_set_option: run the plain CUDA-core kernels also in bf16 mode */
+  SPTS_PAP_WINDOW = 8u,        /* spts_set_option: value = number of trailing queries the probe score averages over
+                                  (1..64; 1 = last token only, Eq. 4; larger windows are the query-length ablation of
+                                  Appendix C: every query attends causally, K and the queries are taken as stored) */
   SPTS_ATTENTION_ONE_TILE = 4u /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
                                   slower kernel kept as a cross-check of the two-tile kernel) */
 };
@@ -151,7 +154,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
                         size_t workspace_bytes, void* cuda_stream, spts_ctx** out);
 void spts_destroy(spts_ctx* ctx);
 
-/* Sets SPTS_REFERENCE_KERNELS or SPTS_ATTENTION_ONE_TILE on/off (value 0/1). */
+/* Sets SPTS_REFERENCE_KERNELS or SPTS_ATTENTION_ONE_TILE on/off (value 0/1), or SPTS_PAP_WINDOW (value 1..64). */
 spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value);
 
 /* Synchronises the context's stream and returns the device status word (then clears it). */

@@ -109,6 +109,28 @@ def pap_score(A, pos, wk, wq, shape):
     return K, q, S / H
 
 
+def pap_score_window(A, pos, wk, wq, shape, window, rnd=identity):
+    """The probe score with a window of query tokens (the query-length ablation of the paper's Appendix C): the
+    attention rows of the last `window` candidates, each over its causal range n <= i, averaged over the window and
+    the H heads.  window = 1 is Eq. 4.  K and the window's queries are rounded with `rnd` (they are taken as stored).
+    Returns (K [N,Hkv,d] after rnd, S [N])."""
+    N = A.shape[0]
+    H, Hkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    G = H // Hkv
+    w = min(window, N)
+    K = rnd(rope((A @ wk.T).reshape(N, Hkv, d), pos, shape.rope_theta))
+    Q = rnd(rope((A[N - w:] @ wq.T).reshape(w, H, d), pos[N - w:], shape.rope_theta))
+    S = np.zeros(N, F64)
+    for a in range(w):
+        i = N - w + a                          # the query's own index: it sees keys 0..i
+        for h in range(H):
+            z = K[: i + 1, h // G, :] @ Q[a, h] / math.sqrt(d)
+            z = z - z.max()
+            e = np.exp(z)
+            S[: i + 1] += e / e.sum()
+    return K, S / (w * H)
+
+
 # ----------------------------------------------------------------------------
 # Eq. 5 / 15 / 16: TopK
 # ----------------------------------------------------------------------------

@@ -20,6 +20,7 @@ SPTS_BF16, SPTS_FP32 = 0, 1
 FORCE_LAST = 1
 OPT_REFERENCE_KERNELS = 2
 OPT_ATTENTION_ONE_TILE = 4
+OPT_PAP_WINDOW = 8
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT",
                 6: "NONFINITE", 7: "UNSUPPORTED"}
@@ -221,6 +222,9 @@ class Spts:
     # ------------------------------------------------------------------ options / status
     def set_reference_kernels(self, on: bool):
         self._check(self.lib.spts_set_option(self.h, OPT_REFERENCE_KERNELS, 1 if on else 0), "spts_set_option")
+
+    def set_pap_window(self, window: int):
+        self._check(self.lib.spts_set_option(self.h, OPT_PAP_WINDOW, int(window)), "spts_set_option")
 
     def set_attention_one_tile(self, on: bool):
         self._check(self.lib.spts_set_option(self.h, OPT_ATTENTION_ONE_TILE, 1 if on else 0), "spts_set_option")

@@ -95,14 +95,20 @@ __global__ void q_last_kernel(const T* __restrict__ x, const T* __restrict__ wq,
 }
 
 // per-head max and sum of exp over the N logits of one head
+// Row r of the logits belongs to query (r % (w * G)) / G of a window of the last w candidates (w = 1: the last
+// token only); that query sees the keys n < N - w + 1 + query (causal).  `scale` multiplies the raw logits.
+__device__ __forceinline__ int pap_row_keys(int r, int N, int w, int G) { return N - w + 1 + (r % (w * G)) / G; }
+
 __global__ void __launch_bounds__(1024)
-pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N, float* __restrict__ stats) {
+pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N_all, int w, int G, float scale,
+                      float* __restrict__ stats) {
   __shared__ float red[32];
   __shared__ float bcast;
   const float* l = logits + (size_t)blockIdx.x * ld;
+  const int N = pap_row_keys(blockIdx.x, N_all, w, G);
   int tid = threadIdx.x;
   float m = -INFINITY;
-  for (int n = tid; n < N; n += blockDim.x) m = fmaxf(m, l[n]);
+  for (int n = tid; n < N; n += blockDim.x) m = fmaxf(m, l[n] * scale);
   m = warp_max(m);
   if ((tid & 31) == 0) red[tid >> 5] = m;
   __syncthreads();
@@ -114,7 +120,7 @@ pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N, float* __
   __syncthreads();
   m = bcast;
   float s = 0.f;
-  for (int n = tid; n < N; n += blockDim.x) s += expf(l[n] - m);
+  for (int n = tid; n < N; n += blockDim.x) s += expf(l[n] * scale - m);
   s = warp_sum(s);
   __syncthreads();
   if ((tid & 31) == 0) red[tid >> 5] = s;
@@ -127,13 +133,32 @@ pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N, float* __
 }
 
 // S[n] = (1/H) sum_h exp(l[h, n] - max_h) / sum_h      (Eq. 4)
-__global__ void pap_mean_kernel(const float* __restrict__ logits, int ld, int N, int H,
-                                const float* __restrict__ stats, float* __restrict__ S) {
+// `rows` rows of logits contribute; with accumulate the result is added to S (one pass per KV head).
+__global__ void pap_mean_kernel(const float* __restrict__ logits, int ld, int N, int rows, int w, int G, float scale,
+                                float inv_count, int accumulate, const float* __restrict__ stats,
+                                float* __restrict__ S) {
   int n = blockIdx.x * blockDim.x + threadIdx.x;
   if (n >= N) return;
   float acc = 0.f;
-  for (int h = 0; h < H; ++h) acc += expf(logits[(size_t)h * ld + n] - stats[2 * h]) / stats[2 * h + 1];
-  S[n] = acc / (float)H;
+  for (int r = 0; r < rows; ++r)
+    if (n < pap_row_keys(r, N, w, G)) acc += expf(logits[(size_t)r * ld + n] * scale - stats[2 * r]) / stats[2 * r + 1];
+  acc *= inv_count;
+  S[n] = accumulate ? S[n] + acc : acc;
+}
+
+// q_kv[kvh][i * G + g][:] = q_win[i][(kvh * G + g) * d + :]: the window's queries regrouped by KV head
+template <typename T>
+__global__ void pap_regroup_kernel(const T* __restrict__ q_win, int w, int Hkv, int G, int d, T* __restrict__ q_kv) {
+  const int total = w * Hkv * G * d;
+  for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < total; t += gridDim.x * blockDim.x) {
+    const int e = t % d, g = (t / d) % G, i = (t / (d * G)) % w, kvh = t / (d * G * w);
+    q_kv[t] = q_win[(size_t)i * Hkv * G * d + (size_t)(kvh * G + g) * d + e];
+  }
+}
+
+__global__ void iota_from_kernel(int32_t* out, int n, int first) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = first + i;
 }
 
 // C[n] = sqrt(sum_p csq[n, p]);  S_ffn[n] = C[n] * S_mha[n]      (Eq. 13-14)
@@ -241,9 +266,43 @@ spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N,
 
 spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, float* S) {
   const int H = ctx->desc.n_q_heads;
-  pap_head_stats_kernel<<<H, 1024, 0, ctx->stream>>>(logits, ld_logits, N, ctx->ws.head_stats);
+  pap_head_stats_kernel<<<H, 1024, 0, ctx->stream>>>(logits, ld_logits, N, 1, 1, 1.0f, ctx->ws.head_stats);
   SPTS_CUDA_OK(ctx);
-  pap_mean_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(logits, ld_logits, N, H, ctx->ws.head_stats, S);
+  pap_mean_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(logits, ld_logits, N, H, 1, 1, 1.0f, 1.0f / (float)H, 0,
+                                                            ctx->ws.head_stats, S);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+// One KV head's share of the windowed probe score: logits [w * G, ld] of that head's query rows against all keys
+// (raw dot products), softmax per row over its causal range, summed into S with weight 1 / (w * H).
+spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, int w, int accumulate,
+                                      float* stats, float* S) {
+  const auto& d = ctx->desc;
+  const int G = d.n_q_heads / d.n_kv_heads, rows = w * G;
+  const float scale = 1.0f / sqrtf((float)d.head_dim);
+  pap_head_stats_kernel<<<rows, 1024, 0, ctx->stream>>>(logits, ld_logits, N, w, G, scale, stats);
+  SPTS_CUDA_OK(ctx);
+  pap_mean_kernel<<<ceil_div(N, 256), 256, 0, ctx->stream>>>(logits, ld_logits, N, rows, w, G, scale,
+                                                            1.0f / (float)(w * d.n_q_heads), accumulate, stats, S);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_pap_regroup(spts_ctx* ctx, const void* q_win, int w, void* q_kv) {
+  const auto& d = ctx->desc;
+  const int G = d.n_q_heads / d.n_kv_heads;
+  const int total = w * d.n_q_heads * d.head_dim;
+  if (d.dtype == SPTS_BF16)
+    pap_regroup_kernel<bf16><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const bf16*)q_win, w, d.n_kv_heads, G, d.head_dim, (bf16*)q_kv);
+  else
+    pap_regroup_kernel<float><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const float*)q_win, w, d.n_kv_heads, G, d.head_dim, (float*)q_kv);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_iota_from(spts_ctx* ctx, int32_t* out, int n, int first) {
+  iota_from_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(out, n, first);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

@@ -28,6 +28,7 @@ ref_gemm_kernel(RefGemmArgs a, const float2* __restrict__ cs, float* __restrict_
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int row0 = blockIdx.y * RB, col0 = blockIdx.x * RB;
   const int half = a.head_dim >> 1;
+  const long ldw = a.ldw ? a.ldw : a.K;
 
   // loader mapping: thread -> (tile row r, 4 consecutive k)
   const int lr = tid >> 2, lk = (tid & 3) * 4;
@@ -60,8 +61,8 @@ ref_gemm_kernel(RefGemmArgs a, const float2* __restrict__ cs, float* __restrict_
       float va = 0.f, vb = 0.f, vb2 = 0.f;
       if (k < a.K) {
         if (a_row >= 0) va = to_f32(A[a_row * a.lda + k]);
-        if (w_row >= 0) vb = to_f32(W[w_row * a.K + k]);
-        if (DUAL && w2_row >= 0) vb2 = to_f32(Wsec[w2_row * a.K + k]);
+        if (w_row >= 0) vb = to_f32(W[w_row * ldw + k]);
+        if (DUAL && w2_row >= 0) vb2 = to_f32(Wsec[w2_row * ldw + k]);
       }
       As[lk + e][lr] = va;
       Bs[lk + e][lr] = vb;
@@ -122,6 +123,7 @@ ref_gemm_kernel(RefGemmArgs a, const float2* __restrict__ cs, float* __restrict_
       if (gj2 >= a.Nout) continue;
       float v = acc[i][j] * rs;
       if (EPI == REF_STORE) {
+        if (a.out_f32 != nullptr) { a.out_f32[(size_t)gi2 * a.ldo + gj2] = v; continue; }
         T o = from_f32<T>(v);
         out[(size_t)gi2 * a.ldo + gj2] = o;
         if (a.out_t) ((T*)a.out_t)[(size_t)gj2 * a.ldt + gi2] = o;

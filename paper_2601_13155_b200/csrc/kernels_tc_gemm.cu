@@ -50,6 +50,7 @@ struct TcParams {
   const float2* cs;             // rotary table [rows, 64]
   const float* q; float* logits; int ld_logits; int group;
   float* csq; int csq_parts;
+  float* out_f32;               // TC_STORE: write fp32 [M, ldo] instead of the bf16 tile
   float* sal_t; int ld_sal;     // TC_SWIGLU: write |silu(g) u| as fp32 [column, row] instead of the bf16 tile
   int* status;
   int num_m, num_n;
@@ -295,6 +296,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             float v[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * rs;
+            if (p.out_f32 != nullptr) {            // unrounded fp32 result (probe logits of the query window)
+              float* o = p.out_f32 + (size_t)grow * p.ldo + n0 + c;
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n0 + c + i < p.Nout) o[i] = v[i];
+              continue;
+            }
             store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
             if (p.out_t != nullptr) {
 #pragma unroll
@@ -468,7 +476,7 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   p.rowscale = a.rowscale; p.out = a.out; p.ldo = a.ldo; p.out_t = a.out_t; p.ldt = a.ldt;
   p.cs = ctx->ws.rope_cs; p.q = a.q; p.logits = a.logits; p.ld_logits = a.ld_logits; p.group = a.group;
   p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
-  p.sal_t = a.sal_t; p.ld_sal = a.ld_sal;
+  p.sal_t = a.sal_t; p.ld_sal = a.ld_sal; p.out_f32 = a.out_f32;
   p.num_m = ceil_div(a.M, BM);
   p.num_n = ceil_div(a.Nout, NT);
   {
@@ -488,7 +496,7 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   }
   CUtensorMap tmA, tmB, tmB2;
   if (!make_map(ctx, &tmA, a.A, (uint64_t)a.a_rows, (uint64_t)a.K, (uint64_t)a.lda, (uint32_t)BM)) return SPTS_ERR_CUDA;
-  if (!make_map(ctx, &tmB, a.W, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
+  if (!make_map(ctx, &tmB, a.W, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)(a.ldw ? a.ldw : a.K), (uint32_t)NT)) return SPTS_ERR_CUDA;
   if (EPI == TC_SWIGLU) {
     if (!make_map(ctx, &tmB2, a.W2, (uint64_t)a.Nout, (uint64_t)a.K, (uint64_t)a.K, (uint32_t)NT)) return SPTS_ERR_CUDA;
   } else {
@@ -543,9 +551,12 @@ spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a) {
   if (ctx->encode_tiled == nullptr) return SPTS_ERR_UNSUPPORTED;
   if ((a.K % 8) || (a.lda % 8) || (reinterpret_cast<uintptr_t>(a.A) & 15) || (reinterpret_cast<uintptr_t>(a.W) & 15))
     return SPTS_ERR_SHAPE;
-  if (a.out == nullptr && epi != TC_SUMSQ && !(epi == TC_SWIGLU && a.sal_t != nullptr)) return SPTS_ERR_INVALID_ARG;
+  if (a.out == nullptr && epi != TC_SUMSQ && !(epi == TC_SWIGLU && a.sal_t != nullptr) &&
+      !(epi == TC_STORE && a.out_f32 != nullptr))
+    return SPTS_ERR_INVALID_ARG;
+  if (a.ldw % 8) return SPTS_ERR_SHAPE;
   if (a.out != nullptr && ((a.ldo % 8) || (reinterpret_cast<uintptr_t>(a.out) & 15))) return SPTS_ERR_SHAPE;
-  if (a.Nout % 8) return SPTS_ERR_SHAPE;
+  if ((a.Nout % 8) && a.out_f32 == nullptr) return SPTS_ERR_SHAPE;
   const bool narrow = a.Nout <= 128;       // a 128-wide tile wastes less on the skinny proxy factors
   switch (epi) {
     case TC_STORE: return narrow ? launch_one<128, TC_STORE>(ctx, a) : launch_one<256, TC_STORE>(ctx, a);

@@ -56,6 +56,14 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws) {
   w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
   w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
   w.ugu = c.take<char>(2 * (size_t)d.ltp_rank * d.hidden * es);
+  {
+    const size_t G = (size_t)d.n_q_heads / d.n_kv_heads;
+    w.pw_logits = c.take<float>((size_t)PAP_MAX_WINDOW * G * Npad);
+    w.pw_stats = c.take<float>(2 * (size_t)PAP_MAX_WINDOW * G);
+    w.q_win = c.take<char>((size_t)PAP_MAX_WINDOW * HD * es);
+    w.q_kv = c.take<char>((size_t)PAP_MAX_WINDOW * HD * es);
+    w.idx_w = c.take<int32_t>(PAP_MAX_WINDOW);
+  }
   w.logits = c.take<float>((size_t)d.n_q_heads * Npad);
   w.head_stats = c.take<float>(2 * (size_t)d.n_q_heads);
   w.s_mha = c.take<float>(N);
@@ -97,6 +105,7 @@ struct Gemm {
   const float* q; float* logits; int ld_logits;
   float* csq;
   float* sal_t; int ld_sal;
+  int ldw; float* out_f32;
 };
 
 spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
@@ -110,6 +119,7 @@ spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
     a.rowscale = g.rowscale; a.out = (bf16*)g.out; a.ldo = g.ldo; a.out_t = (bf16*)g.out_t; a.ldt = g.ldt;
     a.q = g.q; a.logits = g.logits; a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads;
     a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts; a.sal_t = g.sal_t; a.ld_sal = g.ld_sal;
+    a.ldw = g.ldw; a.out_f32 = g.out_f32;
     return launch_tc_gemm(ctx, epi, a);
   }
   RefGemmArgs a;
@@ -118,7 +128,7 @@ spts_status run_gemm(spts_ctx* ctx, int epi, const Gemm& g) {
   a.M = g.M; a.Nout = g.Nout; a.K = g.K; a.rowscale = g.rowscale; a.out = g.out; a.ldo = g.ldo;
   a.out_t = g.out_t; a.ldt = g.ldt; a.head_dim = d.head_dim; a.q = g.q; a.logits = g.logits;
   a.ld_logits = g.ld_logits; a.group = d.n_q_heads / d.n_kv_heads; a.csq = g.csq; a.csq_parts = ctx->ws.csq_parts;
-  a.sal_t = g.sal_t; a.ld_sal = g.ld_sal;
+  a.sal_t = g.sal_t; a.ld_sal = g.ld_sal; a.ldw = g.ldw; a.out_f32 = g.out_f32;
   return launch_ref_gemm(ctx, epi, a);
 }
 
@@ -160,6 +170,42 @@ struct ProfScope {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Probe score averaged over the last `window` queries (the query-length ablation of the paper's Appendix C):
+// S_n = 1 / (window * H) * sum_i sum_h softmax_{n <= i}(q_{i,h} . K_n / sqrt(d)), each query over its causal range.
+// rstd and the rotary table are ready.  K and the window's queries are taken as stored (rounded to the storage
+// type); the logits of one KV head's queries against all keys are one small GEMM with fp32 output.
+spts_status pap_window_tail(spts_ctx* ctx, const spts_layer_weights* w, const void* X, int N, void* K_out, int window,
+                            float* S_out) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int HD = d.n_q_heads * d.head_dim, KD = d.n_kv_heads * d.head_dim, G = d.n_q_heads / d.n_kv_heads;
+  const int ld = (int)align_up((size_t)N, 128);
+  const size_t es = elt_size(d);
+  const double Nd = (double)N, Dd = (double)d.hidden;
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->wk; g.M = N; g.Nout = KD; g.K = d.hidden;
+  g.rowscale = ws.rstd; g.out = K_out; g.ldo = KD;
+  OP(SPTS_OP_KPROJ, 2.0 * Nd * Dd * KD, (Nd * Dd + Nd * KD + Dd * KD) * es, run_gemm(ctx, REF_ROPE, g));
+  ProfScope ps(ctx, SPTS_OP_PAP_SOFTMAX, 2.0 * Nd * window * HD + 2.0 * window * Dd * HD,
+               (Nd * KD + window * Dd) * es + 8.0 * Nd * window * d.n_q_heads);
+  TRY(launch_iota_from(ctx, ws.idx_w, window, N - window));
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.idx = ws.idx_w; g.W = w->wq; g.M = window; g.Nout = HD; g.K = d.hidden;
+  g.rowscale = ws.rstd; g.out = ws.q_win; g.ldo = HD;
+  TRY(run_gemm(ctx, REF_ROPE, g));
+  TRY(launch_pap_regroup(ctx, ws.q_win, window, ws.q_kv));
+  for (int kvh = 0; kvh < d.n_kv_heads; ++kvh) {
+    memset(&g, 0, sizeof(g));
+    g.A = (const char*)ws.q_kv + (size_t)kvh * window * G * d.head_dim * es; g.lda = d.head_dim; g.a_rows = window * G;
+    g.W = (const char*)K_out + (size_t)kvh * d.head_dim * es; g.ldw = KD;
+    g.M = window * G; g.Nout = N; g.K = d.head_dim; g.out_f32 = ws.pw_logits; g.ldo = ld;
+    TRY(run_gemm(ctx, REF_STORE, g));
+    TRY(launch_pap_window_softmax(ctx, ws.pw_logits, ld, N, window, kvh > 0 ? 1 : 0, ws.pw_stats, S_out));
+  }
+  return SPTS_OK;
+}
+
 // PAP (Eq. 4): rstd, rotary table, q of the last row, K of every row with the logits taken from
 // the unrounded keys in the projection's epilogue, then the head-mean softmax.
 spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const int32_t* pos, int N,
@@ -175,9 +221,11 @@ spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
     ctx->rope_pos = pos;
     ctx->rope_n = N;
   }
-  if (want_scores)
+  if (want_scores && (ctx->pap_window < 2 || N < 2))
     OP(SPTS_OP_PREP, 2.0 * Dd * d.n_q_heads * d.head_dim, Dd * d.n_q_heads * d.head_dim * es,
        launch_q_last(ctx, X, ws.rope_cs, N, w->wq, ws.rstd, ws.q));
+  const int window = ctx->pap_window < N ? ctx->pap_window : N;
+  if (want_scores && window > 1) return pap_window_tail(ctx, w, X, N, K_out, window, S_out);
   Gemm g;
   memset(&g, 0, sizeof(g));
   g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = w->wk; g.M = N; g.Nout = KD; g.K = d.hidden;
@@ -263,6 +311,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->rope_trust = false;
   ctx->rope_pos = nullptr;
   ctx->rope_n = 0;
+  ctx->pap_window = 1;
   ctx->prof = new (std::nothrow) Profiler;
   carve(*desc, max_seq, workspace, &ctx->ws);
   ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
@@ -321,6 +370,11 @@ spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
     if (ctx->desc.dtype == SPTS_FP32 || !tc_shape_ok(ctx->desc)) return value ? SPTS_OK : SPTS_ERR_UNSUPPORTED;
     if (!value && ctx->encode_tiled == nullptr) TRY(tc_init(ctx));
     ctx->reference_kernels = value != 0;
+    return SPTS_OK;
+  }
+  if (option == SPTS_PAP_WINDOW) {
+    if (value < 1 || value > PAP_MAX_WINDOW) return SPTS_ERR_INVALID_ARG;
+    ctx->pap_window = value;
     return SPTS_OK;
   }
   if (option == SPTS_ATTENTION_ONE_TILE) {

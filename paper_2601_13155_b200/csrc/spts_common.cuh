@@ -52,6 +52,11 @@ struct Workspace {
   float* q;             // [H*d]
   float2* rope_cs;      // [Nmax, d/2] cos/sin of the rotary angles
   void* vgu_pad;        // [2, Dlow, 2r] zero-padded proxy factors (gate | up)
+  float* pw_logits;     // [PAP_MAX_WINDOW * G, Nmax] probe logits of one KV head's window queries
+  float* pw_stats;      // [2 * PAP_MAX_WINDOW * G]
+  void* q_win;          // [PAP_MAX_WINDOW, H*d] window queries after RoPE
+  void* q_kv;           // the same regrouped by KV head
+  int32_t* idx_w;       // [PAP_MAX_WINDOW] the window's candidate indices
   void* ugu;            // [2r, D] the proxy's first factors stacked (Ug^T over Uu^T): one GEMM reads x once
   float* logits;        // [H, Nmax]
   float* head_stats;    // [2*H] max and sum of exp per head
@@ -92,6 +97,7 @@ struct spts_ctx {
   bool rope_trust;
   const int32_t* rope_pos;
   int rope_n;
+  int pap_window;           // number of trailing queries the probe averages over (1 = the paper's default)
   int64_t launches;
   int sm_count;
   void* encode_tiled;       // cuTensorMapEncodeTiled entry point (tensor-core mode)
@@ -99,6 +105,8 @@ struct spts_ctx {
 };
 
 namespace spts {
+
+static const int PAP_MAX_WINDOW = 64;         // largest query window of the probe (the paper ablates 1, 4 and 64)
 
 // top-k scratch size in uint32 words
 static const int TOPK_CHUNK = 2048;           // elements per CTA in the select / emit kernels
@@ -119,6 +127,10 @@ spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N,
                           const float* rstd, float* q);
 spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void* out);
 spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, float* S);
+spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, int w, int accumulate,
+                                      float* stats, float* S);
+spts_status launch_pap_regroup(spts_ctx* ctx, const void* q_win, int w, void* q_kv);
+spts_status launch_iota_from(spts_ctx* ctx, int32_t* out, int n, int first);
 spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
                              float* C_out, float* S_ffn);
 spts_status launch_fold_gain(spts_ctx* ctx, void* W, const float* g, int out_f, int in_f);
@@ -146,6 +158,8 @@ struct RefGemmArgs {
   const float* q; float* logits; int ld_logits; int group;   // REF_ROPE + PAP: q [H, d], logits [H, ld]
   float* csq; int csq_parts;         // REF_SUMSQ
   float* sal_t; int ld_sal;          // REF_SWIGLU: write |silu(g) u| as fp32 [column, row] instead of `out`
+  int ldw;                           // row stride of W in elements (0: K)
+  float* out_f32;                    // REF_STORE: write fp32 [M, ldo] instead of `out`
 };
 spts_status launch_ref_gemm(spts_ctx* ctx, int epi, const RefGemmArgs& a);
 spts_status launch_ref_attention(spts_ctx* ctx, const void* Q, const void* K, const void* V, int m,
@@ -180,6 +194,8 @@ struct TcGemmArgs {
   const float* q; float* logits; int ld_logits; int group;
   float* csq; int csq_parts;
   float* sal_t; int ld_sal;             // TC_SWIGLU: saliency output (proxy construction)
+  int ldw;                              // row stride of W in elements (0: K)
+  float* out_f32;                       // TC_STORE: fp32 output [M, ldo] instead of `out`
 };
 spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
 spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,

@@ -238,3 +238,36 @@ def test_tiny_and_ragged_sequences(N, ma, mf, ref):
     cache = binding.KvCache(shape, 1, N)
     check_layer_blocks(lib, shape, W, Wd, Wmid, Xd, i32(pos), ma, mf, cache)
     lib.close()
+
+
+@pytest.mark.parametrize("shape,N,ref", [
+    pytest.param(synth.TINY, 389, None, id="tiny-fp32"),
+    pytest.param(SMALL_BF16, 777, False, id="small8b-bf16-tensorcore"),
+    pytest.param(ODD_GROUP_BF16, 300, False, id="oddgroup-bf16-tensorcore"),
+    pytest.param(SMALL_BF16, 40, True, id="small8b-bf16-refkernels-short"),
+])
+@pytest.mark.parametrize("window", [4, 64])
+def test_window_probe_matches_oracle(shape, N, ref, window):
+    """The probe score averaged over the last `window` queries (SPTS_PAP_WINDOW; the paper's query-length ablation):
+    every query over its causal range, K and the queries as stored.  Also through the layer call: its S_out is the
+    windowed score and its attention set the top-k of it."""
+    from paper_2601_13155_b200 import binding
+    lib = _mk(shape, 1024, ref)
+    lib.set_pap_window(window)
+    W, X, Wd = _layer_case(shape, N, 1003, 16, std=0.05)
+    pos = (np.arange(N) * 2 + 5).astype(np.int32)
+    Xd = up(X, shape.dtype)
+    S = lib.pap_score(Wd, Xd, i32(pos))
+    A = O.rmsnorm(X, np.ones(shape.hidden), shape.rms_eps)
+    rnd = O.rounding("bf16" if shape.dtype == "bf16" else "exact")
+    _, So = O.pap_score_window(A, pos, W["wk"].astype(np.float64), W["wq"].astype(np.float64), shape, window, rnd)
+    assert np.abs(host(S) - So).max() <= 2e-4 * So.max()
+    assert abs(host(S).sum() - 1.0) < 1e-4
+    ma = max(1, N // 3)
+    S2 = torch.empty(N, dtype=torch.float32, device=dev())
+    ia = torch.empty(ma, dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip(Wd, Xd, i32(pos), ma, N, binding.KvCache(shape, 1, N), S_out=S2, idx_attn_out=ia)
+    assert torch.equal(S2, S)
+    check_index_set(ia.cpu().numpy(), So, ma)
+    assert lib.device_status() == 0
+    lib.close()

@@ -516,3 +516,30 @@ def test_proxy_build_layout_and_full_rank_limit():
     assert P["importance"][C].min() >= np.delete(P["importance"], C).max()
     g = np.asarray(W["w_gate"], np.float64)[C].T
     assert np.isclose(np.linalg.norm(g - P["ug"].T @ P["vg"].T) ** 2, np.sum(P["sigma"]["g"][4:] ** 2), rtol=1e-10)
+
+
+# ------------------------------------------------------------------ query-window probe (Appendix C ablation)
+def test_window_probe_reduces_to_eq4_and_to_dense_attention_rows():
+    W = _layer()
+    N = 29
+    X = _x(N)
+    pos = np.arange(N) * 2 + 1
+    A = O.rmsnorm(X, np.ones(SH.hidden), SH.rms_eps)
+    wk, wq = W["wk"].astype(np.float64), W["wq"].astype(np.float64)
+    _, _, S1 = O.pap_score(A, pos, wk, wq, SH)
+    _, Sw1 = O.pap_score_window(A, pos, wk, wq, SH, 1)
+    assert np.allclose(Sw1, S1, rtol=1e-12, atol=1e-15)                      # window 1 is Eq. 4
+    # independent route: the dense causal attention probability matrix by torch, mean of its last w rows and heads
+    H, Hkv, d = SH.n_q_heads, SH.n_kv_heads, SH.head_dim
+    K = O.rope((A @ wk.T).reshape(N, Hkv, d), pos, SH.rope_theta)
+    Q = O.rope((A @ wq.T).reshape(N, H, d), pos, SH.rope_theta)
+    Kt = torch.from_numpy(K).repeat_interleave(H // Hkv, dim=1)              # [N, H, d]
+    logits = torch.einsum("ihd,jhd->hij", torch.from_numpy(Q), Kt) / math.sqrt(d)
+    mask = torch.ones(N, N, dtype=torch.bool).tril()
+    P = torch.softmax(logits.masked_fill(~mask, float("-inf")), dim=-1).numpy()     # [H, N, N]
+    for w in (1, 4, 64):
+        ww = min(w, N)
+        want = P[:, N - ww:, :].mean(axis=(0, 1))
+        _, S = O.pap_score_window(A, pos, wk, wq, SH, w)
+        assert np.allclose(S, want, rtol=1e-10, atol=1e-14), w
+        assert abs(S.sum() - 1.0) < 1e-12
