@@ -4,7 +4,7 @@
 One step = one whole prefill of the 32-layer LLaMA-3.1-8B-shaped model (random-init weights,
 synthetic hidden states with heavy tokens) through Algorithm 1: per layer PAP score, top-k,
 reduced attention, LTP score, top-k, reduced FFN; stage-end pruning; first-token head.
-The default workload is BASELINE config 3 (32768-token prompt, four MSDP stages); its line also
+The default workload is configuration "cfg3" (32768-token prompt, four MSDP stages); its line also
 carries `ctx_128k`, the same measurement on config 4 (131072 tokens, one timed step).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2|cfg5] [--impl reference]
@@ -189,7 +189,7 @@ def main():
     else:
         line = prefill_line(args, rep, dev, args.workload, args.steps, max(args.warmup, 3), 2, True)
         if args.workload == "cfg3" and not args.no_128k and not args.layers:
-            # the same measurement at the longest context (BASELINE config 4), kernels already warm
+            # the same measurement at the longest context (cfg4, 131072 tokens), kernels already warm
             torch.cuda.empty_cache()
             sub = prefill_line(args, rep, dev, "cfg4", 1, 1, 0, False)
             if rank == 0:
@@ -203,7 +203,7 @@ def main():
 
 
 def generation_line(args, rep, dev):
-    """BASELINE config 5: a 32768-token prompt is prefilled (Algorithm 1), then `--decode-steps` tokens are decoded
+    """Workload cfg5: a 32768-token prompt is prefilled (Algorithm 1), then `--decode-steps` tokens are decoded
     greedily against the per-layer compressed caches; repeated for keep ratios 1.0 / 0.7 / 0.5 / 0.3 (attention
     and FFN budgets = ceil(keep * prompt), MSDP stages as in config 3) and once with skipping disabled.
     value = generated + prompt tokens per second of the whole request at keep 0.5."""

@@ -109,7 +109,7 @@ def _run_layer_case(name, N, ma, mf, n_rows):
 
 
 def test_config2_layer_sampled_rows():
-    """BASELINE config 2: one 8B-shaped layer, 8192 tokens, attention keep 0.5, FFN keep 0.4."""
+    """Workload cfg2: one 8B-shaped layer, 8192 tokens, attention keep 0.5, FFN keep 0.4."""
     _run_layer_case("cfg2", 8192, 4096, math.ceil(0.4 * 8192), 256)
 
 
