@@ -51,6 +51,27 @@ __global__ void vec_store_kernel(const float* __restrict__ x, int D, T* __restri
   if (i < D) out[i] = from_f32<T>(x[i]);
 }
 
+// Programmatic dependent launch: the kernels of a decode step are short (5-50 us), so each one lets its
+// successor start early (launch_dependents), streams the first chunk of its weights -- which no kernel writes --
+// and only then waits for its predecessor's results (dep_wait = predecessor complete, its writes visible).
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 constexpr int GV_THREADS = 256;   // 8 warps
 constexpr int GV_WARPS = 8;
 
@@ -66,10 +87,19 @@ __device__ __forceinline__ void gemv_rows(const T* (&rowp)[R], int K, const floa
 #pragma unroll
   for (int r = 0; r < R; ++r) acc[r] = 0.f;
   float ss = 0.f;
-  for (int c = (warp * 32 + lane) * V; c < K; c += GV_THREADS * V) {
-    float w[R][V];
+  const int c0 = (warp * 32 + lane) * V;
+  float w[R][V];
+  dep_launch();
+  if (c0 < K) {
 #pragma unroll
-    for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c, w[r]);      // R independent 16-byte loads in flight
+    for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c0, w[r]);     // weights do not depend on the previous kernel
+  }
+  dep_wait();                                                    // x does
+  for (int c = c0; c < K; c += GV_THREADS * V) {
+    if (c != c0) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c, w[r]);    // R independent 16-byte loads in flight
+    }
     float xv[V];
 #pragma unroll
     for (int e = 0; e < V; e += 4) {
@@ -120,24 +150,26 @@ gemv_resid_kernel(const T* __restrict__ W, int rows, int K, const float* __restr
 }
 
 // hm[j] = round(silu(rs * x . Wg[j, :]) * (rs * x . Wu[j, :])),  rs = 1 / sqrt(mean(x^2) + eps)   (Eq. 6)
+// One CTA = four gate rows and the same four up rows (eight streams, like the other kernels, so that four CTAs
+// fit on an SM).
 template <typename T>
 __global__ void __launch_bounds__(GV_THREADS)
 gemv_swiglu_kernel(const T* __restrict__ Wg, const T* __restrict__ Wu, int rows, int K, const float* __restrict__ x,
                    float eps, float* __restrict__ hm) {
-  __shared__ float dots[16];
+  __shared__ float dots[8];
   __shared__ float ss;
-  const int r0 = blockIdx.x * 8;
-  const T* rowp[16];
+  const int r0 = blockIdx.x * 4;
+  const T* rowp[8];
 #pragma unroll
-  for (int r = 0; r < 8; ++r) {
+  for (int r = 0; r < 4; ++r) {
     const size_t off = (size_t)min(r0 + r, rows - 1) * K;
     rowp[r] = Wg + off;
-    rowp[8 + r] = Wu + off;
+    rowp[4 + r] = Wu + off;
   }
-  gemv_rows<T, 16>(rowp, K, x, dots, &ss);
-  if (threadIdx.x < 8 && r0 + threadIdx.x < rows) {
+  gemv_rows<T, 8>(rowp, K, x, dots, &ss);
+  if (threadIdx.x < 4 && r0 + threadIdx.x < rows) {
     const float rs = 1.0f / sqrtf(ss / (float)K + eps);
-    const float g = dots[threadIdx.x] * rs, u = dots[8 + threadIdx.x] * rs;
+    const float g = dots[threadIdx.x] * rs, u = dots[4 + threadIdx.x] * rs;
     hm[r0 + threadIdx.x] = round_through<T>(g / (1.0f + expf(-g)) * u);
   }
 }
@@ -231,6 +263,8 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
   constexpr int NP = 4 * KPW;              // partial states per block
   __shared__ float sm_m[NP][G], sm_l[NP][G];
   __shared__ float sm_o[NP][G][D];
+  dep_launch();
+  dep_wait();                                        // q and the cache's newest row come from the previous kernel
   const int hb = blockIdx.x * G, s = blockIdx.y;
   const int kvh = hb / (H / Hkv);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -315,6 +349,8 @@ dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float
   __shared__ float f[DEC_MAX_SPLIT];
   __shared__ float red[4];
   __shared__ float Msh, Lsh;
+  dep_launch();
+  dep_wait();
   const int h = blockIdx.x, t = threadIdx.x, nw = blockDim.x >> 5;
   const float* ph = part + (size_t)h * nsplit * (d + 2);
   const float m = t < nsplit ? ph[(size_t)t * (d + 2)] : -INFINITY;
@@ -352,6 +388,11 @@ dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float
   att32[h * d + t] = round_through<T>(acc / Lsh);
 }
 
+#define LAUNCH_DEP(ctx, ...)                                                      \
+  do {                                                                            \
+    if (launch_dependent(__VA_ARGS__) != cudaSuccess) return SPTS_ERR_CUDA;       \
+    (ctx)->launches++;                                                            \
+  } while (0)
 #define TRY_DEC(...) do { spts_status s__ = (__VA_ARGS__); if (s__ != SPTS_OK) return s__; } while (0)
 
 template <typename T, int D>
@@ -364,14 +405,13 @@ spts_status launch_attn_partial(spts_ctx* ctx, const float* q32, const spts_kv_l
   const T* vc = (const T*)cache->v;
   // all query heads of a GQA group in one block when the group size is 2, 4 or 8; else one head per block
   if (group % 8 == 0)
-    dec_attn_partial_kernel<T, D, 8><<<dim3(H / 8, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+    LAUNCH_DEP(ctx, dec_attn_partial_kernel<T, D, 8>, dim3(H / 8, nsplit), dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
   else if (group % 4 == 0)
-    dec_attn_partial_kernel<T, D, 4><<<dim3(H / 4, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+    LAUNCH_DEP(ctx, dec_attn_partial_kernel<T, D, 4>, dim3(H / 4, nsplit), dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
   else if (group % 2 == 0)
-    dec_attn_partial_kernel<T, D, 2><<<dim3(H / 2, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
+    LAUNCH_DEP(ctx, dec_attn_partial_kernel<T, D, 2>, dim3(H / 2, nsplit), dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
   else
-    dec_attn_partial_kernel<T, D, 1><<<dim3(H, nsplit), 128, 0, st>>>(q32, kc, vc, len, H, Hkv, nsplit, part);
-  SPTS_CUDA_OK(ctx);
+    LAUNCH_DEP(ctx, dec_attn_partial_kernel<T, D, 1>, dim3(H, nsplit), dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
   return SPTS_OK;
 }
 
@@ -390,24 +430,21 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
   const int slot = cache->len;
   const int per_head = hd / 8;
   const int qkv_blocks = (H + Hkv) * per_head + ceil_div(Hkv * hd, 8);
-  dec_qkv_kernel<T><<<qkv_blocks, GV_THREADS, 0, st>>>((const T*)w->wq, (const T*)w->wk, (const T*)w->wv, H, Hkv, hd, D,
-                                                        x32, d.rms_eps, pos, (double)d.rope_theta, q32, (T*)cache->k,
-                                                        (T*)cache->v, cache->pos, slot);
-  SPTS_CUDA_OK(ctx);
+  LAUNCH_DEP(ctx, dec_qkv_kernel<T>, dim3(qkv_blocks), dim3(GV_THREADS), st, (const T*)w->wq, (const T*)w->wk,
+             (const T*)w->wv, H, Hkv, hd, D, (const float*)x32, d.rms_eps, (int)pos, (double)d.rope_theta, q32,
+             (T*)cache->k, (T*)cache->v, cache->pos, slot);
   cache->len = slot + 1;
   const int len = cache->len;
   const int nsplit = min(DEC_MAX_SPLIT, max(1, len / 128));
   if (hd == 128) TRY_DEC(launch_attn_partial<T, 128>(ctx, q32, cache, len, nsplit, part));
   else TRY_DEC(launch_attn_partial<T, 64>(ctx, q32, cache, len, nsplit, part));
-  dec_attn_combine_kernel<T><<<H, hd, 0, st>>>(part, nsplit, hd, att32);
-  SPTS_CUDA_OK(ctx);
-  gemv_resid_kernel<T><<<ceil_div(D, 8), GV_THREADS, 0, st>>>((const T*)w->wo, D, H * hd, att32, x32);
-  SPTS_CUDA_OK(ctx);
-  gemv_swiglu_kernel<T><<<ceil_div(Dff, 8), GV_THREADS, 0, st>>>((const T*)w->w_gate, (const T*)w->w_up, Dff, D, x32,
-                                                                  d.rms_eps, hm32);
-  SPTS_CUDA_OK(ctx);
-  gemv_resid_kernel<T><<<ceil_div(D, 8), GV_THREADS, 0, st>>>((const T*)w->w_down, D, Dff, hm32, x32);
-  SPTS_CUDA_OK(ctx);
+  LAUNCH_DEP(ctx, dec_attn_combine_kernel<T>, dim3(H), dim3(hd), st, (const float*)part, nsplit, hd, att32);
+  LAUNCH_DEP(ctx, gemv_resid_kernel<T>, dim3(ceil_div(D, 8)), dim3(GV_THREADS), st, (const T*)w->wo, D, H * hd,
+             (const float*)att32, x32);
+  LAUNCH_DEP(ctx, gemv_swiglu_kernel<T>, dim3(ceil_div(Dff, 4)), dim3(GV_THREADS), st, (const T*)w->w_gate,
+             (const T*)w->w_up, Dff, D, (const float*)x32, d.rms_eps, hm32);
+  LAUNCH_DEP(ctx, gemv_resid_kernel<T>, dim3(ceil_div(D, 8)), dim3(GV_THREADS), st, (const T*)w->w_down, D, Dff,
+             (const float*)hm32, x32);
   return SPTS_OK;
 }
 
