@@ -52,7 +52,7 @@ __global__ void vec_store_kernel(const float* __restrict__ x, int D, T* __restri
 }
 
 // Programmatic dependent launch: the kernels of a decode step are short (5-50 us), so each one lets its
-// successor start early (launch_dependents), streams the first chunk of its weights -- which no kernel writes --
+// successor start early (launch_dependents), prefetches its weights -- which no kernel writes -- into L2
 // and only then waits for its predecessor's results (dep_wait = predecessor complete, its writes visible).
 __device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -88,18 +88,17 @@ __device__ __forceinline__ void gemv_rows(const T* (&rowp)[R], int K, const floa
   for (int r = 0; r < R; ++r) acc[r] = 0.f;
   float ss = 0.f;
   const int c0 = (warp * 32 + lane) * V;
-  float w[R][V];
   dep_launch();
-  if (c0 < K) {
-#pragma unroll
-    for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c0, w[r]);     // weights do not depend on the previous kernel
-  }
-  dep_wait();                                                    // x does
+  // the weights do not depend on the previous kernel: pull this thread's chunks towards L2 while it finishes
   for (int c = c0; c < K; c += GV_THREADS * V) {
-    if (c != c0) {
 #pragma unroll
-      for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c, w[r]);    // R independent 16-byte loads in flight
-    }
+    for (int r = 0; r < R; ++r) asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp[r] + c));
+  }
+  dep_wait();                                                    // x does depend on it
+  for (int c = c0; c < K; c += GV_THREADS * V) {
+    float w[R][V];
+#pragma unroll
+    for (int r = 0; r < R; ++r) ld16<T>(rowp[r] + c, w[r]);      // R independent 16-byte loads in flight
     float xv[V];
 #pragma unroll
     for (int e = 0; e < V; e += 4) {
