@@ -100,3 +100,49 @@ def test_compact_matches_oracle(dtype):
         assert np.all(np.diff(po.cpu().numpy()) > 0) if kk > 1 else True
     assert lib.device_status() == 0
     lib.close()
+
+
+def test_host_detectable_errors_are_returned_before_any_launch():
+    """Bad shapes, undersized caches and misaligned pointers come back as status codes (nothing is launched, the
+    buffers stay untouched, the device status stays clean)."""
+    from paper_2601_13155_b200 import binding
+    from paper_2601_13155_b200.binding import SptsError
+    shape = synth.TINY
+    lib = binding.Spts(shape, max_seq=256)
+    W = synth.layer_weights(shape, 3, 0)
+    Wd = binding.LayerWeights(W, shape.dtype)
+    N = 128
+    X, _ = synth.hidden_states(shape, N, 3)
+    Xd = up(X, shape.dtype)
+    X0 = Xd.clone()
+    pos = i32(np.arange(N))
+    launches = lib.launch_count()
+
+    def code(fn):
+        with pytest.raises(SptsError) as e:
+            fn()
+        return e.value.code
+
+    small = binding.KvCache(shape, 1, 16)
+    assert code(lambda: lib.layer_prefill_skip(Wd, Xd, pos, 64, 64, small)) == 3            # WORKSPACE: cache too small
+    ok = binding.KvCache(shape, 1, N)
+    assert code(lambda: lib.layer_prefill_skip(Wd, Xd, pos, 0, 64, ok)) == 1                # INVALID_ARG: m_attn < 1
+    assert code(lambda: lib.layer_prefill_skip(Wd, Xd, pos, N + 1, 64, ok)) == 1            # INVALID_ARG: m_attn > N
+    big = up(synth.hidden_states(shape, 300, 4)[0], shape.dtype)
+    assert code(lambda: lib.pap_score(Wd, big, i32(np.arange(300)))) == 2                    # SHAPE: N > max_seq
+    odd = torch.empty(N * shape.hidden + 1, dtype=lib.dtype, device=dev())[1:].view(N, shape.hidden)
+    assert code(lambda: lib.pap_score(Wd, odd, pos)) == 1                                    # INVALID_ARG: misaligned X
+    S = torch.zeros(N, device=dev())
+    Xo = torch.empty(N, shape.hidden, dtype=lib.dtype, device=dev())
+    assert code(lambda: lib.msdp_compact(Xd, pos, pos.clone(), S, 64, Xd, pos.clone(), pos.clone())) == 1   # aliasing
+    with pytest.raises(SptsError):
+        binding.Spts(replace_shape(shape, head_dim=96), max_seq=64)                           # unsupported shape
+    assert lib.launch_count() == launches
+    assert torch.equal(Xd, X0)
+    assert lib.device_status() == 0
+    lib.close()
+
+
+def replace_shape(shape, **kw):
+    from dataclasses import replace
+    return replace(shape, **kw)
