@@ -140,6 +140,12 @@ def test_bench_stage0_layer_sampled_rows_and_prune():
     lib.close()
 
 
+def test_bench_128k_stage0_layer_sampled_rows():
+    """The longest context's first-stage launch shape (131072 candidates in 64-token heavy clusters, 65536 attention
+    rows, 52429 FFN rows): scores and index sets in full, updates on sampled rows."""
+    _run_layer_case("cfg4", 131072, 65536, math.ceil(0.4 * 131072), 64)
+
+
 def test_bench_last_stage_dense_ragged_layer():
     """The benchmark's last-stage shape: 11469 candidates (not a multiple of any tile), budgets clipped to the
     candidate count, so both blocks run densely without probing."""
