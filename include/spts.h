@@ -29,6 +29,11 @@
  *     (a bounded wait that expired, a non-finite score) set a status word that
  *     spts_last_device_status() returns after synchronising the stream; kernels never trap.
  *   - Pointers must be 16-byte aligned; rows of X, K, V are contiguous.
+ *   - A context is bound to one device and one stream and is not thread-safe: calls on one context must
+ *     not overlap on the host.  Contexts on different streams are independent (each has its workspace).
+ *     spts_layer_prefill_skip() and spts_prefill() use the context's workspace for every intermediate
+ *     (K of all candidates, the selected rows' Q, the attention output, the SwiGLU intermediate, scores,
+ *     index lists), so the workspace grows with max_seq: about 56 KiB per candidate at the 8B shape.
  */
 #ifndef SPTS_H_
 #define SPTS_H_
