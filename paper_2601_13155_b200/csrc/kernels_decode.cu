@@ -38,6 +38,23 @@ template <> __device__ __forceinline__ void ld16<bf16>(const bf16* p, float* out
   }
 }
 
+// The same, read at L2 (ld.global.cg): for data written by the kernel just before this one.  Kernels of a chain of
+// programmatic dependents overlap, so an L1 line of this SM may be older than the predecessor's write.
+template <typename T> __device__ __forceinline__ void ld16_cg(const T* p, float* out);
+template <> __device__ __forceinline__ void ld16_cg<float>(const float* p, float* out) {
+  float4 v = __ldcg(reinterpret_cast<const float4*>(p));
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <> __device__ __forceinline__ void ld16_cg<bf16>(const bf16* p, float* out) {
+  uint4 v = __ldcg(reinterpret_cast<const uint4*>(p));
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    out[2 * i] = __uint_as_float(w[i] << 16);
+    out[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
 template <typename T> __device__ __forceinline__ float round_through(float v) { return to_f32(from_f32<T>(v)); }
 
 template <typename T>
@@ -49,27 +66,6 @@ template <typename T>
 __global__ void vec_store_kernel(const float* __restrict__ x, int D, T* __restrict__ out) {
   int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < D) out[i] = from_f32<T>(x[i]);
-}
-
-// Programmatic dependent launch: the kernels of a decode step are short (5-50 us), so each one lets its
-// successor start early (launch_dependents), prefetches its weights -- which no kernel writes -- into L2
-// and only then waits for its predecessor's results (dep_wait = predecessor complete, its writes visible).
-__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-template <typename... KArgs, typename... Args>
-cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 constexpr int GV_THREADS = 256;   // 8 warps
@@ -102,7 +98,7 @@ __device__ __forceinline__ void gemv_rows(const T* (&rowp)[R], int K, const floa
     float xv[V];
 #pragma unroll
     for (int e = 0; e < V; e += 4) {
-      float4 t = __ldg(reinterpret_cast<const float4*>(x + c + e));
+      float4 t = __ldcg(reinterpret_cast<const float4*>(x + c + e));   // x comes from the previous kernel: read at L2
       xv[e] = t.x; xv[e + 1] = t.y; xv[e + 2] = t.z; xv[e + 3] = t.w;
     }
 #pragma unroll
@@ -144,7 +140,7 @@ gemv_resid_kernel(const T* __restrict__ W, int rows, int K, const float* __restr
   gemv_rows<T, 8>(rowp, K, x, dots, &ss);
   if (threadIdx.x < 8 && r0 + threadIdx.x < rows) {
     const int j = r0 + threadIdx.x;
-    out[j] = round_through<T>(out[j] + dots[threadIdx.x]);
+    out[j] = round_through<T>(__ldcg(&out[j]) + dots[threadIdx.x]);
   }
 }
 
@@ -275,7 +271,7 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
   for (int g = 0; g < G; ++g) {
     m[g] = -INFINITY; l[g] = 0.f;
 #pragma unroll
-    for (int e = 0; e < V; ++e) { q[g][e] = q32[(hb + g) * D + li * V + e] * scale; o[g][e] = 0.f; }
+    for (int e = 0; e < V; ++e) { q[g][e] = __ldcg(&q32[(hb + g) * D + li * V + e]) * scale; o[g][e] = 0.f; }
   }
   const size_t rstride = (size_t)Hkv * D;
   const T* kbase = kc + (size_t)kvh * D + li * V;
@@ -286,10 +282,10 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
     const int ja = jw + sub, jb = ja + STEP;
     const bool hasa = ja < j1, hasb = jb < j1;
     float ka[V], va[V], kb[V], vb[V];
-    ld16<T>(kbase + (size_t)(hasa ? ja : j0) * rstride, ka);
-    ld16<T>(vbase + (size_t)(hasa ? ja : j0) * rstride, va);
-    ld16<T>(kbase + (size_t)(hasb ? jb : j0) * rstride, kb);
-    ld16<T>(vbase + (size_t)(hasb ? jb : j0) * rstride, vb);
+    ld16_cg<T>(kbase + (size_t)(hasa ? ja : j0) * rstride, ka);      // the newest row is the previous kernel's
+    ld16_cg<T>(vbase + (size_t)(hasa ? ja : j0) * rstride, va);
+    ld16_cg<T>(kbase + (size_t)(hasb ? jb : j0) * rstride, kb);
+    ld16_cg<T>(vbase + (size_t)(hasb ? jb : j0) * rstride, vb);
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       float da = 0.f, db = 0.f;
@@ -352,7 +348,7 @@ dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float
   dep_wait();
   const int h = blockIdx.x, t = threadIdx.x, nw = blockDim.x >> 5;
   const float* ph = part + (size_t)h * nsplit * (d + 2);
-  const float m = t < nsplit ? ph[(size_t)t * (d + 2)] : -INFINITY;
+  const float m = t < nsplit ? __ldcg(&ph[(size_t)t * (d + 2)]) : -INFINITY;
   float v = warp_max(m);
   if ((t & 31) == 0) red[t >> 5] = v;
   __syncthreads();
@@ -364,7 +360,7 @@ dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float
   __syncthreads();
   const float fs = m == -INFINITY ? 0.f : expf(m - Msh);
   if (t < nsplit) f[t] = fs;
-  v = warp_sum(t < nsplit ? ph[(size_t)t * (d + 2) + 1] * fs : 0.f);
+  v = warp_sum(t < nsplit ? __ldcg(&ph[(size_t)t * (d + 2) + 1]) * fs : 0.f);
   __syncthreads();                       // red[] has been read by thread 0
   if ((t & 31) == 0) red[t >> 5] = v;
   __syncthreads();
@@ -379,11 +375,11 @@ dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float
   for (; s0 + 8 <= nsplit; s0 += 8) {
     float x[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = ph[(size_t)(s0 + u) * (d + 2) + 2 + t];
+    for (int u = 0; u < 8; ++u) x[u] = __ldcg(&ph[(size_t)(s0 + u) * (d + 2) + 2 + t]);
 #pragma unroll
     for (int u = 0; u < 8; ++u) acc = fmaf(x[u], f[s0 + u], acc);
   }
-  for (; s0 < nsplit; ++s0) acc = fmaf(ph[(size_t)s0 * (d + 2) + 2 + t], f[s0], acc);
+  for (; s0 < nsplit; ++s0) acc = fmaf(__ldcg(&ph[(size_t)s0 * (d + 2) + 2 + t]), f[s0], acc);
   att32[h * d + t] = round_through<T>(acc / Lsh);
 }
 

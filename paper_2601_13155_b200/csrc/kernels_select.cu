@@ -48,19 +48,26 @@ topk_hist_kernel(const float* __restrict__ scores, int N, int k, int pass, int f
   __shared__ bool is_last;
   const int tid = threadIdx.x;
   h[tid] = 0;
-  __syncthreads();
+  // the passes of one selection run as programmatic dependents: the scores were complete before pass 0 started,
+  // so they are read before waiting for the previous pass's bucket choice
+  dep_launch();
   const int shift = 24 - 8 * pass;
   const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (32 - 8 * pass));
-  const uint32_t prefix = pass == 0 ? 0u : sc[SC_PREFIX];
   bool nonfinite = false;
   const int base = blockIdx.x * TOPK_CHUNK;
+  uint32_t keys[TK_PER_THREAD];
 #pragma unroll
   for (int e = 0; e < TK_PER_THREAD; ++e) {
-    int i = base + e * TK_THREADS + tid;
-    if (i < N) {
-      uint32_t key = load_key(scores, i, N, force_last != 0, &nonfinite);
-      if ((key & mask) == prefix) atomicAdd(&h[(key >> shift) & 0xFFu], 1u);
-    }
+    const int i = base + e * TK_THREADS + tid;
+    keys[e] = i < N ? load_key(scores, i, N, force_last != 0, &nonfinite) : 0u;
+  }
+  dep_wait();
+  __syncthreads();
+  const uint32_t prefix = pass == 0 ? 0u : __ldcg(&sc[SC_PREFIX]);   // L2: this SM's L1 may hold the older value
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    const int i = base + e * TK_THREADS + tid;
+    if (i < N && (keys[e] & mask) == prefix) atomicAdd(&h[(keys[e] >> shift) & 0xFFu], 1u);
   }
   if (nonfinite && pass == 0) set_status(status, SPTS_ERR_NONFINITE);
   __syncthreads();
@@ -103,19 +110,26 @@ topk_count_kernel(const float* __restrict__ scores, int N, int force_last, uint3
   __shared__ uint32_t carry_out, carry_eq;
   __shared__ uint32_t sa[TK_THREADS], sb[TK_THREADS];
   const int tid = threadIdx.x;
-  const uint32_t T = sc[SC_PREFIX];
   uint32_t* cta_a = sc + SC_CTA;
   uint32_t* cta_b = sc + SC_CTA + TOPK_MAX_CTAS;
   bool nf = false;
-  uint32_t gt = 0, eq = 0;
   const int base = blockIdx.x * TOPK_CHUNK;
+  dep_launch();
+  uint32_t keys[TK_PER_THREAD];
 #pragma unroll
   for (int e = 0; e < TK_PER_THREAD; ++e) {
-    int i = base + e * TK_THREADS + tid;
+    const int i = base + e * TK_THREADS + tid;
+    keys[e] = i < N ? load_key(scores, i, N, force_last != 0, &nf) : 0u;
+  }
+  dep_wait();                                  // the threshold comes from the last histogram pass
+  const uint32_t T = __ldcg(&sc[SC_PREFIX]);   // (read at L2: an L1 line may predate the previous kernel's write)
+  uint32_t gt = 0, eq = 0;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) {
+    const int i = base + e * TK_THREADS + tid;
     if (i < N) {
-      uint32_t key = load_key(scores, i, N, force_last != 0, &nf);
-      gt += key > T;
-      eq += key == T;
+      gt += keys[e] > T;
+      eq += keys[e] == T;
     }
   }
   gt = __reduce_add_sync(0xffffffffu, gt);
@@ -176,21 +190,24 @@ topk_emit_kernel(const float* __restrict__ scores, int N, int k, int force_last,
                  const uint32_t* __restrict__ sc, int32_t* __restrict__ idx_out) {
   __shared__ uint32_t s_sel[TK_THREADS], s_eq[TK_THREADS];
   const int tid = threadIdx.x;
-  const uint32_t T = sc[SC_PREFIX];
-  const uint32_t need_eq = sc[SC_KREM];
-  const uint32_t out_base = sc[SC_CTA + blockIdx.x];
-  const uint32_t eq_base = sc[SC_CTA + TOPK_MAX_CTAS + blockIdx.x];
   bool nf = false;
   // thread t owns TK_PER_THREAD consecutive elements so that a scan over threads is index order
   const int i0 = blockIdx.x * TOPK_CHUNK + tid * TK_PER_THREAD;
+  dep_launch();
   uint32_t keys[TK_PER_THREAD];
-  uint32_t eq = 0;
 #pragma unroll
   for (int e = 0; e < TK_PER_THREAD; ++e) {
-    int i = i0 + e;
+    const int i = i0 + e;
     keys[e] = i < N ? load_key(scores, i, N, force_last != 0, &nf) : 0u;
-    eq += (i < N && keys[e] == T);
   }
+  dep_wait();                                  // offsets come from the count kernel
+  const uint32_t T = __ldcg(&sc[SC_PREFIX]);
+  const uint32_t need_eq = __ldcg(&sc[SC_KREM]);
+  const uint32_t out_base = __ldcg(&sc[SC_CTA + blockIdx.x]);
+  const uint32_t eq_base = __ldcg(&sc[SC_CTA + TOPK_MAX_CTAS + blockIdx.x]);
+  uint32_t eq = 0;
+#pragma unroll
+  for (int e = 0; e < TK_PER_THREAD; ++e) eq += (i0 + e < N && keys[e] == T);
   s_eq[tid] = eq;
   __syncthreads();
   for (int o = 1; o < TK_THREADS; o <<= 1) {
@@ -266,14 +283,21 @@ spts_status launch_topk(spts_ctx* ctx, const float* scores, int N, int k, uint32
   }
   const int fl = (flags & SPTS_FORCE_LAST) ? 1 : 0;
   if (cudaMemsetAsync(scratch, 0, (4 * 256 + 16) * sizeof(uint32_t), st) != cudaSuccess) return SPTS_ERR_CUDA;
-  for (int pass = 0; pass < 4; ++pass) {
-    topk_hist_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, pass, fl, scratch, ctx->ws.status);
-    SPTS_CUDA_OK(ctx);
+  topk_hist_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, 0, fl, scratch, ctx->ws.status);   // after the memset
+  SPTS_CUDA_OK(ctx);
+  for (int pass = 1; pass < 4; ++pass) {
+    if (launch_dependent(topk_hist_kernel, dim3(nb), dim3(TK_THREADS), st, scores, N, k, pass, fl, scratch,
+                         ctx->ws.status) != cudaSuccess)
+      return SPTS_ERR_CUDA;
+    ctx->launches++;
   }
-  topk_count_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, fl, scratch);
-  SPTS_CUDA_OK(ctx);
-  topk_emit_kernel<<<nb, TK_THREADS, 0, st>>>(scores, N, k, fl, scratch, idx_out);
-  SPTS_CUDA_OK(ctx);
+  if (launch_dependent(topk_count_kernel, dim3(nb), dim3(TK_THREADS), st, scores, N, fl, scratch) != cudaSuccess)
+    return SPTS_ERR_CUDA;
+  ctx->launches++;
+  if (launch_dependent(topk_emit_kernel, dim3(nb), dim3(TK_THREADS), st, scores, N, k, fl, (const uint32_t*)scratch,
+                       idx_out) != cudaSuccess)
+    return SPTS_ERR_CUDA;
+  ctx->launches++;
   return SPTS_OK;
 }
 

@@ -203,6 +203,28 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
 spts_status tc_init(spts_ctx* ctx);          // resolves the tensor-map encoder, sets kernel attributes
 int tc_sumsq_parts(int n_out);               // partial sums per row written by TC_SUMSQ
 
+// Programmatic dependent launch for chains of short kernels (the decode step, the passes of a top-k): a kernel
+// lets its successor start early (dep_launch), does whatever does not depend on its predecessor (prefetching
+// weights, loading keys) and only then waits for the predecessor's results (dep_wait = predecessor complete,
+// its writes visible; a no-op in a kernel that was launched the ordinary way).
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 #define SPTS_CUDA_OK(ctx)                                   \
   do {                                                      \
     cudaError_t e__ = cudaGetLastError();                   \
