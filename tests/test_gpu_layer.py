@@ -271,3 +271,39 @@ def test_window_probe_matches_oracle(shape, N, ref, window):
     check_index_set(ia.cpu().numpy(), So, ma)
     assert lib.device_status() == 0
     lib.close()
+
+
+def test_decode_steps_are_reproducible_bit_for_bit():
+    """The decode kernels of a step overlap (programmatic dependent launches): two runs from the same caches must still
+    give identical logits and tokens, step after step."""
+    from paper_2601_13155_b200 import binding
+    L = 3
+    shape = replace(SMALL_BF16, n_layers=L, vocab=2000)
+    lib = _mk(shape, 1024, False)
+    layers = [synth.layer_weights(shape, 1020, l, std=0.03) for l in range(L)]
+    hw = synth.head_weights(shape, 1020)
+    lws = [binding.LayerWeights(w, "bf16") for w in layers]
+    model = binding.Model(lws, up(hw["lm_head"], "bf16"), up(hw["embed"], "bf16"))
+    n0, steps = 700, 12
+    rng = np.random.default_rng(8)
+    k0 = [up(rng.standard_normal((n0, shape.n_kv_heads, shape.head_dim)).astype(np.float32), "bf16") for _ in range(L)]
+    v0 = [up(rng.standard_normal((n0, shape.n_kv_heads, shape.head_dim)).astype(np.float32), "bf16") for _ in range(L)]
+    runs = []
+    for _ in range(2):
+        cache = binding.KvCache(shape, L, n0 + steps)
+        for l in range(L):
+            cache.k[l][:n0].copy_(k0[l])
+            cache.v[l][:n0].copy_(v0[l])
+            cache.c[l].len = n0
+        tok = torch.zeros(1, dtype=torch.int32, device=dev())
+        out, t_in = [], 11
+        for i in range(steps):
+            lg = torch.empty(shape.vocab, dtype=torch.float32, device=dev())
+            lib.decode_step(model, cache, n0 + i, token_in=t_in, logits_out=lg, token_out=tok)
+            t_in = int(tok.item())
+            out.append((lg.clone(), t_in))
+        runs.append(out)
+    for (a, ta), (b, tb) in zip(*runs):
+        assert ta == tb and torch.equal(a, b)
+    assert lib.device_status() == 0
+    lib.close()
