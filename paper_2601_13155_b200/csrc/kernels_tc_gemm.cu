@@ -371,7 +371,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               float a = __uint_as_float(g[i]) * rs, b = __uint_as_float(u[i]) * rs;
-              v[i] = a / (1.0f + expf(-a)) * b;
+              v[i] = __fdividef(a, 1.0f + __expf(-a)) * b;   // fast exp / divide: ~1e-6 relative, far below the bf16 store
             }
             if (p.sal_t != nullptr) {
               // saliency of the proxy construction: |silu(g) * u| in fp32, one row per channel (transposed)
