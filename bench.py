@@ -34,9 +34,9 @@ import numpy as np
 
 # (workload, operation) -> DRAM bytes of one launch at the workload's stage-0 shape, measured with ncu
 NCU_TRAFFIC_BYTES = {
-    ("cfg3", "gate_up"): 1169.80e6 + 360.51e6,      # tc_gemm_kernel<256, 2, 1>, m_ffn = 13108
-    ("cfg3", "attention"): 359.22e6 + 102.68e6,     # tc_attention_pair_kernel, m_attn = 16384
-    ("cfg3", "down"): 1627.49e6 + 99.70e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
+    ("cfg3", "gate_up"): 1093.77e6 + 361.09e6,      # tc_gemm_kernel<256, 2, 1>, m_ffn = 13108
+    ("cfg3", "attention"): 360.78e6 + 102.51e6,     # tc_attention_pair_kernel, m_attn = 16384
+    ("cfg3", "down"): 1627.55e6 + 99.98e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
 }
 
 
