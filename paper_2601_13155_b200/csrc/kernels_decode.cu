@@ -13,6 +13,8 @@
 //                combine kernel over the slices.
 // The residual vector lives in fp32 scratch and is rounded through the storage type at the same
 // points as the prefill path.
+#include <type_traits>
+
 #include "spts_common.cuh"
 
 namespace spts {
@@ -333,6 +335,205 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
   }
 }
 
+// ---- the same partial attention for bf16 caches, on mma.sync (m16n8k16, fp32 accumulation) ----
+// The CUDA-core kernel above spends ~80 warp instructions per cached row (dot products spread over 16 lanes,
+// shuffles, exponentials repeated in every lane); here a warp takes 16 cached rows per step with 32 MMAs:
+//   S[q, row] = Q K^T   M = up to 16 query heads of the GQA group (rows past the group are zero), N = 8 rows, K = d
+//   O[q, dim] += P V    M = the same queries, N = 8 dims, K = 16 rows
+// Both operands come straight from global memory in 16-byte loads, with no shared-memory staging: a dot product
+// does not care about the order of its terms, so the k index of the first product and the n index of the second
+// are permuted to whatever order the loads deliver.
+//   K:  lane (g, c) = (lane / 4, lane % 4) loads, of row r0 + 8u + g, the 8 elements 32j + 8c .. + 7 (j = 0 .. d/32 - 1);
+//       elements 4h .. 4h + 3 of that chunk are the lane's share of k-step 2j + h, and Q's fragment is built with
+//       the same map.
+//   V:  lane (g, c) loads, of rows r0 + 2c, r0 + 2c + 1, r0 + 8 + 2c, r0 + 9 + 2c, the d/8 elements from g d/8 on;
+//       n-tile v then holds dims {g d/8 + v}, and byte permutes pair the two rows of a k index.
+// S's accumulator fragment is P's A fragment (rows 2c, 2c + 1 of n-tile u = k indices 2c + 8u, 2c + 8u + 1).
+// O is rescaled only in steps where some query's running maximum moved.
+__device__ __forceinline__ void mma_bf16_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1,
+                                               uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1, float c0, float c1,
+                                               float c2, float c3) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+               : "=f"(d0), "=f"(d1), "=f"(d2), "=f"(d3)
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// HI: the block serves more than 8 query heads (fragment rows 8..15 carry heads too).
+template <int D, bool HI>
+__global__ void __launch_bounds__(128, 3)
+dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, const bf16* __restrict__ vc, int len,
+                    int H, int Hkv, int nsplit, float* __restrict__ part) {
+  constexpr int NJ = D / 32;               // 16-byte chunks of a K row per lane
+  constexpr int NT = D / 16;               // k-steps of Q K^T
+  constexpr int NV = D / 8;                // n-tiles of P V = elements of a V row per lane
+  constexpr int VQ = NV / 8;               // 16-byte chunks of a V row per lane
+  constexpr int NQ = HI ? 16 : 8;
+  __shared__ float sm_m[4][NQ], sm_l[4][NQ];
+  __shared__ float sm_o[4][NQ][D];
+  dep_launch();
+  dep_wait();                                        // q and the cache's newest row come from the previous kernel
+  const int G = H / Hkv, qb = (G + 15) / 16;
+  const int kvh = blockIdx.x / qb, qoff = (blockIdx.x % qb) * 16, s = blockIdx.y;
+  const int hb = kvh * G + qoff, nq = min(16, G - qoff);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, c = lane & 3;
+  const int j0 = (int)((long)len * s / nsplit), j1 = (int)((long)len * (s + 1) / nsplit);
+  const float sl = rsqrtf((float)D) * 1.4426950408889634f;
+
+  uint32_t qa[NT][HI ? 4 : 2];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) {
+    const int e = 32 * (t >> 1) + 8 * c + 4 * (t & 1);
+    float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+    if (g < nq) lo = __ldcg(reinterpret_cast<const float4*>(q32 + (size_t)(hb + g) * D + e));
+    qa[t][0] = pack_bf16x2(lo.x, lo.y);
+    qa[t][1] = pack_bf16x2(lo.z, lo.w);
+    if (HI) {
+      if (g + 8 < nq) hi = __ldcg(reinterpret_cast<const float4*>(q32 + (size_t)(hb + g + 8) * D + e));
+      qa[t][2] = pack_bf16x2(hi.x, hi.y);
+      qa[t][3] = pack_bf16x2(hi.z, hi.w);
+    }
+  }
+  float o[NV][HI ? 4 : 2];
+#pragma unroll
+  for (int v = 0; v < NV; ++v)
+#pragma unroll
+    for (int i = 0; i < (HI ? 4 : 2); ++i) o[v][i] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+  const size_t rstride = (size_t)Hkv * D;
+  const bf16* kbase = kc + (size_t)kvh * D + 8 * c;
+  const bf16* vbase = vc + (size_t)kvh * D + g * NV;
+  for (int r0 = j0 + warp * 16; r0 < j1; r0 += 64) {       // the same trip count for every lane of a warp
+    uint4 kq[2][NJ], vq[4][VQ];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const bf16* kp = kbase + (size_t)min(r0 + 8 * u + g, j1 - 1) * rstride;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) kq[u][j] = __ldcg(reinterpret_cast<const uint4*>(kp + 32 * j));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const bf16* vp = vbase + (size_t)min(r0 + 8 * (i >> 1) + 2 * c + (i & 1), j1 - 1) * rstride;
+#pragma unroll
+      for (int x = 0; x < VQ; ++x) vq[i][x] = __ldcg(reinterpret_cast<const uint4*>(vp + 8 * x));
+    }
+    // S = Q K^T for the two 8-row tiles
+    float sc[2][4];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      sc[u][0] = sc[u][1] = sc[u][2] = sc[u][3] = 0.f;
+#pragma unroll
+      for (int t = 0; t < NT; ++t) {
+        const uint4 kk = kq[u][t >> 1];
+        const uint32_t b0 = (t & 1) ? kk.z : kk.x, b1 = (t & 1) ? kk.w : kk.y;
+        mma_bf16_16816(sc[u][0], sc[u][1], sc[u][2], sc[u][3], qa[t][0], HI ? qa[t][2] : 0u, qa[t][1],
+                       HI ? qa[t][3] : 0u, b0, b1, sc[u][0], sc[u][1], sc[u][2], sc[u][3]);
+      }
+      // rows past the slice
+      const int ra = r0 + 8 * u + 2 * c;
+      if (ra >= j1) { sc[u][0] = -INFINITY; sc[u][2] = -INFINITY; }
+      if (ra + 1 >= j1) { sc[u][1] = -INFINITY; sc[u][3] = -INFINITY; }
+    }
+    float x0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+    x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, 1));
+    x0 = fmaxf(x0, __shfl_xor_sync(0xffffffffu, x0, 2));
+    float x1 = -INFINITY;
+    if (HI) {
+      x1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
+      x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, 1));
+      x1 = fmaxf(x1, __shfl_xor_sync(0xffffffffu, x1, 2));
+    }
+    const bool moved = x0 > m0 || (HI && x1 > m1);
+    if (__any_sync(0xffffffffu, moved)) {
+      const float n0 = fmaxf(m0, x0), n1 = fmaxf(m1, x1);
+      const float c0 = exp2f((m0 - n0) * sl), c1 = HI ? exp2f((m1 - n1) * sl) : 0.f;   // first step: exp2(-inf) = 0
+      m0 = n0; l0 *= c0;
+      if (HI) { m1 = n1; l1 *= c1; }
+#pragma unroll
+      for (int v = 0; v < NV; ++v) {
+        o[v][0] *= c0; o[v][1] *= c0;
+        if (HI) { o[v][2] *= c1; o[v][3] *= c1; }
+      }
+    }
+    uint32_t pa[4];
+    {
+      const float b0 = m0 * sl;
+      const float p00 = exp2f(fmaf(sc[0][0], sl, -b0)), p01 = exp2f(fmaf(sc[0][1], sl, -b0));
+      const float p10 = exp2f(fmaf(sc[1][0], sl, -b0)), p11 = exp2f(fmaf(sc[1][1], sl, -b0));
+      l0 += (p00 + p01) + (p10 + p11);
+      pa[0] = pack_bf16x2(p00, p01); pa[2] = pack_bf16x2(p10, p11);
+      pa[1] = 0u; pa[3] = 0u;
+      if (HI) {
+        const float b1 = m1 * sl;
+        const float q00 = exp2f(fmaf(sc[0][2], sl, -b1)), q01 = exp2f(fmaf(sc[0][3], sl, -b1));
+        const float q10 = exp2f(fmaf(sc[1][2], sl, -b1)), q11 = exp2f(fmaf(sc[1][3], sl, -b1));
+        l1 += (q00 + q01) + (q10 + q11);
+        pa[1] = pack_bf16x2(q00, q01); pa[3] = pack_bf16x2(q10, q11);
+      }
+    }
+    // O += P V
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+      const int x = v >> 3, w = (v >> 1) & 3;
+      const uint32_t r00 = (&vq[0][x].x)[w], r01 = (&vq[1][x].x)[w], r10 = (&vq[2][x].x)[w], r11 = (&vq[3][x].x)[w];
+      const uint32_t sel = (v & 1) ? 0x7632u : 0x5410u;
+      const uint32_t b0 = __byte_perm(r00, r01, sel), b1 = __byte_perm(r10, r11, sel);
+      if (HI) {
+        mma_bf16_16816(o[v][0], o[v][1], o[v][2], o[v][3], pa[0], pa[1], pa[2], pa[3], b0, b1, o[v][0], o[v][1],
+                       o[v][2], o[v][3]);
+      } else {
+        float d2, d3;
+        mma_bf16_16816(o[v][0], o[v][1], d2, d3, pa[0], 0u, pa[2], 0u, b0, b1, o[v][0], o[v][1], 0.f, 0.f);
+      }
+    }
+  }
+  // the four lanes of a query hold partial sums of l
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  if (HI) {
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  }
+  if (c == 0) {
+    sm_m[warp][g] = m0; sm_l[warp][g] = l0;
+    if (HI) { sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1; }
+  }
+#pragma unroll
+  for (int v = 0; v < NV; ++v) {
+    // accumulator columns 2c, 2c + 1 of n-tile v are dims (2c) NV + v and (2c + 1) NV + v
+    sm_o[warp][g][(2 * c) * NV + v] = o[v][0];
+    sm_o[warp][g][(2 * c + 1) * NV + v] = o[v][1];
+    if (HI) {
+      sm_o[warp][g + 8][(2 * c) * NV + v] = o[v][2];
+      sm_o[warp][g + 8][(2 * c + 1) * NV + v] = o[v][3];
+    }
+  }
+  __syncthreads();
+  const float scale = rsqrtf((float)D);
+  for (int t = threadIdx.x; t < nq * D; t += 128) {
+    const int q = t / D, dim = t - q * D;
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) M = fmaxf(M, sm_m[w][q]);
+    float L = 0.f, acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const float f = sm_m[w][q] == -INFINITY ? 0.f : exp2f((sm_m[w][q] - M) * sl);
+      L += sm_l[w][q] * f;
+      acc = fmaf(sm_o[w][q][dim], f, acc);
+    }
+    float* pp = part + ((size_t)(hb + q) * nsplit + s) * (D + 2);
+    if (dim == 0) { pp[0] = M * scale; pp[1] = L; }
+    pp[2 + dim] = acc;
+  }
+}
+
 constexpr int DEC_MAX_SPLIT = 64;
 
 // Combines the slices of one query head: thread s < nsplit first takes slice s's (max, sum) so that the global
@@ -398,6 +599,14 @@ spts_status launch_attn_partial(spts_ctx* ctx, const float* q32, const spts_kv_l
   cudaStream_t st = ctx->stream;
   const T* kc = (const T*)cache->k;
   const T* vc = (const T*)cache->v;
+  if constexpr (std::is_same<T, bf16>::value) {
+    const dim3 grid(Hkv * ceil_div(group, 16), nsplit);
+    if (group > 8)
+      LAUNCH_DEP(ctx, dec_attn_mma_kernel<D, true>, grid, dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
+    else
+      LAUNCH_DEP(ctx, dec_attn_mma_kernel<D, false>, grid, dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
+    return SPTS_OK;
+  }
   // all query heads of a GQA group in one block when the group size is 2, 4 or 8; else one head per block
   if (group % 8 == 0)
     LAUNCH_DEP(ctx, dec_attn_partial_kernel<T, D, 8>, dim3(H / 8, nsplit), dim3(128), st, q32, kc, vc, len, H, Hkv, nsplit, part);
@@ -430,7 +639,9 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
              (T*)cache->k, (T*)cache->v, cache->pos, slot);
   cache->len = slot + 1;
   const int len = cache->len;
-  const int nsplit = min(DEC_MAX_SPLIT, max(1, len / 128));
+  int nsplit = min(DEC_MAX_SPLIT, max(1, len / 128));
+  if (std::is_same<T, bf16>::value)      // the tensor-core kernel holds three blocks per SM: keep the slices to one wave
+    nsplit = max(1, min(nsplit, 3 * ctx->sm_count / (Hkv * ceil_div(H / Hkv, 16))));
   if (hd == 128) TRY_DEC(launch_attn_partial<T, 128>(ctx, q32, cache, len, nsplit, part));
   else TRY_DEC(launch_attn_partial<T, 64>(ctx, q32, cache, len, nsplit, part));
   LAUNCH_DEP(ctx, dec_attn_combine_kernel<T>, dim3(H), dim3(hd), st, (const float*)part, nsplit, hd, att32);

@@ -307,3 +307,52 @@ def test_decode_steps_are_reproducible_bit_for_bit():
         assert ta == tb and torch.equal(a, b)
     assert lib.device_status() == 0
     lib.close()
+
+
+DECODE_HEAD_LAYOUTS = {
+    # name: (query heads, KV heads, head dim) -- the GQA group decides how the query heads fill the 16 fragment rows
+    "group4_d128": (8, 2, 128),        # the 8B layout: rows 0..3 of one block
+    "group7_d128": (7, 1, 128),        # an odd group (the Qwen layout)
+    "group12_d128": (12, 1, 128),      # both halves of the fragment carry heads
+    "group20_d64": (20, 1, 64),        # two blocks per KV head (16 + 4 query heads), head dim 64
+    "group1_d64": (4, 4, 64),          # no grouping
+}
+
+
+@pytest.mark.parametrize("layout", sorted(DECODE_HEAD_LAYOUTS))
+@pytest.mark.parametrize("n0", [5, 2077])
+def test_decode_attention_over_long_caches(layout, n0):
+    """Decode against synthetic caches long enough for many slices per head (2077 rows: 16 ragged slices, each
+    shared by four warps in 16-row groups with a masked tail) and against a 5-row cache, for head layouts that fill
+    the tensor-core fragments differently.  Two steps, so the second reads the row the first appended."""
+    from paper_2601_13155_b200 import binding
+    H, Hkv, hd = DECODE_HEAD_LAYOUTS[layout]
+    shape = replace(synth.LLAMA8B, hidden=256, n_q_heads=H, n_kv_heads=Hkv, head_dim=hd, ffn_dim=512,
+                    ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1000)
+    lib = _mk(shape, 1024, hd != 128)           # the prefill tensor-core kernels want head dim 128; decode has no such limit
+    # a large W_o and no FFN update (W_down = 0): the step's output is dominated by the attention result
+    W = zero_down(synth.layer_weights(shape, 1030, 0, std=0.05))
+    W["wo"] = synth.quantize(W["wo"] * np.float32(8.0), "bf16")
+    hw = synth.head_weights(shape, 1030)
+    model = binding.Model([binding.LayerWeights(W, "bf16")], up(hw["lm_head"], "bf16"), up(hw["embed"], "bf16"))
+    rng = np.random.default_rng(n0)
+    k0 = up((3.0 * rng.standard_normal((n0, Hkv, hd))).astype(np.float32), "bf16")
+    v0 = up(rng.standard_normal((n0, Hkv, hd)).astype(np.float32), "bf16")
+    cache = binding.KvCache(shape, 1, n0 + 2)
+    cache.k[0][:n0].copy_(k0)
+    cache.v[0][:n0].copy_(v0)
+    cache.pos[0][:n0].copy_(i32(np.arange(n0)))
+    cache.c[0].len = n0
+    oc = [{"K": host(k0), "V": host(v0), "pos": np.arange(n0)}]
+    tok = torch.zeros(1, dtype=torch.int32, device=dev())
+    for step, token in enumerate((3, 998)):
+        xo = torch.empty(shape.hidden, dtype=lib.dtype, device=dev())
+        lg = torch.empty(shape.vocab, dtype=torch.float32, device=dev())
+        lib.decode_step(model, cache, n0 + step, token_in=token, x_out=xo, logits_out=lg, token_out=tok)
+        x, lgo, _ = O.decode_step(hw["embed"][token], n0 + step, [W], shape, oc, np.ones(shape.hidden), hw["lm_head"],
+                                  mode="bf16")
+        check_output(host(xo), x, "bf16", scale=2)
+        assert rel_rms_err(host(lg), lgo) <= 2 * TOL["bf16"]
+        check_output(host(cache.k[0][n0 + step]), oc[0]["K"][n0 + step], "bf16")
+    assert cache.length(0) == n0 + 2 and lib.device_status() == 0
+    lib.close()
