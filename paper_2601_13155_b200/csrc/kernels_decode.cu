@@ -220,19 +220,24 @@ dec_qkv_kernel(const T* __restrict__ wq, const T* __restrict__ wk, const T* __re
 #pragma unroll
     for (int r = 0; r < 8; ++r) rowp[r] = wv + (size_t)min(v0 + r, Hkv * d - 1) * K;
   }
+  // the rotary factors depend on the position only: the (slow) double-precision evaluation runs while the
+  // previous kernel is still finishing, ahead of the dependency wait inside gemv_rows
+  const int t = threadIdx.x;
+  float cf = 1.f, sf = 0.f;
+  if (kind != 2 && t < 4) {
+    const double inv = exp2(-(double)(2 * (i0 + t)) / (double)d * log2(theta));
+    double sn, cs;
+    sincos((double)pos * inv, &sn, &cs);
+    cf = (float)cs; sf = (float)sn;
+  }
   gemv_rows<T, 8>(rowp, K, x, dots, &ss);
   const float rs = 1.0f / sqrtf(ss / (float)K + eps);
-  const int t = threadIdx.x;
   if (kind == 2) {
     if (t < 8 && v0 + t < Hkv * d) vc[(size_t)slot * Hkv * d + v0 + t] = from_f32<T>(dots[t] * rs);
     return;
   }
   if (t < 4) {
     const int i = i0 + t;
-    const double inv = exp2(-(double)(2 * i) / (double)d * log2(theta));
-    double sn, cs;
-    sincos((double)pos * inv, &sn, &cs);
-    const float cf = (float)cs, sf = (float)sn;
     const float a = dots[t] * rs, bb2 = dots[4 + t] * rs;
     const float r1 = a * cf - bb2 * sf, r2 = bb2 * cf + a * sf;
     if (kind == 0) {
@@ -346,8 +351,9 @@ dec_attn_partial_kernel(const float* __restrict__ q32, const T* __restrict__ kc,
 //   K:  lane (g, c) = (lane / 4, lane % 4) loads, of row r0 + 8u + g, the 8 elements 32j + 8c .. + 7 (j = 0 .. d/32 - 1);
 //       elements 4h .. 4h + 3 of that chunk are the lane's share of k-step 2j + h, and Q's fragment is built with
 //       the same map.
-//   V:  lane (g, c) loads, of rows r0 + 2c, r0 + 2c + 1, r0 + 8 + 2c, r0 + 9 + 2c, the d/8 elements from g d/8 on;
-//       n-tile v then holds dims {g d/8 + v}, and byte permutes pair the two rows of a k index.
+//   V:  lane (g, c) loads, of rows r0 + 2c, r0 + 2c + 1, r0 + 8 + 2c, r0 + 9 + 2c, the 8 elements 64x + 8g .. + 7
+//       (x = 0 .. d/64 - 1; the eight lanes of a row read 128 contiguous bytes per load); n-tile v = 8x + e then
+//       holds dims {64x + 8g + e}, and byte permutes pair the two rows of a k index.
 // S's accumulator fragment is P's A fragment (rows 2c, 2c + 1 of n-tile u = k indices 2c + 8u, 2c + 8u + 1).
 // O is rescaled only in steps where some query's running maximum moved.
 __device__ __forceinline__ void mma_bf16_16816(float& d0, float& d1, float& d2, float& d3, uint32_t a0, uint32_t a1,
@@ -374,9 +380,11 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
   constexpr int VQ = NV / 8;               // 16-byte chunks of a V row per lane
   constexpr int NQ = HI ? 16 : 8;
   __shared__ float sm_m[4][NQ], sm_l[4][NQ];
-  __shared__ float sm_o[4][NQ][D];
+  // a lane's accumulators are, per x, the 16 dims 64x + 16c .. + 15: stored as [query][c][x][16] with four floats of
+  // padding per (query, c), the 16-byte stores of a quarter warp fall into distinct banks
+  constexpr int OC = 16 * VQ + 4;
+  __shared__ __align__(16) float sm_o[4][NQ][4][OC];
   dep_launch();
-  dep_wait();                                        // q and the cache's newest row come from the previous kernel
   const int G = H / Hkv, qb = (G + 15) / 16;
   const int kvh = blockIdx.x / qb, qoff = (blockIdx.x % qb) * 16, s = blockIdx.y;
   const int hb = kvh * G + qoff, nq = min(16, G - qoff);
@@ -385,6 +393,47 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
   const int j0 = (int)((long)len * s / nsplit), j1 = (int)((long)len * (s + 1) / nsplit);
   const float sl = rsqrtf((float)D) * 1.4426950408889634f;
 
+  float o[NV][HI ? 4 : 2];
+#pragma unroll
+  for (int v = 0; v < NV; ++v)
+#pragma unroll
+    for (int i = 0; i < (HI ? 4 : 2); ++i) o[v][i] = 0.f;
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+  const size_t rstride = (size_t)Hkv * D;
+  const bf16* kbase = kc + (size_t)kvh * D + 8 * c;
+  const bf16* vbase = vc + (size_t)kvh * D + g * 8;
+  // Only q and the cache's newest row (index len - 1) come from the previous kernel.  Ahead of the dependency
+  // wait the warp loads its first 16 rows into registers -- unless they reach the newest row -- and pulls its
+  // later rows towards L2, so that the cache streams in while the projection kernel is still running.
+  uint4 kq[2][NJ], vq[4][VQ];
+  auto load_rows = [&](int r0) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const bf16* kp = kbase + (size_t)min(r0 + 8 * u + g, j1 - 1) * rstride;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) kq[u][j] = __ldcg(reinterpret_cast<const uint4*>(kp + 32 * j));
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const bf16* vp = vbase + (size_t)min(r0 + 8 * (i >> 1) + 2 * c + (i & 1), j1 - 1) * rstride;
+#pragma unroll
+      for (int x = 0; x < VQ; ++x) vq[i][x] = __ldcg(reinterpret_cast<const uint4*>(vp + 64 * x));
+    }
+  };
+  const int r_first = j0 + warp * 16;
+  bool loaded = false;
+  if (r_first < j1 && r_first + 16 <= len - 1) { load_rows(r_first); loaded = true; }
+  for (int r0 = r_first + (loaded ? 64 : 0); r0 < j1; r0 += 64) {
+    // 16 rows x (D * 2) bytes of K and of V = 128-byte lines, spread over the lanes
+    for (int ln = lane; ln < 16 * (D * 2 / 128); ln += 32) {
+      const int row = min(r0 + ln / (D * 2 / 128), j1 - 1);
+      const size_t off = ((size_t)row * Hkv + kvh) * D + (ln % (D * 2 / 128)) * 64;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(kc + off));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(vc + off));
+    }
+  }
+  dep_wait();
   uint32_t qa[NT][HI ? 4 : 2];
 #pragma unroll
   for (int t = 0; t < NT; ++t) {
@@ -399,30 +448,9 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
       qa[t][3] = pack_bf16x2(hi.z, hi.w);
     }
   }
-  float o[NV][HI ? 4 : 2];
-#pragma unroll
-  for (int v = 0; v < NV; ++v)
-#pragma unroll
-    for (int i = 0; i < (HI ? 4 : 2); ++i) o[v][i] = 0.f;
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-
-  const size_t rstride = (size_t)Hkv * D;
-  const bf16* kbase = kc + (size_t)kvh * D + 8 * c;
-  const bf16* vbase = vc + (size_t)kvh * D + g * NV;
-  for (int r0 = j0 + warp * 16; r0 < j1; r0 += 64) {       // the same trip count for every lane of a warp
-    uint4 kq[2][NJ], vq[4][VQ];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const bf16* kp = kbase + (size_t)min(r0 + 8 * u + g, j1 - 1) * rstride;
-#pragma unroll
-      for (int j = 0; j < NJ; ++j) kq[u][j] = __ldcg(reinterpret_cast<const uint4*>(kp + 32 * j));
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const bf16* vp = vbase + (size_t)min(r0 + 8 * (i >> 1) + 2 * c + (i & 1), j1 - 1) * rstride;
-#pragma unroll
-      for (int x = 0; x < VQ; ++x) vq[i][x] = __ldcg(reinterpret_cast<const uint4*>(vp + 8 * x));
-    }
+  for (int r0 = r_first; r0 < j1; r0 += 64) {       // the same trip count for every lane of a warp
+    if (!loaded) load_rows(r0);
+    loaded = false;
     // S = Q K^T for the two 8-row tiles
     float sc[2][4];
 #pragma unroll
@@ -504,16 +532,20 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
     sm_m[warp][g] = m0; sm_l[warp][g] = l0;
     if (HI) { sm_m[warp][g + 8] = m1; sm_l[warp][g + 8] = l1; }
   }
+  // accumulator columns 2c, 2c + 1 of n-tile 8x + e are dims 64x + 16c + e and 64x + 16c + 8 + e
 #pragma unroll
-  for (int v = 0; v < NV; ++v) {
-    // accumulator columns 2c, 2c + 1 of n-tile v are dims (2c) NV + v and (2c + 1) NV + v
-    sm_o[warp][g][(2 * c) * NV + v] = o[v][0];
-    sm_o[warp][g][(2 * c + 1) * NV + v] = o[v][1];
-    if (HI) {
-      sm_o[warp][g + 8][(2 * c) * NV + v] = o[v][2];
-      sm_o[warp][g + 8][(2 * c + 1) * NV + v] = o[v][3];
-    }
-  }
+  for (int x = 0; x < VQ; ++x)
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int e4 = 0; e4 < 2; ++e4) {
+        const int v = 8 * x + 4 * e4;
+        *reinterpret_cast<float4*>(&sm_o[warp][g][c][16 * x + 8 * i + 4 * e4]) =
+            make_float4(o[v][i], o[v + 1][i], o[v + 2][i], o[v + 3][i]);
+        if (HI)
+          *reinterpret_cast<float4*>(&sm_o[warp][g + 8][c][16 * x + 8 * i + 4 * e4]) =
+              make_float4(o[v][2 + i], o[v + 1][2 + i], o[v + 2][2 + i], o[v + 3][2 + i]);
+      }
   __syncthreads();
   const float scale = rsqrtf((float)D);
   for (int t = threadIdx.x; t < nq * D; t += 128) {
@@ -526,7 +558,7 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
     for (int w = 0; w < 4; ++w) {
       const float f = sm_m[w][q] == -INFINITY ? 0.f : exp2f((sm_m[w][q] - M) * sl);
       L += sm_l[w][q] * f;
-      acc = fmaf(sm_o[w][q][dim], f, acc);
+      acc = fmaf(sm_o[w][q][(dim >> 4) & 3][16 * (dim >> 6) + (dim & 15)], f, acc);
     }
     float* pp = part + ((size_t)(hb + q) * nsplit + s) * (D + 2);
     if (dim == 0) { pp[0] = M * scale; pp[1] = L; }
@@ -536,52 +568,58 @@ dec_attn_mma_kernel(const float* __restrict__ q32, const bf16* __restrict__ kc, 
 
 constexpr int DEC_MAX_SPLIT = 64;
 
-// Combines the slices of one query head: thread s < nsplit first takes slice s's (max, sum) so that the global
-// maximum and the weights exp(max_s - M) come from one parallel step; then thread t sums dimension t over the
-// slices with the loads of eight slices in flight.  blockDim = d >= nsplit.
+// Combines the slices of one query head.  Thread s < nsplit takes slice s's (max, sum), so the global maximum and
+// the weights exp(max_s - M) come from one parallel step; then the block's 512 / d thread groups each sum one
+// dimension per thread over every (512 / d)-th slice, all of a group's loads in flight together, and the groups
+// meet in shared memory.  d divides 512, nsplit <= 64.
 template <typename T>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(512)
 dec_attn_combine_kernel(const float* __restrict__ part, int nsplit, int d, float* __restrict__ att32) {
   __shared__ float f[DEC_MAX_SPLIT];
   __shared__ float red[4];
-  __shared__ float Msh, Lsh;
+  __shared__ float accs[512];
   dep_launch();
   dep_wait();
-  const int h = blockIdx.x, t = threadIdx.x, nw = blockDim.x >> 5;
+  const int h = blockIdx.x, t = threadIdx.x;
   const float* ph = part + (size_t)h * nsplit * (d + 2);
-  const float m = t < nsplit ? __ldcg(&ph[(size_t)t * (d + 2)]) : -INFINITY;
+  float m = -INFINITY, l = 0.f;
+  if (t < nsplit) {
+    m = __ldcg(&ph[(size_t)t * (d + 2)]);
+    l = __ldcg(&ph[(size_t)t * (d + 2) + 1]);
+  }
   float v = warp_max(m);
-  if ((t & 31) == 0) red[t >> 5] = v;
+  if (t < 64 && (t & 31) == 0) red[t >> 5] = v;
   __syncthreads();
-  if (t == 0) {
-    float M = red[0];
-    for (int w = 1; w < nw; ++w) M = fmaxf(M, red[w]);
-    Msh = M;
-  }
-  __syncthreads();
-  const float fs = m == -INFINITY ? 0.f : expf(m - Msh);
+  const float M = fmaxf(red[0], red[1]);
+  const float fs = m == -INFINITY ? 0.f : expf(m - M);
   if (t < nsplit) f[t] = fs;
-  v = warp_sum(t < nsplit ? __ldcg(&ph[(size_t)t * (d + 2) + 1]) * fs : 0.f);
-  __syncthreads();                       // red[] has been read by thread 0
-  if ((t & 31) == 0) red[t >> 5] = v;
+  v = warp_sum(l * fs);
+  if (t < 64 && (t & 31) == 0) red[2 + (t >> 5)] = v;
   __syncthreads();
-  if (t == 0) {
-    float L = 0.f;
-    for (int w = 0; w < nw; ++w) L += red[w];
-    Lsh = L;
-  }
-  __syncthreads();
+  const float L = red[2] + red[3];
+  const int ngrp = 512 / d, grp = t / d, dim = t - grp * d;
+  constexpr int U = 16;
   float acc = 0.f;
-  int s0 = 0;
-  for (; s0 + 8 <= nsplit; s0 += 8) {
-    float x[8];
+  for (int s0 = grp; s0 < nsplit; s0 += ngrp * U) {
+    float x[U];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = __ldcg(&ph[(size_t)(s0 + u) * (d + 2) + 2 + t]);
+    for (int u = 0; u < U; ++u) {
+      const int s = s0 + u * ngrp;
+      x[u] = s < nsplit ? __ldcg(&ph[(size_t)s * (d + 2) + 2 + dim]) : 0.f;
+    }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) acc = fmaf(x[u], f[s0 + u], acc);
+    for (int u = 0; u < U; ++u) {
+      const int s = s0 + u * ngrp;
+      if (s < nsplit) acc = fmaf(x[u], f[s], acc);
+    }
   }
-  for (; s0 < nsplit; ++s0) acc = fmaf(__ldcg(&ph[(size_t)s0 * (d + 2) + 2 + t]), f[s0], acc);
-  att32[h * d + t] = round_through<T>(acc / Lsh);
+  accs[t] = acc;
+  __syncthreads();
+  if (t < d) {
+    float a = 0.f;
+    for (int gq = 0; gq < ngrp; ++gq) a += accs[gq * d + t];
+    att32[h * d + t] = round_through<T>(a / L);
+  }
 }
 
 #define LAUNCH_DEP(ctx, ...)                                                      \
@@ -644,7 +682,7 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
     nsplit = max(1, min(nsplit, 3 * ctx->sm_count / (Hkv * ceil_div(H / Hkv, 16))));
   if (hd == 128) TRY_DEC(launch_attn_partial<T, 128>(ctx, q32, cache, len, nsplit, part));
   else TRY_DEC(launch_attn_partial<T, 64>(ctx, q32, cache, len, nsplit, part));
-  LAUNCH_DEP(ctx, dec_attn_combine_kernel<T>, dim3(H), dim3(hd), st, (const float*)part, nsplit, hd, att32);
+  LAUNCH_DEP(ctx, dec_attn_combine_kernel<T>, dim3(H), dim3(512), st, (const float*)part, nsplit, hd, att32);
   LAUNCH_DEP(ctx, gemv_resid_kernel<T>, dim3(ceil_div(D, 8)), dim3(GV_THREADS), st, (const T*)w->wo, D, H * hd,
              (const float*)att32, x32);
   LAUNCH_DEP(ctx, gemv_swiglu_kernel<T>, dim3(ceil_div(Dff, 4)), dim3(GV_THREADS), st, (const T*)w->w_gate,
