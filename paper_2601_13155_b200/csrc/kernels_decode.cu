@@ -696,7 +696,12 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
 
 size_t decode_scratch_floats(const spts_model_desc& d) {
   return (size_t)d.hidden + 2 * (size_t)d.n_q_heads * d.head_dim + (size_t)d.ffn_dim +
-         (size_t)d.n_q_heads * DEC_MAX_SPLIT * (d.head_dim + 2) + 64;
+         (size_t)d.n_q_heads * DEC_MAX_SPLIT * (d.head_dim + 2) + 64 + 2 * ARGMAX_BLOCKS;
+}
+
+// [ARGMAX_BLOCKS] values, then [ARGMAX_BLOCKS] indices: the tail of the decode scratch
+float* argmax_scratch(spts_ctx* ctx) {
+  return (float*)ctx->ws.dec + decode_scratch_floats(ctx->desc) - 2 * ARGMAX_BLOCKS;
 }
 
 spts_status launch_decode_load(spts_ctx* ctx, const void* x) {

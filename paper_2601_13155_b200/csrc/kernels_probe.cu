@@ -194,35 +194,55 @@ __global__ void pad_proxy_kernel(const T* __restrict__ vg, const T* __restrict__
   out[total + t] = c < r ? zero : vu[row * r + (c - r)];
 }
 
-// argmax with the lowest index on ties (single block)
-__global__ void __launch_bounds__(1024)
-argmax_kernel(const float* __restrict__ logits, int n, int32_t* __restrict__ out) {
-  __shared__ float bv[32];
-  __shared__ int bi[32];
-  int tid = threadIdx.x;
-  float best = -INFINITY;
-  int besti = 0x7FFFFFFF;
-  for (int i = tid; i < n; i += blockDim.x) {
-    float v = logits[i];
-    if (v > best || (v == best && i < besti)) { best = v; besti = i; }
-  }
-  for (int o = 16; o > 0; o >>= 1) {
-    float ov = __shfl_xor_sync(0xffffffffu, best, o);
-    int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-    if (ov > best || (ov == best && oi < besti)) { best = ov; besti = oi; }
-  }
+// argmax with the lowest index on ties (NaN never wins; 0 if nothing does), in two steps: every block reduces one
+// contiguous share of the logits to (value, index), then one block reduces the shares.
+__device__ __forceinline__ void argmax_take(float& best, int& besti, float v, int i) {
+  if (v > best || (v == best && i < besti)) { best = v; besti = i; }
+}
+
+__device__ __forceinline__ void argmax_block(float& best, int& besti, float* bv, int* bi) {
+  const int tid = threadIdx.x;
+  for (int o = 16; o > 0; o >>= 1)
+    argmax_take(best, besti, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, besti, o));
   if ((tid & 31) == 0) { bv[tid >> 5] = best; bi[tid >> 5] = besti; }
   __syncthreads();
   if (tid < 32) {
     best = tid < (blockDim.x >> 5) ? bv[tid] : -INFINITY;
     besti = tid < (blockDim.x >> 5) ? bi[tid] : 0x7FFFFFFF;
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, best, o);
-      int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-      if (ov > best || (ov == best && oi < besti)) { best = ov; besti = oi; }
-    }
-    if (tid == 0) *out = besti == 0x7FFFFFFF ? 0 : besti;
+    for (int o = 16; o > 0; o >>= 1)
+      argmax_take(best, besti, __shfl_xor_sync(0xffffffffu, best, o), __shfl_xor_sync(0xffffffffu, besti, o));
   }
+}
+
+__global__ void __launch_bounds__(256)
+argmax_partial_kernel(const float* __restrict__ logits, int n, float* __restrict__ pv, int* __restrict__ pi) {
+  __shared__ float bv[32];
+  __shared__ int bi[32];
+  const int per = (n + gridDim.x - 1) / gridDim.x;
+  const int i0 = blockIdx.x * per, i1 = min(n, i0 + per);
+  float best = -INFINITY;
+  int besti = 0x7FFFFFFF;
+  for (int i = i0 + threadIdx.x; i < i1; i += 4 * 256) {        // four loads in flight per thread
+    float v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = i + u * 256 < i1 ? logits[i + u * 256] : -INFINITY;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (i + u * 256 < i1) argmax_take(best, besti, v[u], i + u * 256);
+  }
+  argmax_block(best, besti, bv, bi);
+  if (threadIdx.x == 0) { pv[blockIdx.x] = best; pi[blockIdx.x] = besti; }
+}
+
+__global__ void __launch_bounds__(ARGMAX_BLOCKS)
+argmax_final_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int32_t* __restrict__ out) {
+  __shared__ float bv[32];
+  __shared__ int bi[32];
+  float best = pv[threadIdx.x];
+  int besti = pi[threadIdx.x];
+  if (!(best == best)) { best = -INFINITY; besti = 0x7FFFFFFF; }
+  argmax_block(best, besti, bv, bi);
+  if (threadIdx.x == 0) *out = besti == 0x7FFFFFFF ? 0 : besti;
 }
 
 }  // namespace
@@ -346,7 +366,11 @@ spts_status launch_head(spts_ctx* ctx, const void* x_row, const void* lm_head, f
   s = launch_head_logits(ctx, (const float*)ctx->ws.dec, lm_head, logits);
   if (s != SPTS_OK) return s;
   if (token_out != nullptr) {
-    argmax_kernel<<<1, 1024, 0, ctx->stream>>>(logits, ctx->desc.vocab, token_out);
+    float* pv = argmax_scratch(ctx);
+    int* pi = (int*)(pv + ARGMAX_BLOCKS);
+    argmax_partial_kernel<<<ARGMAX_BLOCKS, 256, 0, ctx->stream>>>(logits, ctx->desc.vocab, pv, pi);
+    SPTS_CUDA_OK(ctx);
+    argmax_final_kernel<<<1, ARGMAX_BLOCKS, 0, ctx->stream>>>(pv, pi, token_out);
     SPTS_CUDA_OK(ctx);
   }
   return SPTS_OK;

@@ -166,7 +166,9 @@ spts_status launch_ref_attention(spts_ctx* ctx, const void* Q, const void* K, co
                                  void* O);
 
 // ---- kernels_decode.cu
+constexpr int ARGMAX_BLOCKS = 128;     // partial results of the two-step argmax over the logits
 size_t decode_scratch_floats(const spts_model_desc& d);
+float* argmax_scratch(spts_ctx* ctx);
 spts_status launch_decode_load(spts_ctx* ctx, const void* x);     // x [D] -> fp32 residual scratch
 spts_status launch_decode_store(spts_ctx* ctx, void* x);          // fp32 residual scratch -> x [D]
 spts_status launch_decode_layer(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_layer* cache,
