@@ -14,7 +14,7 @@ import torch
 
 from oracle import spts_oracle as O
 from paper_2601_13155_b200 import synth
-from parity_utils import check_index_set, check_output, dev, host
+from parity_utils import TOL, check_index_set, check_output, dev, host, rel_rms_err
 
 pytestmark = pytest.mark.gpu
 
@@ -180,4 +180,58 @@ def test_proxy_build_at_the_8b_layer_shape():
     assert np.linalg.norm(prod_g - want["ug"].T @ want["vg"].T) <= 1e-2 * np.linalg.norm(W["w_gate"][C])
     prod_d = host(got["ud"]) @ host(got["vd"])
     assert np.linalg.norm(prod_d - want["ud"] @ want["vd"]) <= 1e-2 * np.linalg.norm(W["w_down"][:, C])
+    lib.close()
+
+
+def test_decode_steps_at_the_8b_shape():
+    """Two decode steps of a two-layer LLaMA-3.1-8B-shaped model (full vocabulary) against caches of 16384 and 12288
+    rows -- the launch shapes the generation benchmark times: hidden state and logits against the oracle, the
+    appended cache rows, and the token against the argmax of the library's own logits."""
+    from paper_2601_13155_b200 import binding
+    L = 2
+    shape = replace(synth.LLAMA8B, n_layers=L)
+    layers, hostW = [], []
+    for l in range(L):
+        t = synth.device_layer_weights(shape, 1005, l, dev())
+        lw = binding.LayerWeights.__new__(binding.LayerWeights)
+        lw.t = t
+        lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+        layers.append(lw)
+        hostW.append(_host_weights(t))
+    hw = synth.device_head_weights(shape, 1005, dev())
+    model = binding.Model(layers, hw["lm_head"], hw["embed"])
+    lm_host = hw["lm_head"].float().cpu().numpy()
+    emb_host = hw["embed"].float().cpu().numpy()
+    lens = (16384, 12288)
+    cache = binding.KvCache(shape, L, [n + 2 for n in lens])
+    g = torch.Generator(device=dev())
+    g.manual_seed(77)
+    oc = []
+    for l, n in enumerate(lens):
+        k = (2.0 * torch.randn((n, shape.n_kv_heads, shape.head_dim), generator=g, device=dev())).to(torch.bfloat16)
+        v = torch.randn((n, shape.n_kv_heads, shape.head_dim), generator=g, device=dev()).to(torch.bfloat16)
+        cache.k[l][:n].copy_(k)
+        cache.v[l][:n].copy_(v)
+        cache.pos[l][:n].copy_(torch.arange(n, dtype=torch.int32, device=dev()))
+        cache.c[l].len = n
+        oc.append({"K": host(k), "V": host(v), "pos": np.arange(n)})
+    lib = binding.Spts(shape, max_seq=1024)
+    tok = torch.zeros(1, dtype=torch.int32, device=dev())
+    for step, token in enumerate((11, 90001)):
+        xo = torch.empty(shape.hidden, dtype=torch.bfloat16, device=dev())
+        lg = torch.empty(shape.vocab, dtype=torch.float32, device=dev())
+        lib.decode_step(model, cache, 40000 + step, token_in=token, x_out=xo, logits_out=lg, token_out=tok)
+        assert lib.device_status() == 0
+        x, lgo, _ = O.decode_step(emb_host[token], 40000 + step, hostW, shape, oc, np.ones(shape.hidden), lm_host,
+                                  mode="bf16")
+        check_output(host(xo), x, "bf16", scale=3)         # the same bounds as the small decode cases
+        lgh = host(lg)
+        assert rel_rms_err(lgh, lgo) <= 3 * TOL["bf16"]
+        assert int(tok.item()) == int(np.argmax(lgh))
+        for l, n in enumerate(lens):
+            assert cache.length(l) == n + step + 1
+            # one 1024-element row: a single rounding flip of an entry in [4, 8) is 2^-5, above 2e-2 of the row's
+            # RMS (~1.3), and the helper's allowance of such flips is a fraction of the element count
+            check_output(host(cache.k[l][n + step]), oc[l]["K"][n + step], "bf16", scale=2)
+            check_output(host(cache.v[l][n + step]), oc[l]["V"][n + step], "bf16", scale=2)
     lib.close()
