@@ -87,10 +87,22 @@ __device__ __forceinline__ void gemv_rows(const T* (&rowp)[R], int K, const floa
   float ss = 0.f;
   const int c0 = (warp * 32 + lane) * V;
   dep_launch();
-  // the weights do not depend on the previous kernel: pull this thread's chunks towards L2 while it finishes
-  for (int c = c0; c < K; c += GV_THREADS * V) {
+  // The weights do not depend on the previous kernel: the block's rows are pulled towards L2 while it finishes,
+  // one bulk prefetch per 8 KiB piece of a row (far fewer requests than a prefetch per 16-byte chunk, and measured
+  // twice as effective on the step time).  Rows are 16-byte multiples (K is a multiple of 8 elements).
+  {
+    constexpr int PIECE = 8192;
+    const int row_bytes = K * (int)sizeof(T);
+    const int npiece = (row_bytes + PIECE - 1) / PIECE;
+    for (int u = threadIdx.x; u < R * npiece; u += GV_THREADS) {
+      const int r = u / npiece, pc = u - r * npiece;
+      const int bytes = min(PIECE, row_bytes - pc * PIECE) & ~15;
+      const char* src = nullptr;
 #pragma unroll
-    for (int r = 0; r < R; ++r) asm volatile("prefetch.global.L2 [%0];" ::"l"(rowp[r] + c));
+      for (int rr = 0; rr < R; ++rr)
+        if (rr == r) src = reinterpret_cast<const char*>(rowp[rr]) + (size_t)pc * PIECE;
+      if (bytes > 0) asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+    }
   }
   dep_wait();                                                    // x does depend on it
   for (int c = c0; c < K; c += GV_THREADS * V) {
