@@ -65,8 +65,11 @@ enum {
   SPTS_PAP_WINDOW = 8u,        /* spts_set_option: value = number of trailing queries the probe score averages over
                                   (1..64; 1 = last token only, Eq. 4; larger windows are the query-length ablation of
                                   Appendix C: every query attends causally, K and the queries are taken as stored) */
-  SPTS_ATTENTION_ONE_TILE = 4u /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
+  SPTS_ATTENTION_ONE_TILE = 4u, /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
                                   slower kernel kept as a cross-check of the two-tile kernel) */
+  SPTS_FFN_SCORE_PAP_ONLY = 16u /* spts_set_option: T_f = TopK(S_mha, m_ffn) -- the FFN block selects by the attention
+                                  probe's score alone (Eq. 4) and the proxy FFN of Eq. 12-14 is not evaluated: the
+                                  criterion the paper's proxy-network ablation (Table 4) compares Eq. 14 against */
 };
 
 typedef struct {

@@ -224,10 +224,13 @@ def _w64(W):
 
 
 def layer_prefill_skip(X, pos, W, shape, m_attn, m_ffn, g_attn=None, g_ffn=None,
-                       mode="exact", force_last=True):
+                       mode="exact", force_last=True, ffn_criterion="ltp"):
     """One decoder layer with token skipping.  m_attn == N / m_ffn == N is the
     dense block (TopK of everything).  Returns a dict with the updated X, the
-    scores, both index sets and the layer's KV cache entries."""
+    scores, both index sets and the layer's KV cache entries.
+
+    ffn_criterion: "ltp" selects the FFN's tokens by Eq. 14 (proxy norm times S_mha);
+    "pap" by S_mha alone (Eq. 4), the criterion Table 4 compares the proxy network against."""
     rnd = rounding(mode)
     W = _w64(W)
     X = np.array(X, dtype=F64)
@@ -252,7 +255,10 @@ def layer_prefill_skip(X, pos, W, shape, m_attn, m_ffn, g_attn=None, g_ffn=None,
 
     # --- LTP + reduced FFN (on the updated residual; S_mha from before the update)
     B = rmsnorm(X, g2, shape.rms_eps)
-    C, S_ffn = ltp_score(B, S_mha, W, rnd)
+    if ffn_criterion == "pap":
+        C, S_ffn = None, S_mha
+    else:
+        C, S_ffn = ltp_score(B, S_mha, W, rnd)
     Tf = topk_select(S_ffn, m_ffn, force_last)
     X[Tf] = rnd(X[Tf] + ffn(B[Tf], W["w_gate"], W["w_up"], W["w_down"], rnd))
 

@@ -21,6 +21,7 @@ FORCE_LAST = 1
 OPT_REFERENCE_KERNELS = 2
 OPT_ATTENTION_ONE_TILE = 4
 OPT_PAP_WINDOW = 8
+OPT_FFN_SCORE_PAP_ONLY = 16
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT",
                 6: "NONFINITE", 7: "UNSUPPORTED"}
@@ -225,6 +226,10 @@ class Spts:
 
     def set_pap_window(self, window: int):
         self._check(self.lib.spts_set_option(self.h, OPT_PAP_WINDOW, int(window)), "spts_set_option")
+
+    def set_ffn_score_pap_only(self, on: bool):
+        """T_f = TopK(S_mha, m_ffn): the FFN criterion without the proxy network (Table 4's baseline row)."""
+        self._check(self.lib.spts_set_option(self.h, OPT_FFN_SCORE_PAP_ONLY, 1 if on else 0), "spts_set_option")
 
     def set_attention_one_tile(self, on: bool):
         self._check(self.lib.spts_set_option(self.h, OPT_ATTENTION_ONE_TILE, 1 if on else 0), "spts_set_option")

@@ -308,6 +308,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->sm_count = prop.multiProcessorCount;
   ctx->encode_tiled = nullptr;
   ctx->attn_one_tile = false;
+  ctx->ffn_score_pap_only = false;
   ctx->rope_trust = false;
   ctx->rope_pos = nullptr;
   ctx->rope_n = 0;
@@ -379,6 +380,10 @@ spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
   }
   if (option == SPTS_ATTENTION_ONE_TILE) {
     ctx->attn_one_tile = value != 0;
+    return SPTS_OK;
+  }
+  if (option == SPTS_FFN_SCORE_PAP_ONLY) {
+    ctx->ffn_score_pap_only = value != 0;
     return SPTS_OK;
   }
   return SPTS_ERR_INVALID_ARG;
@@ -490,8 +495,12 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   const int32_t* idx_f = nullptr;
   if (sel_f) {
     int32_t* jf = idx_ffn_out ? idx_ffn_out : ws.idx_f;
-    TRY(ltp_pipeline(ctx, w, X, S, N, nullptr, ws.s_ffn));
-    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_ffn, launch_topk(ctx, ws.s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
+    const float* s_ffn = S;                            // Table 4's baseline criterion: the probe's score as it is
+    if (!ctx->ffn_score_pap_only) {
+      TRY(ltp_pipeline(ctx, w, X, S, N, nullptr, ws.s_ffn));
+      s_ffn = ws.s_ffn;
+    }
+    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_ffn, launch_topk(ctx, s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
     idx_f = jf;
   } else if (idx_ffn_out) {
     TRY(launch_topk(ctx, S, N, N, flags, idx_ffn_out, ws.topk_scratch));

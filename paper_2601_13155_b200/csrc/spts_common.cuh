@@ -92,6 +92,7 @@ struct spts_ctx {
   spts::Workspace ws;
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
   bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
+  bool ffn_score_pap_only;   // T_f from S_mha alone (no proxy FFN)
   // rotary table reuse inside spts_prefill: positions only change at a stage end, so the table computed for
   // (pos pointer, N) stays valid for the following layers of the stage
   bool rope_trust;

@@ -356,3 +356,36 @@ def test_decode_attention_over_long_caches(layout, n0):
         check_output(host(cache.k[0][n0 + step]), oc[0]["K"][n0 + step], "bf16")
     assert cache.length(0) == n0 + 2 and lib.device_status() == 0
     lib.close()
+
+
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", False)])
+def test_ffn_selection_by_the_attention_score_alone(dtype, ref):
+    """The setting of the paper's proxy-network ablation (Table 4): attention dense, 40 % of the tokens skipped in the
+    FFN block, selected by S_mha (Eq. 4) alone.  T_f must be exactly TopK of the library's own S_mha, the update must
+    match the oracle run with the same criterion, and switching the option off must bring Eq. 14 back."""
+    shape = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    N, mf = 640, 384
+    lib = _mk(shape, 1024, ref)
+    W, X, lw = _layer_case(shape, N, 1041, heavy=16, std=0.03)
+    from paper_2601_13155_b200 import binding
+    pos = i32(np.arange(N) * 3 + 1)
+    out = {}
+    for on in (True, False):
+        lib.set_ffn_score_pap_only(on)
+        Xd = up(X, shape.dtype)
+        S = torch.empty(N, dtype=torch.float32, device=dev())
+        jf = torch.empty(mf, dtype=torch.int32, device=dev())
+        lib.layer_prefill_skip(lw, Xd, pos, N, mf, binding.KvCache(shape, 1, N), S_out=S, idx_ffn_out=jf)
+        assert lib.device_status() == 0
+        out[on] = (host(Xd), host(S).astype(np.float32), jf.cpu().numpy())
+    xg, Sg, jg = out[True]
+    assert np.array_equal(jg, O.topk_select(Sg, mf, True))
+    mode = "bf16" if shape.dtype == "bf16" else "exact"
+    want = O.layer_prefill_skip(X, np.arange(N) * 3 + 1, W, shape, N, mf, mode=mode, ffn_criterion="pap")
+    assert np.abs(Sg - want["S_mha"]).max() <= 2e-4 * want["S_mha"].max()
+    check_index_set(jg, want["S_mha"], mf)
+    same = np.setdiff1d(np.arange(N), np.setxor1d(jg, want["idx_ffn"]))
+    check_output(xg[same], want["X"][same], shape.dtype)
+    # with the option off the proxy decides again: a different set on these inputs
+    assert not np.array_equal(out[False][2], jg)
+    lib.close()

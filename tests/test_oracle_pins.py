@@ -543,3 +543,24 @@ def test_window_probe_reduces_to_eq4_and_to_dense_attention_rows():
         _, S = O.pap_score_window(A, pos, wk, wq, SH, w)
         assert np.allclose(S, want, rtol=1e-10, atol=1e-14), w
         assert abs(S.sum() - 1.0) < 1e-12
+
+
+def test_attention_score_criterion_selects_the_attention_set():
+    """Table 4's baseline criterion (FFN tokens chosen by Eq. 4 alone): with equal budgets T_f is T_a, since both are
+    TopK of the same score; with dense attention it is the brute-force top of S_mha; and a proxy whose response norm is
+    the same for every token (C = const) makes Eq. 14 choose the same set."""
+    W = _layer()
+    N = 48
+    X = _x(N)
+    pos = np.arange(N)
+    r = O.layer_prefill_skip(X, pos, W, SH, 20, 20, ffn_criterion="pap")
+    assert np.array_equal(r["idx_ffn"], r["idx_attn"]) and r["C"] is None
+    assert np.array_equal(r["S_ffn"], r["S_mha"])
+    r2 = O.layer_prefill_skip(X, pos, W, SH, N, 17, ffn_criterion="pap")
+    assert np.array_equal(r2["idx_ffn"], np.sort(_brute_topk(r2["S_mha"], 17, True)))
+    # Eq. 14 with a constant C orders tokens as S_mha does
+    C = np.full(N, 3.5)
+    assert np.array_equal(O.topk_select(C * r2["S_mha"], 17, True), r2["idx_ffn"])
+    # and the criterion matters: the proxy's choice differs on these inputs
+    r3 = O.layer_prefill_skip(X, pos, W, SH, N, 17)
+    assert not np.array_equal(r3["idx_ffn"], r2["idx_ffn"])
