@@ -240,6 +240,24 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
                                     uint32_t flags, spts_kv_layer* cache, float* S_mha_out,
                                     int32_t* idx_attn_out, int32_t* idx_ffn_out);
 
+/* The same layer for several independent prompts packed row after row into X [total, D] (the paper evaluates one
+ * prompt at a time; Algorithm 1 applies to each prompt on its own, and that is what this call computes):
+ * sequence b owns rows [seq_start[b], seq_start[b + 1]) of X and pos, has its own budgets m_attn[b], m_ffn[b]
+ * (1 <= m <= its length) and its own cache caches[b].  seq_start [n_seq + 1], m_attn [n_seq], m_ffn [n_seq] and the
+ * caches array are HOST memory; seq_start[0] == 0 and total = seq_start[n_seq] <= max_seq.
+ * Everything that Eq. 4, 5 and 15 define per prompt stays per prompt: the probe uses each sequence's own last
+ * token, its softmax runs over that sequence's candidates, TopK selects within the sequence (SPTS_FORCE_LAST keeps
+ * each sequence's last row), attention is causal within the sequence.  The attention blocks run one sequence after
+ * the other; the row normalisation, the proxy FFN of Eq. 12-14 and the selected rows' SwiGLU FFN (Eq. 6) run once
+ * over the packed rows of all sequences -- one gathered GEMM with a ragged index list.  Every row gets the bits the
+ * single-sequence call gives it.
+ * Optional outputs: S_mha_out [total]; idx_attn_out [sum m_attn] and idx_ffn_out [sum m_ffn], sequence after
+ * sequence, each numbered from the sequence's own first row. */
+spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos,
+                                          int n_seq, const int32_t* seq_start, const int32_t* m_attn,
+                                          const int32_t* m_ffn, uint32_t flags, spts_kv_layer* caches,
+                                          float* S_mha_out, int32_t* idx_attn_out, int32_t* idx_ffn_out);
+
 /* Stage-end pruning, Eq. 16 / Algorithm 1 "X <- X[T^{l+1}, :]": keeps the
  * n_next = min(N, N_{s+1}) candidates with the largest S_mha, in token order.  Out of place:
  * X_out [n_next, D], pos_out, orig_out [n_next] must not alias the inputs; idx_out [n_next]

@@ -63,7 +63,8 @@ EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_opti
            "spts_last_device_status", "spts_launch_count", "spts_fold_norm_gain", "spts_pap_score",
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
            "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
-           "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build")
+           "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build",
+           "spts_layer_prefill_skip_batch")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -96,6 +97,9 @@ def load_library() -> C.CDLL:
                                      vp, vp, vp, vp, vp, vp, vp]
     lib.spts_layer_prefill_skip.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, i32, i32, u32,
                                             C.POINTER(KvLayerC), vp, vp, vp]
+    lib.spts_layer_prefill_skip_batch.argtypes = [vp, C.POINTER(LayerWeightsC), vp, vp, i32, C.POINTER(C.c_int32),
+                                                  C.POINTER(C.c_int32), C.POINTER(C.c_int32), u32,
+                                                  C.POINTER(KvLayerC), vp, vp, vp]
     lib.spts_msdp_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, vp, vp, vp, vp]
     lib.spts_first_token.argtypes = [vp, vp, vp, vp, vp]
     lib.spts_prefill.argtypes = [vp, C.POINTER(ModelWeightsC), C.POINTER(LayerPlanC), vp, vp, vp, vp, vp, vp,
@@ -288,6 +292,17 @@ class Spts:
                                                      flags, C.byref(cache.c[layer]), _ptr(S_out),
                                                      _ptr(idx_attn_out), _ptr(idx_ffn_out)),
                     "spts_layer_prefill_skip")
+
+    def layer_prefill_skip_batch(self, w: LayerWeights, X, pos, seq_start, m_attn, m_ffn, caches: KvCache,
+                                 flags: int = FORCE_LAST, S_out=None, idx_attn_out=None, idx_ffn_out=None):
+        """Several prompts packed into X; `caches` holds one entry per sequence (a KvCache built with
+        n_layers = number of sequences); seq_start, m_attn, m_ffn are host integer lists."""
+        n_seq = len(m_attn)
+        arr = lambda v: (C.c_int32 * len(v))(*[int(x) for x in v])
+        self._check(self.lib.spts_layer_prefill_skip_batch(self.h, C.byref(w.c), _ptr(X), _ptr(pos), n_seq,
+                                                           arr(seq_start), arr(m_attn), arr(m_ffn), flags, caches.c,
+                                                           _ptr(S_out), _ptr(idx_attn_out), _ptr(idx_ffn_out)),
+                    "spts_layer_prefill_skip_batch")
 
     def msdp_compact(self, X_in, pos_in, orig_in, S_mha, n_next: int, X_out, pos_out, orig_out, idx_out=None,
                      flags: int = FORCE_LAST):

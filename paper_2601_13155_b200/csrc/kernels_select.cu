@@ -315,6 +315,19 @@ spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* id
   return SPTS_OK;
 }
 
+// dst[i] = src[i] + offset: a sequence's own row numbers -> rows of the packed batch
+__global__ void offset_i32_kernel(const int32_t* __restrict__ src, int n, int offset, int32_t* __restrict__ dst) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i] + offset;
+}
+
+spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offset, int32_t* dst) {
+  if (n == 0) return SPTS_OK;
+  offset_i32_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(src, n, offset, dst);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
 spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst) {
   if (n == 0) return SPTS_OK;
   gather_i32_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(src, idx, n, dst);

@@ -277,6 +277,82 @@ spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   return SPTS_OK;
 }
 
+// PAP + reduced MHA of one sequence (Eq. 4, 5, Eq. 2 for the attention block): X rows updated in place, cache filled.
+// want_scores: S is needed later (FFN selection or the caller asked for it).
+spts_status attention_block(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos, int N, int m_attn,
+                            bool want_scores_later, uint32_t flags, spts_kv_layer* cache, float* S,
+                            int32_t* idx_attn_out) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int D = d.hidden, HD = d.n_q_heads * d.head_dim, KD = d.n_kv_heads * d.head_dim;
+  const size_t es = elt_size(d);
+  const bool sel_a = m_attn < N;
+  const bool want_scores = sel_a || want_scores_later;
+  const bool tc = use_tc(ctx);
+
+  // ---- PAP + reduced MHA
+  void* k_dst = sel_a ? ws.k_all : cache->k;
+  TRY(pap_pipeline(ctx, w, X, pos, N, k_dst, want_scores, S));
+  const int32_t* idx_a = nullptr;
+  if (sel_a) {
+    int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
+    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_attn, launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
+    OP(SPTS_OP_KV_GATHER, 0.0, 2.0 * m_attn * (double)KD * es + 8.0 * m_attn,
+       launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
+    OP(SPTS_OP_KV_GATHER, 0.0, 12.0 * m_attn, launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
+    idx_a = ia;
+  } else {
+    if (cudaMemcpyAsync(cache->pos, pos, (size_t)N * sizeof(int32_t), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+      return SPTS_ERR_CUDA;
+    if (idx_attn_out) TRY(launch_topk(ctx, S, N, N, flags, idx_attn_out, ws.topk_scratch));
+  }
+  const int ldvt = (int)align_up((size_t)m_attn, 128);
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_a; g.W = w->wq; g.M = m_attn; g.Nout = HD; g.K = D;
+  g.rowscale = ws.rstd; g.out = ws.q_act; g.ldo = HD;
+  const double Ma = (double)m_attn, Dd = (double)D, esd = (double)es;
+  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * HD, (Ma * Dd + Ma * HD + Dd * HD) * esd, run_gemm(ctx, REF_ROPE, g));
+  g.W = w->wv; g.Nout = KD; g.out = cache->v; g.ldo = KD;
+  if (tc) { g.out_t = ws.v_t; g.ldt = ldvt; }
+  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * KD, (Ma * Dd + 2.0 * Ma * KD + Dd * KD) * esd, run_gemm(ctx, REF_STORE, g));
+  ProfScope* ps_att = new ProfScope(ctx, SPTS_OP_ATTN, 2.0 * HD * Ma * (Ma + 1.0), (2.0 * Ma * HD + 2.0 * Ma * KD) * esd);
+  spts_status s_att = SPTS_OK;
+  if (tc) s_att = (launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)cache->v, (const bf16*)ws.v_t, ldvt, m_attn,
+                                  (bf16*)ws.o_att));
+  else s_att = launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att);
+  delete ps_att;
+  TRY(s_att);
+  memset(&g, 0, sizeof(g));
+  g.A = ws.o_att; g.lda = HD; g.a_rows = m_attn; g.dst_idx = idx_a; g.W = w->wo; g.M = m_attn; g.Nout = D; g.K = HD;
+  g.out = X; g.ldo = D;
+  OP(SPTS_OP_OPROJ, 2.0 * Ma * Dd * HD, (Ma * HD + 2.0 * Ma * Dd + Dd * HD) * esd, run_gemm(ctx, REF_RESID, g));
+  cache->len = m_attn;
+
+  return SPTS_OK;
+}
+
+// SwiGLU FFN on the rows `idx_f` (nullptr: all a_rows rows) of X with the residual scatter (Eq. 6, Eq. 2); X is
+// normalised through ws.rstd
+spts_status ffn_gemms(spts_ctx* ctx, const spts_layer_weights* w, void* X, int N, const int32_t* idx_f, int m_ffn) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int D = d.hidden;
+  const double Mf = (double)m_ffn, Dd = (double)D, esd = (double)elt_size(d);
+  Gemm g;
+  memset(&g, 0, sizeof(g));
+  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_f; g.W = w->w_gate; g.W2 = w->w_up; g.M = m_ffn; g.Nout = d.ffn_dim;
+  g.K = D; g.rowscale = ws.rstd; g.out = ws.hm; g.ldo = d.ffn_dim;
+  OP(SPTS_OP_GATEUP, 4.0 * Mf * Dd * d.ffn_dim, (Mf * Dd + Mf * d.ffn_dim + 2.0 * Dd * d.ffn_dim) * esd,
+     run_gemm(ctx, REF_SWIGLU, g));
+  memset(&g, 0, sizeof(g));
+  g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = m_ffn; g.dst_idx = idx_f; g.W = w->w_down; g.M = m_ffn; g.Nout = D;
+  g.K = d.ffn_dim; g.out = X; g.ldo = D;
+  OP(SPTS_OP_DOWN, 2.0 * Mf * Dd * d.ffn_dim, (Mf * d.ffn_dim + 2.0 * Mf * Dd + Dd * d.ffn_dim) * esd,
+     run_gemm(ctx, REF_RESID, g));
+  return SPTS_OK;
+}
+
 spts_status check_ctx(const spts_ctx* ctx) { return ctx == nullptr ? SPTS_ERR_INVALID_ARG : SPTS_OK; }
 
 }  // namespace
@@ -444,54 +520,12 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   if (!aligned16(X) || !aligned16(cache->k) || !aligned16(cache->v)) return SPTS_ERR_INVALID_ARG;
   const auto& d = ctx->desc;
   Workspace& ws = ctx->ws;
-  const int D = d.hidden, HD = d.n_q_heads * d.head_dim, KD = d.n_kv_heads * d.head_dim;
-  const size_t es = elt_size(d);
-  const bool sel_a = m_attn < N, sel_f = m_ffn < N;
-  const bool want_scores = sel_a || sel_f || S_mha_out != nullptr;
+  const bool sel_f = m_ffn < N;
   float* S = S_mha_out ? S_mha_out : ws.s_mha;
-  const bool tc = use_tc(ctx);
-
-  // ---- PAP + reduced MHA
-  void* k_dst = sel_a ? ws.k_all : cache->k;
-  TRY(pap_pipeline(ctx, w, X, pos, N, k_dst, want_scores, S));
-  const int32_t* idx_a = nullptr;
-  if (sel_a) {
-    int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
-    OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_attn, launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
-    OP(SPTS_OP_KV_GATHER, 0.0, 2.0 * m_attn * (double)KD * es + 8.0 * m_attn,
-       launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
-    OP(SPTS_OP_KV_GATHER, 0.0, 12.0 * m_attn, launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
-    idx_a = ia;
-  } else {
-    if (cudaMemcpyAsync(cache->pos, pos, (size_t)N * sizeof(int32_t), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
-      return SPTS_ERR_CUDA;
-    if (idx_attn_out) TRY(launch_topk(ctx, S, N, N, flags, idx_attn_out, ws.topk_scratch));
-  }
-  const int ldvt = (int)align_up((size_t)m_attn, 128);
-  Gemm g;
-  memset(&g, 0, sizeof(g));
-  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_a; g.W = w->wq; g.M = m_attn; g.Nout = HD; g.K = D;
-  g.rowscale = ws.rstd; g.out = ws.q_act; g.ldo = HD;
-  const double Ma = (double)m_attn, Mf = (double)m_ffn, Dd = (double)D, esd = (double)es;
-  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * HD, (Ma * Dd + Ma * HD + Dd * HD) * esd, run_gemm(ctx, REF_ROPE, g));
-  g.W = w->wv; g.Nout = KD; g.out = cache->v; g.ldo = KD;
-  if (tc) { g.out_t = ws.v_t; g.ldt = ldvt; }
-  OP(SPTS_OP_QVPROJ, 2.0 * Ma * Dd * KD, (Ma * Dd + 2.0 * Ma * KD + Dd * KD) * esd, run_gemm(ctx, REF_STORE, g));
-  ProfScope* ps_att = new ProfScope(ctx, SPTS_OP_ATTN, 2.0 * HD * Ma * (Ma + 1.0), (2.0 * Ma * HD + 2.0 * Ma * KD) * esd);
-  spts_status s_att = SPTS_OK;
-  if (tc) s_att = (launch_tc_attention(ctx, (const bf16*)ws.q_act, (const bf16*)cache->k, (const bf16*)cache->v, (const bf16*)ws.v_t, ldvt, m_attn,
-                                  (bf16*)ws.o_att));
-  else s_att = launch_ref_attention(ctx, ws.q_act, cache->k, cache->v, m_attn, ws.o_att);
-  delete ps_att;
-  TRY(s_att);
-  memset(&g, 0, sizeof(g));
-  g.A = ws.o_att; g.lda = HD; g.a_rows = m_attn; g.dst_idx = idx_a; g.W = w->wo; g.M = m_attn; g.Nout = D; g.K = HD;
-  g.out = X; g.ldo = D;
-  OP(SPTS_OP_OPROJ, 2.0 * Ma * Dd * HD, (Ma * HD + 2.0 * Ma * Dd + Dd * HD) * esd, run_gemm(ctx, REF_RESID, g));
-  cache->len = m_attn;
+  TRY(attention_block(ctx, w, X, pos, N, m_attn, sel_f || S_mha_out != nullptr, flags, cache, S, idx_attn_out));
 
   // ---- LTP + reduced FFN on the updated residual
-  OP(SPTS_OP_PREP, 0.0, (double)N * Dd * esd + 4.0 * N, launch_rstd(ctx, X, N, ws.rstd));
+  OP(SPTS_OP_PREP, 0.0, (double)N * d.hidden * (double)elt_size(d) + 4.0 * N, launch_rstd(ctx, X, N, ws.rstd));
   const int32_t* idx_f = nullptr;
   if (sel_f) {
     int32_t* jf = idx_ffn_out ? idx_ffn_out : ws.idx_f;
@@ -505,17 +539,68 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   } else if (idx_ffn_out) {
     TRY(launch_topk(ctx, S, N, N, flags, idx_ffn_out, ws.topk_scratch));
   }
-  memset(&g, 0, sizeof(g));
-  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_f; g.W = w->w_gate; g.W2 = w->w_up; g.M = m_ffn; g.Nout = d.ffn_dim;
-  g.K = D; g.rowscale = ws.rstd; g.out = ws.hm; g.ldo = d.ffn_dim;
-  OP(SPTS_OP_GATEUP, 4.0 * Mf * Dd * d.ffn_dim, (Mf * Dd + Mf * d.ffn_dim + 2.0 * Dd * d.ffn_dim) * esd,
-     run_gemm(ctx, REF_SWIGLU, g));
-  memset(&g, 0, sizeof(g));
-  g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = m_ffn; g.dst_idx = idx_f; g.W = w->w_down; g.M = m_ffn; g.Nout = D;
-  g.K = d.ffn_dim; g.out = X; g.ldo = D;
-  OP(SPTS_OP_DOWN, 2.0 * Mf * Dd * d.ffn_dim, (Mf * d.ffn_dim + 2.0 * Mf * Dd + Dd * d.ffn_dim) * esd,
-     run_gemm(ctx, REF_RESID, g));
-  return SPTS_OK;
+  return ffn_gemms(ctx, w, X, N, idx_f, m_ffn);
+}
+
+spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos,
+                                          int n_seq, const int32_t* seq_start, const int32_t* m_attn,
+                                          const int32_t* m_ffn, uint32_t flags, spts_kv_layer* caches,
+                                          float* S_mha_out, int32_t* idx_attn_out, int32_t* idx_ffn_out) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || X == nullptr || pos == nullptr || caches == nullptr || seq_start == nullptr ||
+      m_attn == nullptr || m_ffn == nullptr)
+    return SPTS_ERR_INVALID_ARG;
+  if (n_seq < 1 || seq_start[0] != 0) return SPTS_ERR_INVALID_ARG;
+  const int total = seq_start[n_seq];
+  if (total < 1 || total > ctx->max_seq) return SPTS_ERR_SHAPE;
+  if (!aligned16(X)) return SPTS_ERR_INVALID_ARG;
+  bool any_sel_f = false;
+  for (int b = 0; b < n_seq; ++b) {
+    const int Nb = seq_start[b + 1] - seq_start[b];
+    if (Nb < 1) return SPTS_ERR_INVALID_ARG;
+    if (m_attn[b] < 1 || m_attn[b] > Nb || m_ffn[b] < 1 || m_ffn[b] > Nb) return SPTS_ERR_INVALID_ARG;
+    const spts_kv_layer& c = caches[b];
+    if (c.k == nullptr || c.v == nullptr || c.pos == nullptr) return SPTS_ERR_INVALID_ARG;
+    if (c.capacity < m_attn[b]) return SPTS_ERR_WORKSPACE;
+    if (!aligned16(c.k) || !aligned16(c.v)) return SPTS_ERR_INVALID_ARG;
+    any_sel_f = any_sel_f || m_ffn[b] < Nb;
+  }
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const size_t row_bytes = (size_t)d.hidden * elt_size(d);
+  float* S = S_mha_out ? S_mha_out : ws.s_mha;
+  // ---- attention blocks, one sequence after the other: the probe's softmax, the selection and the causal mask
+  //      are per sequence.  The rotary table is rebuilt for every slice.
+  int off_a = 0;
+  for (int b = 0; b < n_seq; ++b) {
+    const int s0 = seq_start[b], Nb = seq_start[b + 1] - s0;
+    ctx->rope_trust = false;
+    TRY(attention_block(ctx, w, (char*)X + (size_t)s0 * row_bytes, pos + s0, Nb, m_attn[b],
+                        m_ffn[b] < Nb || S_mha_out != nullptr, flags, &caches[b], S + s0,
+                        idx_attn_out ? idx_attn_out + off_a : nullptr));
+    off_a += m_attn[b];
+  }
+  // ---- FFN block over the packed rows: one norm pass, one proxy chain, one gathered FFN for all sequences
+  OP(SPTS_OP_PREP, 0.0, (double)total * (double)row_bytes + 4.0 * total, launch_rstd(ctx, X, total, ws.rstd));
+  const float* s_ffn = S;
+  if (any_sel_f && !ctx->ffn_score_pap_only) {
+    TRY(ltp_pipeline(ctx, w, X, S, total, nullptr, ws.s_ffn));
+    s_ffn = ws.s_ffn;
+  }
+  int off_f = 0;
+  for (int b = 0; b < n_seq; ++b) {
+    const int s0 = seq_start[b], Nb = seq_start[b + 1] - s0, mf = m_ffn[b];
+    int32_t* local = idx_ffn_out ? idx_ffn_out + off_f : ws.idx_p;
+    if (mf < Nb) {
+      OP(SPTS_OP_TOPK, 0.0, 4.0 * Nb + 4.0 * mf, launch_topk(ctx, s_ffn + s0, Nb, mf, flags, local, ws.topk_scratch));
+      if (any_sel_f) TRY(launch_offset_i32(ctx, local, mf, s0, ws.idx_f + off_f));
+    } else {
+      if (idx_ffn_out) TRY(launch_iota_from(ctx, local, Nb, 0));
+      if (any_sel_f) TRY(launch_iota_from(ctx, ws.idx_f + off_f, Nb, s0));
+    }
+    off_f += mf;
+  }
+  return ffn_gemms(ctx, w, X, total, any_sel_f ? ws.idx_f : nullptr, off_f);
 }
 
 spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* pos_in, const int32_t* orig_in,

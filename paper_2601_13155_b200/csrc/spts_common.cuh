@@ -120,6 +120,7 @@ spts_status launch_topk(spts_ctx* ctx, const float* scores, int N, int k, uint32
 spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* idx, int n_rows,
                                int row_bytes, void* dst);
 spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst);
+spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offset, int32_t* dst);
 
 // ---- kernels_probe.cu
 spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd);

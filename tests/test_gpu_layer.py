@@ -389,3 +389,64 @@ def test_ffn_selection_by_the_attention_score_alone(dtype, ref):
     # with the option off the proxy decides again: a different set on these inputs
     assert not np.array_equal(out[False][2], jg)
     lib.close()
+
+
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", False)])
+def test_packed_batch_equals_one_call_per_sequence(dtype, ref):
+    """spts_layer_prefill_skip_batch on four ragged prompts (one of them dense in the FFN, one dense in attention, one a
+    single token) against spts_layer_prefill_skip on each prompt alone: hidden states, scores, both index lists and the
+    caches must agree bit for bit -- the packed FFN GEMMs compute every row exactly as the per-sequence ones do -- and
+    the single-sequence call is what the oracle comparisons above cover."""
+    from paper_2601_13155_b200 import binding
+    shape = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    lens = [300, 1, 517, 130]
+    ma = [150, 1, 517, 70]
+    mf = [120, 1, 200, 130]
+    start = np.concatenate([[0], np.cumsum(lens)])
+    total = int(start[-1])
+    lib = _mk(shape, 1024, ref)
+    W, X, lw = _layer_case(shape, total, 1051, heavy=20, std=0.03)
+    pos_h = np.concatenate([np.arange(n) * 2 + 5 * b for b, n in enumerate(lens)]).astype(np.int32)
+    pos = i32(pos_h)
+    # one call per sequence
+    Xs = up(X, shape.dtype)
+    Ss = torch.zeros(total, dtype=torch.float32, device=dev())
+    single = binding.KvCache(shape, len(lens), [m + 1 for m in ma])
+    ia_s, jf_s = [], []
+    for b, n in enumerate(lens):
+        s0 = int(start[b])
+        ia = torch.empty(ma[b], dtype=torch.int32, device=dev())
+        jf = torch.empty(mf[b], dtype=torch.int32, device=dev())
+        lib.layer_prefill_skip(lw, Xs[s0:s0 + n], pos[s0:s0 + n], ma[b], mf[b], single, layer=b, S_out=Ss[s0:s0 + n],
+                               idx_attn_out=ia, idx_ffn_out=jf)
+        ia_s.append(ia)
+        jf_s.append(jf)
+    # the packed call
+    Xb = up(X, shape.dtype)
+    Sb = torch.zeros(total, dtype=torch.float32, device=dev())
+    packed = binding.KvCache(shape, len(lens), [m + 1 for m in ma])
+    ia_b = torch.empty(sum(ma), dtype=torch.int32, device=dev())
+    jf_b = torch.empty(sum(mf), dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip_batch(lw, Xb, pos, start, ma, mf, packed, S_out=Sb, idx_attn_out=ia_b, idx_ffn_out=jf_b)
+    assert lib.device_status() == 0
+    assert torch.equal(Xb, Xs)
+    assert torch.equal(ia_b, torch.cat(ia_s)) and torch.equal(jf_b, torch.cat(jf_s))
+    for b, n in enumerate(lens):
+        s0 = int(start[b])
+        if ma[b] < n or mf[b] < n:
+            assert torch.equal(Sb[s0:s0 + n], Ss[s0:s0 + n])
+        assert packed.length(b) == ma[b] == single.length(b)
+        assert torch.equal(packed.k[b][:ma[b]], single.k[b][:ma[b]])
+        assert torch.equal(packed.v[b][:ma[b]], single.v[b][:ma[b]])
+        assert torch.equal(packed.pos[b][:ma[b]], single.pos[b][:ma[b]])
+    # and without the optional outputs
+    Xc = up(X, shape.dtype)
+    lib.layer_prefill_skip_batch(lw, Xc, pos, start, ma, mf, binding.KvCache(shape, len(lens), [m + 1 for m in ma]))
+    assert torch.equal(Xc, Xs)
+    # host-side argument checks: a budget above the sequence length, a start list that does not begin at 0
+    with pytest.raises(binding.SptsError):
+        lib.layer_prefill_skip_batch(lw, Xc, pos, start, [150, 2, 517, 70], mf, packed)
+    with pytest.raises(binding.SptsError):
+        lib.layer_prefill_skip_batch(lw, Xc, pos, start + 1, ma, mf, packed)
+    assert lib.device_status() == 0
+    lib.close()
