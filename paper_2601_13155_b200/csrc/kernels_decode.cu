@@ -10,7 +10,12 @@
 //                SwiGLU of the gate / up pair; residual update (O and down projections).
 //   attention    one CTA = one KV head x one slice of the cache, serving the whole GQA group of
 //                query heads at once (each cached row is read once), online softmax, then a
-//                combine kernel over the slices.
+//                combine kernel over the slices.  bf16 caches: warp-level tensor-core MMAs with
+//                both operands loaded from global memory in fragment order (dec_attn_mma_kernel);
+//                fp32 caches: CUDA cores (dec_attn_partial_kernel).
+//   launches     every kernel of a step is a programmatic dependent of the one before: it lets
+//                its successor start, pulls what does not depend on its predecessor (weights,
+//                old cache rows) towards L2 or into registers, and only then waits.
 // The residual vector lives in fp32 scratch and is rounded through the storage type at the same
 // points as the prefill path.
 #include <type_traits>
