@@ -38,6 +38,12 @@ NCU_TRAFFIC_BYTES = {
     ("cfg3", "attention"): 360.78e6 + 102.51e6,     # tc_attention_pair_kernel, m_attn = 16384
     ("cfg3", "down"): 1627.55e6 + 99.98e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
 }
+# Decode step at the 8B shape, from the ncu capture of a 4-layer case against 16384 cached rows per layer
+# (profiles/decode_step_8b_4layers.md): the five weight-streaming kernels of a layer move 453.3 MB, the attention
+# kernel 67.4 MB for 16384 rows = 4114 B per cached row.  Both grow in proportion (layers, cached rows), which is
+# how the figure is scaled to the 32-layer step against the benchmark's caches.
+NCU_DECODE_WEIGHT_BYTES_PER_LAYER = 453.3e6
+NCU_DECODE_KV_BYTES_PER_ROW = 4114.0
 
 
 def parse():
@@ -302,7 +308,10 @@ def generation_line(args, rep, dev):
                           "tokens_per_s": (N + T) * world / ((pd + dd) * 1e-3), "kv_token_layers": kv_d},
                 "keep_sweep": sweep,
                 "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                             "traffic": None, "kernel": "decode step (all layers, dense arm)", "launches": dk["calls"],
+                             "traffic": (L * NCU_DECODE_WEIGHT_BYTES_PER_LAYER + NCU_DECODE_KV_BYTES_PER_ROW * L * (N + T / 2.0))
+                             if shape == synth.LLAMA8B else None,
+                             "traffic_note": "ncu capture of a 4-layer case, scaled by layers and cached rows (see profiles/)",
+                             "kernel": "decode step (all layers, dense arm)", "launches": dk["calls"],
                              "ms_per_launch": dk["ms"] / dk["calls"],
                              "peak_source": "measured (copy)" if peaks else "fallback"},
                 "gpu_launches": int(lib.launch_count())}
