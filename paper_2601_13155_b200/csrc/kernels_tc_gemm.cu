@@ -38,6 +38,12 @@ template <int BN> struct Cfg {
   static constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 1024 + 256;
   static constexpr int TMEM_COLS = 2 * BN;
 };
+// The rotary epilogue stages, per epilogue warp, the (cos, sin) pairs of its 32 rows for half the frequencies:
+// 32 rows x 256 bytes x 4 warps, after the barrier block.
+constexpr int ROPE_STAGE_BYTES = 4 * 32 * 256;
+template <int BN, int EPI> constexpr int gemm_smem_bytes() {
+  return Cfg<BN>::SMEM_BYTES + (EPI == TC_ROPE ? ROPE_STAGE_BYTES : 0);
+}
 
 struct TcParams {
   const int32_t* idx;
@@ -312,25 +318,54 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
       } else if (EPI == TC_ROPE) {
+        // Rotary embedding on the 128-wide heads of the tile (and, for the probe, the logits q_h . k of Eq. 4 from
+        // the unrounded keys).  The table row of a token (64 (cos, sin) pairs, 512 bytes) is the same for every head
+        // and every column tile; read per lane it is a 32-line gather per load, and that gather cost 11 % of the
+        // gathered Q projection.  So each warp stages its 32 rows' pairs for one half of the frequencies in shared
+        // memory -- two rows per load instruction, 16 lanes x 16 bytes each, fully used sectors -- and both heads of
+        // the tile read them from there (16-byte chunks XOR-swizzled by the row so that neither the staging stores
+        // nor the per-row reads conflict).
         const float inv_sqrt_d = 0.08838834764831845f;   // 1 / sqrt(128)
-#pragma unroll 1
-        for (int hh = 0; hh < BN / 128; ++hh) {
-          const int hcol = n0 + hh * 128;               // first column of this head
-          float dots[8];
+        constexpr int NH = BN / 128;                     // heads per tile
+        uint8_t* stage = gen + STAGES * (A_STAGE_BYTES + C::B_STAGE_BYTES) + 256 + quarter * (32 * 256);
+        float dots[NH][8];
 #pragma unroll
-          for (int g = 0; g < 8; ++g) dots[g] = 0.f;
+        for (int hh = 0; hh < NH; ++hh)
+#pragma unroll
+          for (int g = 0; g < 8; ++g) dots[hh][g] = 0.f;
 #pragma unroll 1
-          for (int jj = 0; jj < 2; ++jj) {
+        for (int jj = 0; jj < 2; ++jj) {
+          __syncwarp();                                  // the previous half's readers are done
+          {
+            float4 v[16];                                // all 16 loads in flight before the first store
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              const int r = 2 * k + (lane >> 4);
+              const int srow = __shfl_sync(0xffffffffu, src, r);
+              const int rok = __shfl_sync(0xffffffffu, (int)row_ok, r);
+              v[k] = make_float4(1.f, 0.f, 1.f, 0.f);
+              if (rok) v[k] = __ldg(reinterpret_cast<const float4*>(p.cs) + (size_t)srow * 32 + jj * 16 + (lane & 15));
+            }
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+              const int r = 2 * k + (lane >> 4), ch = lane & 15;
+              *reinterpret_cast<float4*>(stage + r * 256 + ((ch ^ (r & 15)) << 4)) = v[k];
+            }
+          }
+          __syncwarp();
+#pragma unroll
+          for (int hh = 0; hh < NH; ++hh) {
+            const int hcol = n0 + hh * 128;               // first column of this head
             uint32_t lo[32], hi[32];
             tmem_ld32(tacc + hh * 128 + jj * 32, lo);
             tmem_ld32(tacc + hh * 128 + 64 + jj * 32, hi);
             tmem_ld_wait();
             if (row_ok && hcol < p.Nout) {
               float a[32], b[32];
-              const float4* cs4 = reinterpret_cast<const float4*>(p.cs + (size_t)src * 64 + jj * 32);
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
-                float4 c2 = cs4[i >> 1];                 // (cos, sin) of two consecutive frequencies
+                // (cos, sin) of two consecutive frequencies
+                const float4 c2 = *reinterpret_cast<const float4*>(stage + lane * 256 + ((((i >> 1)) ^ (lane & 15)) << 4));
                 float x0 = __uint_as_float(lo[i]) * rs, y0 = __uint_as_float(hi[i]) * rs;
                 float x1 = __uint_as_float(lo[i + 1]) * rs, y1 = __uint_as_float(hi[i + 1]) * rs;
                 a[i] = x0 * c2.x - y0 * c2.y;
@@ -343,20 +378,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               store32_bf16(o + 64, b, 0, 32);
               if (p.logits != nullptr) {
                 const int kvh = hcol >> 7;
-                for (int g = 0; g < p.group && g < 8; ++g) {
-                  const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
-                  float d = dots[g];
 #pragma unroll
-                  for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
-                  dots[g] = d;
+                for (int g = 0; g < 8; ++g) {
+                  if (g < p.group) {
+                    const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
+                    float d = dots[hh][g];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
+                    dots[hh][g] = d;
+                  }
                 }
               }
             }
           }
-          if (p.logits != nullptr && row_ok && hcol < p.Nout) {
-            const int kvh = hcol >> 7;
-            for (int g = 0; g < p.group && g < 8; ++g)
-              p.logits[(size_t)(kvh * p.group + g) * p.ld_logits + grow] = dots[g] * inv_sqrt_d;
+        }
+        if (p.logits != nullptr && row_ok) {
+#pragma unroll
+          for (int hh = 0; hh < NH; ++hh) {
+            const int hcol = n0 + hh * 128;
+            if (hcol < p.Nout) {
+              const int kvh = hcol >> 7;
+#pragma unroll
+              for (int g = 0; g < 8; ++g)
+                if (g < p.group) p.logits[(size_t)(kvh * p.group + g) * p.ld_logits + grow] = dots[hh][g] * inv_sqrt_d;
+            }
           }
         }
       } else if (EPI == TC_SWIGLU) {
@@ -504,7 +549,7 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   }
   const int tiles = p.num_m * p.num_n;
   const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-  tc_gemm_kernel<BN, EPI, GATHER><<<grid, GATHER ? GEMM_THREADS + 32 * GATHER_WARPS : GEMM_THREADS, Cfg<BN>::SMEM_BYTES,
+  tc_gemm_kernel<BN, EPI, GATHER><<<grid, GATHER ? GEMM_THREADS + 32 * GATHER_WARPS : GEMM_THREADS, gemm_smem_bytes<BN, EPI>(),
                                     ctx->stream>>>(tmA, tmB, tmB2, p);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
@@ -523,10 +568,10 @@ spts_status launch_one(spts_ctx* ctx, const TcGemmArgs& a) {
 template <int BN, int EPI>
 bool set_smem_attr() {
   bool ok = cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+                                 gemm_smem_bytes<BN, EPI>()) == cudaSuccess;
   if (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU)
     ok = ok && cudaFuncSetAttribute(tc_gemm_kernel<BN, EPI, (EPI == TC_STORE || EPI == TC_ROPE || EPI == TC_SWIGLU)>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM_BYTES) == cudaSuccess;
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, gemm_smem_bytes<BN, EPI>()) == cudaSuccess;
   return ok;
 }
 
