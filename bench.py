@@ -34,9 +34,9 @@ import numpy as np
 
 # (workload, operation) -> DRAM bytes of one launch at the workload's stage-0 shape, measured with ncu
 NCU_TRAFFIC_BYTES = {
-    ("cfg3", "gate_up"): 1093.77e6 + 361.09e6,      # tc_gemm_kernel<256, 2, 1>, m_ffn = 13108
-    ("cfg3", "attention"): 360.78e6 + 102.51e6,     # tc_attention_pair_kernel, m_attn = 16384
-    ("cfg3", "down"): 1627.55e6 + 99.98e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
+    ("cfg3", "gate_up"): 1054.47e6 + 360.71e6,      # tc_gemm_kernel<256, 2, 1>, m_ffn = 13108
+    ("cfg3", "attention"): 360.84e6 + 102.60e6,     # tc_attention_pair_kernel, m_attn = 16384
+    ("cfg3", "down"): 1622.88e6 + 100.31e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
 }
 # Decode step at the 8B shape, from the ncu capture of a 4-layer case against 16384 cached rows per layer
 # (profiles/decode_step_8b_4layers.md): the five weight-streaming kernels of a layer move 453.3 MB, the attention
