@@ -30,11 +30,15 @@ __device__ __forceinline__ void load16<bf16>(const bf16* p, float* out) {
 }
 
 // rstd[n] = 1 / sqrt(mean(x_n^2) + eps); one warp per row.
+// With a row list (idx != nullptr) only the N listed rows are recomputed: the rows a block did not update keep the
+// statistic they had.
 template <typename T>
-__global__ void rstd_kernel(const T* __restrict__ X, int N, int D, float eps, float* __restrict__ rstd) {
+__global__ void rstd_kernel(const T* __restrict__ X, const int32_t* __restrict__ idx, int N, int D, float eps,
+                            float* __restrict__ rstd) {
   constexpr int V = Vec16<T>::N;
   int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= N) return;
+  if (idx != nullptr) row = idx[row];
   int lane = threadIdx.x & 31;
   const T* x = X + (size_t)row * D;
   float s = 0.f;
@@ -251,9 +255,22 @@ spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd) {
   const int D = ctx->desc.hidden;
   const int wpb = 8;
   if (ctx->desc.dtype == SPTS_BF16)
-    rstd_kernel<bf16><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const bf16*)X, N, D, ctx->desc.rms_eps, rstd);
+    rstd_kernel<bf16><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const bf16*)X, nullptr, N, D, ctx->desc.rms_eps, rstd);
   else
-    rstd_kernel<float><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const float*)X, N, D, ctx->desc.rms_eps, rstd);
+    rstd_kernel<float><<<ceil_div(N, wpb), wpb * 32, 0, ctx->stream>>>((const float*)X, nullptr, N, D, ctx->desc.rms_eps, rstd);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+// rstd[idx[i]] for i < n: the statistic of the listed rows only
+spts_status launch_rstd_rows(spts_ctx* ctx, const void* X, const int32_t* idx, int n, float* rstd) {
+  const int D = ctx->desc.hidden;
+  const int wpb = 8;
+  if (n == 0) return SPTS_OK;
+  if (ctx->desc.dtype == SPTS_BF16)
+    rstd_kernel<bf16><<<ceil_div(n, wpb), wpb * 32, 0, ctx->stream>>>((const bf16*)X, idx, n, D, ctx->desc.rms_eps, rstd);
+  else
+    rstd_kernel<float><<<ceil_div(n, wpb), wpb * 32, 0, ctx->stream>>>((const float*)X, idx, n, D, ctx->desc.rms_eps, rstd);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

@@ -525,7 +525,15 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
   TRY(attention_block(ctx, w, X, pos, N, m_attn, sel_f || S_mha_out != nullptr, flags, cache, S, idx_attn_out));
 
   // ---- LTP + reduced FFN on the updated residual
-  OP(SPTS_OP_PREP, 0.0, (double)N * d.hidden * (double)elt_size(d) + 4.0 * N, launch_rstd(ctx, X, N, ws.rstd));
+  // ws.rstd still holds the statistics of the layer's input (the probe computed them for every row); only the rows
+  // the attention block updated have changed
+  if (m_attn < N) {
+    const int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
+    OP(SPTS_OP_PREP, 0.0, (double)m_attn * d.hidden * (double)elt_size(d) + 8.0 * m_attn,
+       launch_rstd_rows(ctx, X, ia, m_attn, ws.rstd));
+  } else {
+    OP(SPTS_OP_PREP, 0.0, (double)N * d.hidden * (double)elt_size(d) + 4.0 * N, launch_rstd(ctx, X, N, ws.rstd));
+  }
   const int32_t* idx_f = nullptr;
   if (sel_f) {
     int32_t* jf = idx_ffn_out ? idx_ffn_out : ws.idx_f;

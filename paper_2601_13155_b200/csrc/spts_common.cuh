@@ -124,6 +124,7 @@ spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offs
 
 // ---- kernels_probe.cu
 spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd);
+spts_status launch_rstd_rows(spts_ctx* ctx, const void* X, const int32_t* idx, int n, float* rstd);
 spts_status launch_rope_table(spts_ctx* ctx, const int32_t* pos, int N, float2* cs);
 spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N, const void* wq,
                           const float* rstd, float* q);
