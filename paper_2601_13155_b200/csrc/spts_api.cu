@@ -215,7 +215,13 @@ spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   const int KD = d.n_kv_heads * d.head_dim;
   const int ld = (int)align_up((size_t)N, 128);
   const double es = (double)elt_size(d), Nd = (double)N, Dd = (double)d.hidden;
-  OP(SPTS_OP_PREP, 0.0, Nd * Dd * es + 4.0 * Nd, launch_rstd(ctx, X, N, ws.rstd));
+  if (ctx->rstd_rows != nullptr && ctx->rstd_x == X && ctx->rstd_n == N) {
+    // inside spts_prefill: only the rows the previous layer's FFN block updated have a new statistic
+    OP(SPTS_OP_PREP, 0.0, ctx->rstd_nrows * (Dd * es + 8.0), launch_rstd_rows(ctx, X, ctx->rstd_rows, ctx->rstd_nrows, ws.rstd));
+  } else {
+    OP(SPTS_OP_PREP, 0.0, Nd * Dd * es + 4.0 * Nd, launch_rstd(ctx, X, N, ws.rstd));
+  }
+  ctx->rstd_rows = nullptr;
   if (!(ctx->rope_trust && ctx->rope_pos == pos && ctx->rope_n == N)) {
     OP(SPTS_OP_PREP, 0.0, Nd * (4.0 + 4.0 * d.head_dim), launch_rope_table(ctx, pos, N, ws.rope_cs));
     ctx->rope_pos = pos;
@@ -385,6 +391,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->encode_tiled = nullptr;
   ctx->attn_one_tile = false;
   ctx->ffn_score_pap_only = false;
+  ctx->rstd_rows = nullptr;
   ctx->rope_trust = false;
   ctx->rope_pos = nullptr;
   ctx->rope_n = 0;
@@ -724,8 +731,8 @@ spts_status spts_prefill(spts_ctx* ctx, const spts_model_weights* mw, const spts
   // stays valid until the buffers swap
   struct RopeTrust {
     spts_ctx* c;
-    explicit RopeTrust(spts_ctx* cc) : c(cc) { c->rope_trust = true; c->rope_pos = nullptr; }
-    ~RopeTrust() { c->rope_trust = false; c->rope_pos = nullptr; }
+    explicit RopeTrust(spts_ctx* cc) : c(cc) { c->rope_trust = true; c->rope_pos = nullptr; c->rstd_rows = nullptr; }
+    ~RopeTrust() { c->rope_trust = false; c->rope_pos = nullptr; c->rstd_rows = nullptr; }
   } rope_guard(ctx);
   void* xc = X; int32_t* pc = pos; int32_t* oc = orig;
   void* xa = X_alt; int32_t* pa = pos_alt; int32_t* oa = orig_alt;
@@ -737,6 +744,12 @@ spts_status spts_prefill(spts_ctx* ctx, const spts_model_weights* mw, const spts
     if (prune && (xa == nullptr || pa == nullptr || oa == nullptr)) return SPTS_ERR_INVALID_ARG;
     TRY(spts_layer_prefill_skip(ctx, &mw->layers[l], xc, pc, cur, p.m_attn, p.m_ffn, flags, &caches[l],
                                 prune ? ctx->ws.s_mha : nullptr, nullptr, nullptr));
+    // The layer left ws.rstd current for its post-attention residual; its FFN block then changed the rows in
+    // ws.idx_f only.  Without a compaction the next layer's first norm pass can be limited to those rows.
+    ctx->rstd_rows = nullptr;
+    if (!prune && p.m_ffn < cur) {
+      ctx->rstd_rows = ctx->ws.idx_f; ctx->rstd_nrows = p.m_ffn; ctx->rstd_x = xc; ctx->rstd_n = cur;
+    }
     if (prune) {
       TRY(spts_msdp_compact(ctx, xc, pc, oc, ctx->ws.s_mha, cur, p.prune_to, flags, xa, pa, oa, nullptr));
       void* tx = xc; xc = xa; xa = tx;

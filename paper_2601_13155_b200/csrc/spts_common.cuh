@@ -93,6 +93,8 @@ struct spts_ctx {
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
   bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
   bool ffn_score_pap_only;   // T_f from S_mha alone (no proxy FFN)
+  // set by spts_prefill between two layers: ws.rstd is current for the rows of rstd_x [rstd_n] except the listed ones
+  const int32_t* rstd_rows; int rstd_nrows; const void* rstd_x; int rstd_n;
   // rotary table reuse inside spts_prefill: positions only change at a stage end, so the table computed for
   // (pos pointer, N) stays valid for the following layers of the stage
   bool rope_trust;
