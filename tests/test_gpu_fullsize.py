@@ -140,6 +140,12 @@ def test_bench_stage0_layer_sampled_rows_and_prune():
     lib.close()
 
 
+def test_bench_stage1_layer_sampled_rows():
+    """The benchmark's second-stage launch shape: 24576 candidates left by the first prune, budgets still 16384 / 13108
+    (two thirds of the rows in the attention block: other tile counts and gather densities than the first stage)."""
+    _run_layer_case("cfg3", 24576, 16384, 13108, 128)
+
+
 def test_bench_128k_stage0_layer_sampled_rows():
     """The longest context's first-stage launch shape (131072 candidates in 64-token heavy clusters, 65536 attention
     rows, 52429 FFN rows): scores and index sets in full, updates on sampled rows."""
