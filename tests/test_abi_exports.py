@@ -51,6 +51,9 @@ def test_host_argument_checks_need_no_gpu(lib_path):
     lib = binding.load_library()
     assert lib.spts_topk_select(None, None, 4, 2, 0, None) == 1        # SPTS_ERR_INVALID_ARG
     assert lib.spts_launch_count(None) == 0
+    # a call without a context is refused before anything is touched
+    assert lib.spts_layer_prefill_skip_batch(None, None, None, None, 2, None, None, None, 0, None, None, None, None) == 1
+    assert lib.spts_set_option(None, 16, 1) == 1
 
 
 def test_product_schedule_matches_budget_rule():
