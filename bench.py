@@ -399,7 +399,7 @@ def paper_protocol_line(args, rep, dev):
     return line
 
 
-def per_operation(table, tensor_ops, peaks):
+def per_operation(table, tensor_ops, peaks, wname=None):
     """Every operation of one instrumented prefill against the roofline that bounds it: algorithmic FLOPs (tensor-core
     operations) or bytes (the rest) over the CUDA-event time summed over the layers, as a fraction of the measured peak
     (sustained cuBLAS bf16 TFLOP/s, copy GB/s)."""
@@ -416,6 +416,8 @@ def per_operation(table, tensor_ops, peaks):
             ach = v["bytes"] / sec / 1e9
             out[k] = {"ms": round(v["ms"], 3), "calls": v["calls"], "bound": "hbm", "achieved_gbs": round(ach, 1),
                       "frac_of_measured_peak": round(ach / bw_peak, 3)}
+        if (wname, k) in NCU_TRAFFIC_BYTES:      # DRAM bytes of one launch at the first-stage shape (ncu capture)
+            out[k]["dram_traffic_stage0_launch"] = NCU_TRAFFIC_BYTES[(wname, k)]
     return out
 
 
@@ -570,7 +572,7 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
             "algorithmic_tflop_per_step": total_flops / 1e12,
             "achieved_tflops_whole_step": total_flops / 1e12 / (ms_step * 1e-3),
             "breakdown_ms": {k: round(v["ms"], 3) for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"])},
-            "per_operation": per_operation(table, tensor_ops, peaks),
+            "per_operation": per_operation(table, tensor_ops, peaks, wname),
         }
         if args.breakdown:
             for k, v in sorted(table.items(), key=lambda kv: -kv[1]["ms"]):
