@@ -122,6 +122,17 @@ typedef struct {
   int32_t prune_to;
 } spts_layer_plan;
 
+/* One stage of the MSDP schedule (Section 3.4; the settings of Section 4.1 are given in this form): the last
+ * layer of the stage (0-indexed), the fixed active budgets M_fixed of its attention and FFN blocks (<= 0: that
+ * block runs on every candidate in this stage) and the candidate count N_{s+1} the stage end prunes to by
+ * Eq. 16 (<= 0: the stage end does not prune). */
+typedef struct {
+  int32_t last_layer;
+  int32_t m_attn_fixed;
+  int32_t m_ffn_fixed;
+  int32_t n_next;
+} spts_msdp_stage;
+
 typedef struct {
   const spts_layer_weights* layers; /* host array [n_layers] */
   const void* lm_head;              /* [vocab, D] */
@@ -266,6 +277,19 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
                               const int32_t* orig_in, const float* S_mha, int N, int n_next,
                               uint32_t flags, void* X_out, int32_t* pos_out, int32_t* orig_out,
                               int32_t* idx_out);
+
+/* The budget rule of Multi-Stage Delayed Pruning (Section 3.4: M^l = min(|T^l|, M^l_fixed); Algorithm 1's
+ * "M <- min(N, M_fix)" lines and the candidate update of Eq. 16), evaluated on the host: fills plan_out [n_layers]
+ * (HOST memory) for a prompt of n_prompt tokens.  `stages` [n_stages] (HOST memory) is ordered by last_layer;
+ * layer l belongs to the first stage whose last_layer >= l, layers after the last boundary to the last stage (they
+ * keep its budgets).  Layers before `skip_from` run densely (m_attn = m_ffn = current candidate count) as the
+ * paper's shallow layers do.  A stage's last layer gets prune_to = n_next when that is positive and smaller than
+ * the current candidate count, and the later layers see that many candidates.  Optional outputs (host):
+ * *n_final = candidates left after the last layer; *kv_token_layers = sum of m_attn over the layers, the number
+ * of (token, layer) pairs the prefill leaves in the KV caches.  Pure host arithmetic: needs no context and no GPU.
+ * Errors: SPTS_ERR_INVALID_ARG for null pointers, n_layers / n_prompt / n_stages < 1, stages out of order. */
+spts_status spts_msdp_plan(int n_layers, int n_prompt, int skip_from, const spts_msdp_stage* stages, int n_stages,
+                           spts_layer_plan* plan_out, int32_t* n_final, int64_t* kv_token_layers);
 
 /* Offline construction of the low-rank proxy FFN of one layer (Section 3.3, "Low-rank Proxy FFN"):
  *   z(x) = |silu(x W_gate) * (x W_up)| for every calibration token x (rows of calib [n_cal, D], the hidden states

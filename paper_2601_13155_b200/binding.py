@@ -55,6 +55,11 @@ class LayerPlanC(C.Structure):
     _fields_ = [("m_attn", C.c_int32), ("m_ffn", C.c_int32), ("prune_to", C.c_int32)]
 
 
+class MsdpStageC(C.Structure):
+    _fields_ = [("last_layer", C.c_int32), ("m_attn_fixed", C.c_int32), ("m_ffn_fixed", C.c_int32),
+                ("n_next", C.c_int32)]
+
+
 class ModelWeightsC(C.Structure):
     _fields_ = [("layers", C.POINTER(LayerWeightsC)), ("lm_head", C.c_void_p), ("embed", C.c_void_p)]
 
@@ -64,7 +69,7 @@ EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_opti
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
            "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
            "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build",
-           "spts_layer_prefill_skip_batch")
+           "spts_layer_prefill_skip_batch", "spts_msdp_plan")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -101,6 +106,8 @@ def load_library() -> C.CDLL:
                                                   C.POINTER(C.c_int32), C.POINTER(C.c_int32), u32,
                                                   C.POINTER(KvLayerC), vp, vp, vp]
     lib.spts_msdp_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, vp, vp, vp, vp]
+    lib.spts_msdp_plan.argtypes = [i32, i32, i32, C.POINTER(MsdpStageC), i32, C.POINTER(LayerPlanC),
+                                   C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
     lib.spts_first_token.argtypes = [vp, vp, vp, vp, vp]
     lib.spts_prefill.argtypes = [vp, C.POINTER(ModelWeightsC), C.POINTER(LayerPlanC), vp, vp, vp, vp, vp, vp,
                                  i32, u32, C.POINTER(KvLayerC), C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
@@ -302,7 +309,7 @@ class Spts:
         self._check(self.lib.spts_layer_prefill_skip_batch(self.h, C.byref(w.c), _ptr(X), _ptr(pos), n_seq,
                                                            arr(seq_start), arr(m_attn), arr(m_ffn), flags, caches.c,
                                                            _ptr(S_out), _ptr(idx_attn_out), _ptr(idx_ffn_out)),
-                    "spts_layer_prefill_skip_batch")
+                    "spts_layer_prefill_skip_batch", "spts_msdp_plan")
 
     def msdp_compact(self, X_in, pos_in, orig_in, S_mha, n_next: int, X_out, pos_out, orig_out, idx_out=None,
                      flags: int = FORCE_LAST):

@@ -638,6 +638,30 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
   return SPTS_OK;
 }
 
+spts_status spts_msdp_plan(int n_layers, int n_prompt, int skip_from, const spts_msdp_stage* stages, int n_stages,
+                           spts_layer_plan* plan_out, int32_t* n_final, int64_t* kv_token_layers) {
+  if (stages == nullptr || plan_out == nullptr || n_layers < 1 || n_prompt < 1 || n_stages < 1) return SPTS_ERR_INVALID_ARG;
+  for (int s = 1; s < n_stages; ++s)
+    if (stages[s].last_layer <= stages[s - 1].last_layer) return SPTS_ERR_INVALID_ARG;
+  int cur = n_prompt, s = 0;
+  int64_t kv = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    while (s + 1 < n_stages && stages[s].last_layer < l) ++s;
+    const spts_msdp_stage& st = stages[s];
+    spts_layer_plan p;
+    const bool skip = l >= skip_from;
+    p.m_attn = (skip && st.m_attn_fixed > 0 && st.m_attn_fixed < cur) ? st.m_attn_fixed : cur;   // M^l = min(|T^l|, M_fixed)
+    p.m_ffn = (skip && st.m_ffn_fixed > 0 && st.m_ffn_fixed < cur) ? st.m_ffn_fixed : cur;
+    p.prune_to = (l == st.last_layer && st.n_next > 0 && st.n_next < cur) ? st.n_next : 0;       // |T^{l+1}| of Eq. 16
+    plan_out[l] = p;
+    kv += p.m_attn;
+    if (p.prune_to) cur = p.prune_to;
+  }
+  if (n_final) *n_final = cur;
+  if (kv_token_layers) *kv_token_layers = kv;
+  return SPTS_OK;
+}
+
 namespace {
 constexpr int PROXY_SWEEPS = 14;
 struct ProxyScratch {

@@ -6,30 +6,32 @@ import math
 from typing import List, Sequence, Tuple
 
 
+def _msdp_plan(n_layers: int, n_prompt: int, skip_from: int, stages) -> List[Tuple[int, int, int]]:
+    """spts_msdp_plan (the budget rule lives in the library, on the host side of the C boundary):
+    stages = [(last_layer, m_attn_fixed, m_ffn_fixed, n_next)]."""
+    import ctypes as C
+    from . import binding
+    lib = binding.load_library()
+    st = (binding.MsdpStageC * len(stages))(*[binding.MsdpStageC(*[int(v) for v in t]) for t in stages])
+    out = (binding.LayerPlanC * n_layers)()
+    code = lib.spts_msdp_plan(n_layers, n_prompt, skip_from, st, len(stages), out, None, None)
+    if code != 0:
+        raise binding.SptsError(code, "spts_msdp_plan")
+    return [(int(p.m_attn), int(p.m_ffn), int(p.prune_to)) for p in out]
+
+
 def stage_plan(n_layers: int, n_prompt: int, stage_first_layer: Sequence[int], stage_tokens: Sequence[int],
                m_attn_fixed, m_ffn_fixed, skip_from: int = 0) -> List[Tuple[int, int, int]]:
     """Returns [(m_attn, m_ffn, prune_to)] per layer; prune_to == 0 when the layer does not end a stage.
 
-    stage_tokens[s] is the candidate count N_s of stage s; the budgets are a single value or one per stage.
-    Layers before `skip_from` run densely."""
+    stage_tokens[s] is the candidate count N_s of stage s (N_0 is the prompt length); the budgets are a single value
+    or one per stage.  Layers before `skip_from` run densely."""
     ns = len(stage_first_layer)
     ma = list(m_attn_fixed) if hasattr(m_attn_fixed, "__len__") else [m_attn_fixed] * ns
     mf = list(m_ffn_fixed) if hasattr(m_ffn_fixed, "__len__") else [m_ffn_fixed] * ns
-    cur = n_prompt
-    out = []
-    for l in range(n_layers):
-        s = max(i for i in range(ns) if stage_first_layer[i] <= l)
-        if l == stage_first_layer[s]:
-            cur = min(cur, stage_tokens[s])
-        ends = s + 1 < ns and l + 1 == stage_first_layer[s + 1]
-        nxt = min(cur, stage_tokens[s + 1]) if ends else 0
-        if l >= skip_from:
-            out.append((min(cur, ma[s]), min(cur, mf[s]), nxt))
-        else:
-            out.append((cur, cur, nxt))
-        if ends:
-            cur = nxt
-    return out
+    stages = [(stage_first_layer[s + 1] - 1 if s + 1 < ns else n_layers - 1, ma[s], mf[s],
+               stage_tokens[s + 1] if s + 1 < ns else 0) for s in range(ns)]
+    return _msdp_plan(n_layers, min(n_prompt, stage_tokens[0]), skip_from, stages)
 
 
 def workload_plan(w, keep_attn=None, keep_ffn=None, dense: bool = False):
@@ -62,23 +64,17 @@ def paper_plan(model: str, n_prompt: int, ltp: bool = True, msdp: bool = True):
     ltp=False leaves the FFN dense (the "PAP only" row of the paper's component ablation, Table 2);
     msdp=False keeps every token a candidate in every layer (budgets unchanged, no pruning)."""
     n_layers, skip_from, ends, budgets_ki, prune_ki = PAPER_SCHEDULES[model]
-    ki = 1024
-    budgets = tuple(b * ki for b in budgets_ki)
-    cur = n_prompt
-    out = []
-    for l in range(n_layers):
-        if l < skip_from:
-            out.append((cur, cur, 0))
-            continue
-        s = next((i for i, e in enumerate(ends) if l <= e), len(ends) - 1)
-        m = min(cur, budgets[s])
-        nxt = 0
-        if msdp and l in ends:
-            nxt = min(cur, budgets[ends.index(l)] - prune_ki * ki)
-        out.append((m, m if ltp else cur, nxt if nxt < cur else 0))
-        if nxt and nxt < cur:
-            cur = nxt
-    return out
+    return scaled_paper_plan(n_layers, n_prompt, skip_from, ends, [b * 1024 for b in budgets_ki], prune_ki * 1024,
+                             ltp=ltp, msdp=msdp)
+
+
+def scaled_paper_plan(n_layers: int, n_prompt: int, skip_from: int, ends: Sequence[int], budgets: Sequence[int],
+                      prune_below: int, ltp: bool = True, msdp: bool = True):
+    """A schedule of the paper's form with every number given in tokens: dense layers before `skip_from`, stage s
+    ends after layer ends[s] with active budget budgets[s] and prunes the candidates to budgets[s] - prune_below;
+    the layers after the last boundary keep the last budget."""
+    stages = [(e, b, b if ltp else 0, b - prune_below if msdp else 0) for e, b in zip(ends, budgets)]
+    return _msdp_plan(n_layers, n_prompt, skip_from, stages)
 
 
 def paper_llama_plan(n_prompt: int, n_layers: int = 32, ltp: bool = True, msdp: bool = True):

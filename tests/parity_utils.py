@@ -47,6 +47,22 @@ def check_index_set(got_idx, oracle_scores, k, force_last=True, band=1e-3):
     return len(diff) // 2
 
 
+def index_set_report(got_idx, oracle_scores, k, force_last=True, band=1e-3):
+    """Measures, without asserting, how a selected set differs from the oracle's: `diff` = tokens of the oracle's set
+    that are missing (= tokens selected instead), `outside_band` = how many of the differing tokens (both sides) have
+    an oracle score farther than `band` (relative) from the k-th score, `max_rel_dist` = the farthest of them."""
+    got = np.asarray(got_idx, np.int64)
+    assert got.shape[0] == k and np.all(np.diff(got) > 0)
+    s = np.asarray(oracle_scores, np.float64)
+    want = O.topk_select(s, k, force_last)
+    body = want[want != len(s) - 1] if force_last and k > 1 else want
+    kth = np.sort(s[body])[0]
+    diff = np.setxor1d(got, want)
+    dist = np.abs(s[diff] - kth) / abs(kth) if len(diff) else np.zeros(0)
+    return {"diff": len(diff) // 2, "outside_band": int((dist > band).sum()),
+            "max_rel_dist": float(dist.max()) if len(diff) else 0.0}
+
+
 TOL = {"bf16": 2e-2, "fp32": 1e-4}
 
 
@@ -57,25 +73,46 @@ def bf16_ulp(x):
     return 2.0 ** (e - 7)
 
 
-def check_output(got, want, dtype, scale=1.0):
+class OutputStats(dict):
+    """What check_output measured: max_rel (largest error outside the tolerated one-ulp cases, relative to the RMS),
+    worst_rel (largest error of all), flips (elements beyond the tolerance that are exactly a one-ulp disagreement),
+    flip_rows (the rows they sit in, at most 16 listed), elements."""
+
+
+REPORT = []          # one entry per check_output call of the running test; printed by the conftest hook
+
+
+def check_output(got, want, dtype, scale=1.0, what="output"):
     """Layer outputs: max-abs error <= tol * RMS(want).  In bf16 storage a single element whose
     fp32-accumulated value and fp64 value fall on different sides of a rounding boundary differs by
     one bf16 ulp, which for the large entries of heavy rows exceeds tol * RMS on its own; such
-    elements are allowed one ulp and must be rare (< 0.1 % of the elements)."""
+    elements are allowed one ulp and must be rare (< 0.1 % of the elements).  Returns OutputStats (the number and
+    the rows of the tolerated one-ulp cases among them) and appends them to REPORT, which every GPU test prints."""
     got = np.asarray(got, np.float64)
     want = np.asarray(want, np.float64)
     tol = TOL[dtype] * scale
     rms = max(np.sqrt(np.mean(want ** 2)), 1e-30)
     err = np.abs(got - want)
     over = err > tol * rms
+    stats = OutputStats(what=what, elements=int(want.size), tol=tol, worst_rel=float(err.max() / rms) if err.size else 0.0,
+                        flips=0, flip_rows=[], max_rel=0.0)
     if dtype == "fp32":
         assert not over.any(), f"max-abs error {err.max() / rms:.3e} of RMS exceeds {tol:.1e}"
-        return float(err.max() / rms)
+        stats["max_rel"] = stats["worst_rel"]
+        REPORT.append(stats)
+        return stats
     flips = over & (err <= 1.001 * bf16_ulp(want))
     bad = over & ~flips
     assert not bad.any(), f"max-abs error {err[bad].max() / rms:.3e} of RMS exceeds {tol:.1e} (beyond one bf16 ulp)"
     assert flips.sum() <= max(1, 1e-3 * want.size), f"{int(flips.sum())} one-ulp disagreements"
-    return float(err[~over].max() / rms) if (~over).any() else 0.0
+    stats["flips"] = int(flips.sum())
+    if stats["flips"]:
+        rows = np.unique(np.nonzero(flips)[0]) if flips.ndim > 1 else np.nonzero(flips)[0]
+        stats["flip_rows"] = [int(r) for r in rows[:16]]
+        stats["n_flip_rows"] = int(len(rows))
+    stats["max_rel"] = float(err[~over].max() / rms) if (~over).any() else 0.0
+    REPORT.append(stats)
+    return stats
 
 
 def zero_down(W):

@@ -97,3 +97,32 @@ def test_paper_llama_plan_matches_oracle_and_table3():
     assert p[20] == (4096, 6144, 0)                                  # 6144 candidates left after two prunes
     p = schedule.paper_llama_plan(32768, msdp=False)
     assert all(c == 0 for _, _, c in p) and p[31] == (2048, 2048, 0) and p[12] == (9216, 9216, 0)
+
+
+def test_msdp_plan_call_counts_and_errors():
+    """spts_msdp_plan through the C boundary: the optional outputs (final candidate count, cached token-layer pairs:
+    the paper's LLaMA setting at 32 Ki tokens gives the 6.63 of Table 3 in units of 64 Ki pairs) and the host
+    errors (null pointers, empty inputs, stages out of order)."""
+    import ctypes as C
+    from paper_2601_13155_b200 import binding
+    lib = binding.load_library()
+    Ki = 1024
+    st = (binding.MsdpStageC * 4)(*[binding.MsdpStageC(e, b * Ki, b * Ki, (b - 1) * Ki)
+                                    for e, b in zip((13, 18, 23, 28), (9, 7, 4, 2))])
+    out = (binding.LayerPlanC * 32)()
+    nf, kv = C.c_int32(0), C.c_int64(0)
+    assert lib.spts_msdp_plan(32, 32 * Ki, 10, st, 4, out, C.byref(nf), C.byref(kv)) == 0
+    assert nf.value == 1 * Ki and f"{kv.value / Ki / 64 + 1e-9:.2f}" == "6.63"     # 6.625 exactly
+    assert [(out[l].m_attn, out[l].m_ffn, out[l].prune_to) for l in (0, 9, 10, 13, 14, 28, 29, 31)] == [
+        (32 * Ki, 32 * Ki, 0), (32 * Ki, 32 * Ki, 0), (9 * Ki, 9 * Ki, 0), (9 * Ki, 9 * Ki, 8 * Ki),
+        (7 * Ki, 7 * Ki, 0), (2 * Ki, 2 * Ki, 1 * Ki), (1 * Ki, 1 * Ki, 0), (1 * Ki, 1 * Ki, 0)]
+    # a prompt shorter than every budget: nothing is skipped, nothing is pruned
+    assert lib.spts_msdp_plan(32, 700, 10, st, 4, out, C.byref(nf), None) == 0
+    assert nf.value == 700 and all((out[l].m_attn, out[l].m_ffn, out[l].prune_to) == (700, 700, 0) for l in range(32))
+    assert lib.spts_msdp_plan(32, 32 * Ki, 10, None, 4, out, None, None) == 1
+    assert lib.spts_msdp_plan(32, 32 * Ki, 10, st, 4, None, None, None) == 1
+    assert lib.spts_msdp_plan(0, 32 * Ki, 10, st, 4, out, None, None) == 1
+    assert lib.spts_msdp_plan(32, 0, 10, st, 4, out, None, None) == 1
+    assert lib.spts_msdp_plan(32, 32 * Ki, 10, st, 0, out, None, None) == 1
+    bad = (binding.MsdpStageC * 2)(binding.MsdpStageC(5, 8, 8, 4), binding.MsdpStageC(5, 4, 4, 2))
+    assert lib.spts_msdp_plan(8, 100, 0, bad, 2, out, None, None) == 1
