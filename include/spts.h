@@ -53,7 +53,8 @@ typedef enum {
   SPTS_ERR_CUDA = 4,
   SPTS_ERR_TIMEOUT = 5,
   SPTS_ERR_NONFINITE = 6,
-  SPTS_ERR_UNSUPPORTED = 7
+  SPTS_ERR_UNSUPPORTED = 7,
+  SPTS_ERR_INDEX = 8      /* SPTS_DEBUG_CHECKS: an index list was out of range or not strictly ascending */
 } spts_status;
 
 enum { SPTS_BF16 = 0, SPTS_FP32 = 1 };
@@ -67,6 +68,9 @@ enum {
                                   Appendix C: every query attends causally, K and the queries are taken as stored) */
   SPTS_ATTENTION_ONE_TILE = 4u, /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
                                   slower kernel kept as a cross-check of the two-tile kernel) */
+  SPTS_DEBUG_CHECKS = 32u,     /* spts_set_option: after every selection a small kernel checks the index list
+                                  (0 <= idx < N, strictly ascending) and records SPTS_ERR_INDEX in the device status
+                                  word; nothing traps.  Off by default (one extra launch per selection) */
   SPTS_FFN_SCORE_PAP_ONLY = 16u /* spts_set_option: T_f = TopK(S_mha, m_ffn) -- the FFN block selects by the attention
                                   probe's score alone (Eq. 4) and the proxy FFN of Eq. 12-14 is not evaluated: the
                                   criterion the paper's proxy-network ablation (Table 4) compares Eq. 14 against */
@@ -173,11 +177,32 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
                         size_t workspace_bytes, void* cuda_stream, spts_ctx** out);
 void spts_destroy(spts_ctx* ctx);
 
-/* Sets SPTS_REFERENCE_KERNELS or SPTS_ATTENTION_ONE_TILE on/off (value 0/1), or SPTS_PAP_WINDOW (value 1..64). */
+/* Sets SPTS_REFERENCE_KERNELS, SPTS_ATTENTION_ONE_TILE, SPTS_FFN_SCORE_PAP_ONLY or SPTS_DEBUG_CHECKS on/off
+ * (value 0/1), or SPTS_PAP_WINDOW (value 1..64). */
 spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value);
 
 /* Synchronises the context's stream and returns the device status word (then clears it). */
 spts_status spts_last_device_status(spts_ctx* ctx);
+
+/* Guard bands (the paper has no counterpart: a stand-in for a memory checker).  Every slice the library carves out
+ * of the caller's workspace is followed by a 256-byte band that spts_create() fills with a fixed pattern and no
+ * kernel has any business writing.  spts_check_guards synchronises the stream, reads the bands back and stores the
+ * number of bands that no longer hold the pattern in *n_corrupt (HOST memory); a non-zero count means some kernel
+ * wrote past the end of its slice. */
+spts_status spts_check_guards(spts_ctx* ctx, int32_t* n_corrupt);
+
+/* The check SPTS_DEBUG_CHECKS runs after every selection, on a list the caller provides: idx [n] (device) must lie
+ * in [0, N) and ascend strictly, otherwise SPTS_ERR_INDEX is recorded in the device status word (read it with
+ * spts_last_device_status).  The kernel only reads the n entries; it never dereferences them. */
+spts_status spts_debug_check_index_list(spts_ctx* ctx, const int32_t* idx, int n, int N);
+
+/* Exercises the give-up path of the bounded waits (again no counterpart in the paper).  Every mbarrier wait of the
+ * tensor-core kernels ends after a time limit: the waiting thread raises a CTA-wide flag, the other roles see it
+ * and return from their own waits, the CTA lets copies in flight land, records SPTS_ERR_TIMEOUT in the device
+ * status word and exits normally.  This call launches one tiny CTA that runs exactly that code on two barriers
+ * nobody ever arrives on, with the limit shortened to limit_us microseconds (1..100000), so a test can see the
+ * status come back and the context stay usable.  The production kernels are not involved. */
+spts_status spts_selftest_wait_timeout(spts_ctx* ctx, uint32_t limit_us);
 
 /* Number of kernels the library has launched on this context so far. */
 int64_t spts_launch_count(const spts_ctx* ctx);
@@ -250,6 +275,15 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
                                     const int32_t* pos, int N, int m_attn, int m_ffn,
                                     uint32_t flags, spts_kv_layer* cache, float* S_mha_out,
                                     int32_t* idx_attn_out, int32_t* idx_ffn_out);
+
+/* The attention step of the reduced MHA on its own (Algorithm 1: O^ <- F_MHA(Q^, K^, V^), before W_O): causal
+ * grouped-query attention among m rows in their compact order, row i attending to rows j <= i,
+ *   O[i, h] = softmax_j(Q[i, h] . K[j, h / (H/Hkv)] / sqrt(d)) V[j, h / (H/Hkv)].
+ * Q [m, H, d] and K [m, Hkv, d] are taken as given (after RoPE), V [m, Hkv, d]; O_out [m, H*d]; all in the storage
+ * type, 16-byte aligned, none aliasing another.  1 <= m <= max_seq.  This is the kernel spts_layer_prefill_skip
+ * runs between the Q/V projections and the O projection; the call exists so that it can be checked and timed on
+ * operands of the caller's choosing. */
+spts_status spts_reduced_attention(spts_ctx* ctx, const void* Q, const void* K, const void* V, int m, void* O_out);
 
 /* The same layer for several independent prompts packed row after row into X [total, D] (the paper evaluates one
  * prompt at a time; Algorithm 1 applies to each prompt on its own, and that is what this call computes):

@@ -22,9 +22,10 @@ OPT_REFERENCE_KERNELS = 2
 OPT_ATTENTION_ONE_TILE = 4
 OPT_PAP_WINDOW = 8
 OPT_FFN_SCORE_PAP_ONLY = 16
+OPT_DEBUG_CHECKS = 32
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "WORKSPACE", 4: "CUDA", 5: "TIMEOUT",
-                6: "NONFINITE", 7: "UNSUPPORTED"}
+                6: "NONFINITE", 7: "UNSUPPORTED", 8: "INDEX"}
 
 
 class SptsError(RuntimeError):
@@ -69,7 +70,8 @@ EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_opti
            "spts_ltp_score", "spts_topk_select", "spts_layer_prefill_skip", "spts_msdp_compact",
            "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
            "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build",
-           "spts_layer_prefill_skip_batch", "spts_msdp_plan")
+           "spts_layer_prefill_skip_batch", "spts_msdp_plan", "spts_check_guards", "spts_selftest_wait_timeout",
+           "spts_debug_check_index_list", "spts_reduced_attention")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -108,6 +110,10 @@ def load_library() -> C.CDLL:
     lib.spts_msdp_compact.argtypes = [vp, vp, vp, vp, vp, i32, i32, u32, vp, vp, vp, vp]
     lib.spts_msdp_plan.argtypes = [i32, i32, i32, C.POINTER(MsdpStageC), i32, C.POINTER(LayerPlanC),
                                    C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+    lib.spts_check_guards.argtypes = [vp, C.POINTER(C.c_int32)]
+    lib.spts_selftest_wait_timeout.argtypes = [vp, u32]
+    lib.spts_debug_check_index_list.argtypes = [vp, vp, i32, i32]
+    lib.spts_reduced_attention.argtypes = [vp, vp, vp, vp, i32, vp]
     lib.spts_first_token.argtypes = [vp, vp, vp, vp, vp]
     lib.spts_prefill.argtypes = [vp, C.POINTER(ModelWeightsC), C.POINTER(LayerPlanC), vp, vp, vp, vp, vp, vp,
                                  i32, u32, C.POINTER(KvLayerC), C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
@@ -245,6 +251,22 @@ class Spts:
     def set_attention_one_tile(self, on: bool):
         self._check(self.lib.spts_set_option(self.h, OPT_ATTENTION_ONE_TILE, 1 if on else 0), "spts_set_option")
 
+    def set_debug_checks(self, on: bool):
+        """Every selected index list is checked on the device (range, strictly ascending); SPTS_ERR_INDEX otherwise."""
+        self._check(self.lib.spts_set_option(self.h, OPT_DEBUG_CHECKS, 1 if on else 0), "spts_set_option")
+
+    def check_guards(self) -> int:
+        """Number of guard bands between the workspace slices that no longer hold their pattern (0 = intact)."""
+        n = C.c_int32(-1)
+        self._check(self.lib.spts_check_guards(self.h, C.byref(n)), "spts_check_guards")
+        return int(n.value)
+
+    def debug_check_index_list(self, idx, N: int):
+        self._check(self.lib.spts_debug_check_index_list(self.h, _ptr(idx), idx.shape[0], N), "spts_debug_check_index_list")
+
+    def selftest_wait_timeout(self, limit_us: int = 1000):
+        self._check(self.lib.spts_selftest_wait_timeout(self.h, int(limit_us)), "spts_selftest_wait_timeout")
+
     def device_status(self) -> int:
         return int(self.lib.spts_last_device_status(self.h))
 
@@ -300,6 +322,15 @@ class Spts:
                                                      _ptr(idx_attn_out), _ptr(idx_ffn_out)),
                     "spts_layer_prefill_skip")
 
+    def reduced_attention(self, Q, K, V, O_out=None):
+        """spts_reduced_attention: causal GQA attention among the m rows of Q [m,H,d], K, V [m,Hkv,d] -> [m, H*d]."""
+        m = Q.shape[0]
+        if O_out is None:
+            O_out = torch.empty(m, self.shape.n_q_heads * self.shape.head_dim, dtype=self.dtype, device=self.device)
+        self._check(self.lib.spts_reduced_attention(self.h, _ptr(Q), _ptr(K), _ptr(V), m, _ptr(O_out)),
+                    "spts_reduced_attention")
+        return O_out
+
     def layer_prefill_skip_batch(self, w: LayerWeights, X, pos, seq_start, m_attn, m_ffn, caches: KvCache,
                                  flags: int = FORCE_LAST, S_out=None, idx_attn_out=None, idx_ffn_out=None):
         """Several prompts packed into X; `caches` holds one entry per sequence (a KvCache built with
@@ -309,7 +340,8 @@ class Spts:
         self._check(self.lib.spts_layer_prefill_skip_batch(self.h, C.byref(w.c), _ptr(X), _ptr(pos), n_seq,
                                                            arr(seq_start), arr(m_attn), arr(m_ffn), flags, caches.c,
                                                            _ptr(S_out), _ptr(idx_attn_out), _ptr(idx_ffn_out)),
-                    "spts_layer_prefill_skip_batch", "spts_msdp_plan")
+                    "spts_layer_prefill_skip_batch", "spts_msdp_plan", "spts_check_guards", "spts_selftest_wait_timeout",
+           "spts_debug_check_index_list", "spts_reduced_attention")
 
     def msdp_compact(self, X_in, pos_in, orig_in, S_mha, n_next: int, X_out, pos_out, orig_out, idx_out=None,
                      flags: int = FORCE_LAST):

@@ -692,8 +692,7 @@ spts_status decode_layer_t(spts_ctx* ctx, const spts_layer_weights* w, spts_kv_l
   LAUNCH_DEP(ctx, dec_qkv_kernel<T>, dim3(qkv_blocks), dim3(GV_THREADS), st, (const T*)w->wq, (const T*)w->wk,
              (const T*)w->wv, H, Hkv, hd, D, (const float*)x32, d.rms_eps, (int)pos, (double)d.rope_theta, q32,
              (T*)cache->k, (T*)cache->v, cache->pos, slot);
-  cache->len = slot + 1;
-  const int len = cache->len;
+  const int len = slot + 1;                  // the host-side cache->len is advanced by the caller once the whole step is enqueued
   int nsplit = min(DEC_MAX_SPLIT, max(1, len / 128));
   if (std::is_same<T, bf16>::value)      // the tensor-core kernel holds three blocks per SM: keep the slices to one wave
     nsplit = max(1, min(nsplit, 3 * ctx->sm_count / (Hkv * ceil_div(H / Hkv, 16))));

@@ -326,6 +326,30 @@ spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld
   return SPTS_OK;
 }
 
+// out_t[c, r] = in[r, c] for a bf16 matrix [rows, cols] (row stride cols) into [cols, ldt]: the transposed copy of V
+// the tensor-core attention reads, for values that did not come out of the library's own V projection.
+__global__ void transpose_bf16_kernel(const bf16* __restrict__ in, int rows, int cols, bf16* __restrict__ out_t, int ldt) {
+  __shared__ bf16 tile[32][33];
+  const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int r = r0 + i, c = c0 + threadIdx.x;
+    if (r < rows && c < cols) tile[i][threadIdx.x] = in[(size_t)r * cols + c];
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int c = c0 + i, r = r0 + threadIdx.x;
+    if (r < rows && c < cols) out_t[(size_t)c * ldt + r] = tile[threadIdx.x][i];
+  }
+}
+
+spts_status launch_transpose_bf16(spts_ctx* ctx, const void* in, int rows, int cols, void* out_t, int ldt) {
+  if (rows <= 0 || cols <= 0) return SPTS_OK;
+  transpose_bf16_kernel<<<dim3(ceil_div(cols, 32), ceil_div(rows, 32)), dim3(32, 8), 0, ctx->stream>>>(
+      (const bf16*)in, rows, cols, (bf16*)out_t, ldt);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
 spts_status launch_pap_regroup(spts_ctx* ctx, const void* q_win, int w, void* q_kv) {
   const auto& d = ctx->desc;
   const int G = d.n_q_heads / d.n_kv_heads;

@@ -328,6 +328,23 @@ spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offs
   return SPTS_OK;
 }
 
+// SPTS_DEBUG_CHECKS: an index list must lie in [0, N) and ascend strictly; a violation is recorded, never trapped on
+__global__ void check_index_list_kernel(const int32_t* __restrict__ idx, int n, int N, int* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int v = idx[i];
+  bool bad = v < 0 || v >= N;
+  if (i > 0 && idx[i - 1] >= v) bad = true;
+  if (bad) set_status(status, SPTS_ERR_INDEX);
+}
+
+spts_status launch_check_index_list(spts_ctx* ctx, const int32_t* idx, int n, int N) {
+  if (n == 0) return SPTS_OK;
+  check_index_list_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(idx, n, N, ctx->ws.status);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
 spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst) {
   if (n == 0) return SPTS_OK;
   gather_i32_kernel<<<ceil_div(n, 256), 256, 0, ctx->stream>>>(src, idx, n, dst);

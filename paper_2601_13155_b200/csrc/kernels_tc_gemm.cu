@@ -388,6 +388,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     dots[hh][g] = d;
                   }
                 }
+                // query heads beyond the eight kept in registers (GQA groups larger than 8): their partial sums
+                // over this half of the frequencies go through the logits row itself (same thread, same address)
+                for (int g = 8; g < p.group; ++g) {
+                  const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
+                  float d = 0.f;
+#pragma unroll
+                  for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
+                  float* lp = p.logits + (size_t)(kvh * p.group + g) * p.ld_logits + grow;
+                  *lp = jj == 0 ? d : (*lp + d) * inv_sqrt_d;
+                }
               }
             }
           }
@@ -493,6 +503,36 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   }
 }
 
+// The give-up path of the bounded waits on its own: two roles wait on barriers nobody arrives on.  Warp 0's wait
+// runs into the (shortened) limit and raises the abort flag; warp 1's wait has a limit far away and must return
+// because of the flag.  Then the same teardown as the kernels above: status word, drain delay, normal exit.
+__global__ void __launch_bounds__(64, 1) wait_selftest_kernel(uint64_t limit_ns, int* status, int* observed) {
+  __shared__ __align__(8) uint64_t bar_store[2];
+  __shared__ int abort_store;
+  volatile int* abort_flag = &abort_store;
+  const uint32_t bar0 = smem_u32(&bar_store[0]), bar1 = smem_u32(&bar_store[1]);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint64_t t0 = globaltimer_ns();
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    mbar_init(bar0, 1);
+    mbar_init(bar1, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (lane == 0) {
+    const bool ok = warp == 0 ? mbar_wait(bar0, 0, abort_flag, t0, limit_ns) : mbar_wait(bar1, 0, abort_flag, t0);
+    observed[warp] = ok ? 1 : 2;            // 2 = the wait was abandoned
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) set_status(status, SPTS_ERR_TIMEOUT);
+    const uint64_t t1 = globaltimer_ns();
+    while (globaltimer_ns() - t1 < 200000ull) { }
+    __syncthreads();
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -578,6 +618,13 @@ bool set_smem_attr() {
 }  // namespace
 
 int tc_sumsq_parts(int n_out) { return ceil_div(n_out, 256); }
+
+spts_status launch_wait_selftest(spts_ctx* ctx, uint32_t limit_us) {
+  // observed[] lives behind the status word: ws.status has 64 ints, the first is the status itself
+  wait_selftest_kernel<<<1, 64, 0, ctx->stream>>>((uint64_t)limit_us * 1000ull, ctx->ws.status, ctx->ws.status + 8);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
 
 spts_status tc_gemm_init(spts_ctx* ctx) {
   void* fn = nullptr;

@@ -12,13 +12,17 @@ using namespace spts;
 
 namespace {
 
+// Hands out 256-byte aligned slices; every slice is followed by a guard band (GUARD_BYTES) whose offset is recorded.
 struct Carver {
   char* base;
   size_t off;
+  std::vector<size_t>* guards;
   template <typename T> T* take(size_t count) {
     off = align_up(off, 256);
     T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
-    off += count * sizeof(T);
+    off = align_up(off + count * sizeof(T), 256);
+    if (guards) guards->push_back(off);
+    off += GUARD_BYTES;
     return p;
   }
 };
@@ -42,8 +46,8 @@ bool tc_shape_ok(const spts_model_desc& d) {
          d.ltp_dlow % 64 == 0 && d.ltp_rank % 16 == 0 && (d.n_q_heads * d.head_dim) % 64 == 0;
 }
 
-size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws) {
-  Carver c{reinterpret_cast<char*>(base), 0};
+size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std::vector<size_t>* guards = nullptr) {
+  Carver c{reinterpret_cast<char*>(base), 0, guards};
   Workspace w;
   memset(&w, 0, sizeof(w));
   const size_t es = elt_size(d);
@@ -303,6 +307,7 @@ spts_status attention_block(spts_ctx* ctx, const spts_layer_weights* w, void* X,
   if (sel_a) {
     int32_t* ia = idx_attn_out ? idx_attn_out : ws.idx_a;
     OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_attn, launch_topk(ctx, S, N, m_attn, flags, ia, ws.topk_scratch));
+    if (ctx->debug_checks) TRY(launch_check_index_list(ctx, ia, m_attn, N));
     OP(SPTS_OP_KV_GATHER, 0.0, 2.0 * m_attn * (double)KD * es + 8.0 * m_attn,
        launch_gather_rows(ctx, ws.k_all, ia, m_attn, (int)(KD * es), cache->k));
     OP(SPTS_OP_KV_GATHER, 0.0, 12.0 * m_attn, launch_gather_i32(ctx, pos, ia, m_attn, cache->pos));
@@ -396,16 +401,23 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->rope_pos = nullptr;
   ctx->rope_n = 0;
   ctx->pap_window = 1;
+  ctx->debug_checks = false;
   ctx->prof = new (std::nothrow) Profiler;
-  carve(*desc, max_seq, workspace, &ctx->ws);
+  ctx->ws_base = reinterpret_cast<char*>(workspace);
+  carve(*desc, max_seq, workspace, &ctx->ws, &ctx->guard_offsets);
+  for (size_t off : ctx->guard_offsets)
+    if (cudaMemsetAsync(ctx->ws_base + off, GUARD_PATTERN, GUARD_BYTES, ctx->stream) != cudaSuccess) {
+      spts_destroy(ctx);
+      return SPTS_ERR_CUDA;
+    }
   ctx->reference_kernels = (desc->dtype == SPTS_FP32) || !tc_shape_ok(*desc);
   if (!ctx->reference_kernels) {
     spts_status s = tc_init(ctx);
-    if (s != SPTS_OK) { delete ctx; return s; }
+    if (s != SPTS_OK) { spts_destroy(ctx); return s; }
   }
-  if (cudaMemsetAsync(ctx->ws.status, 0, 64 * sizeof(int), ctx->stream) != cudaSuccess) { delete ctx; return SPTS_ERR_CUDA; }
+  if (cudaMemsetAsync(ctx->ws.status, 0, 64 * sizeof(int), ctx->stream) != cudaSuccess) { spts_destroy(ctx); return SPTS_ERR_CUDA; }
   if (cudaMemsetAsync(ctx->ws.topk_scratch, 0, TOPK_SCRATCH_WORDS * sizeof(uint32_t), ctx->stream) != cudaSuccess) {
-    delete ctx;
+    spts_destroy(ctx);
     return SPTS_ERR_CUDA;
   }
   *out = ctx;
@@ -465,6 +477,10 @@ spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
     ctx->attn_one_tile = value != 0;
     return SPTS_OK;
   }
+  if (option == SPTS_DEBUG_CHECKS) {
+    ctx->debug_checks = value != 0;
+    return SPTS_OK;
+  }
   if (option == SPTS_FFN_SCORE_PAP_ONLY) {
     ctx->ffn_score_pap_only = value != 0;
     return SPTS_OK;
@@ -482,6 +498,34 @@ spts_status spts_last_device_status(spts_ctx* ctx) {
 }
 
 int64_t spts_launch_count(const spts_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+spts_status spts_check_guards(spts_ctx* ctx, int32_t* n_corrupt) {
+  TRY(check_ctx(ctx));
+  if (n_corrupt == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return SPTS_ERR_CUDA;
+  unsigned char band[GUARD_BYTES];
+  int bad = 0;
+  for (size_t off : ctx->guard_offsets) {
+    if (cudaMemcpy(band, ctx->ws_base + off, GUARD_BYTES, cudaMemcpyDeviceToHost) != cudaSuccess) return SPTS_ERR_CUDA;
+    bool intact = true;
+    for (int i = 0; i < GUARD_BYTES; ++i) intact = intact && band[i] == GUARD_PATTERN;
+    bad += intact ? 0 : 1;
+  }
+  *n_corrupt = bad;
+  return SPTS_OK;
+}
+
+spts_status spts_debug_check_index_list(spts_ctx* ctx, const int32_t* idx, int n, int N) {
+  TRY(check_ctx(ctx));
+  if (idx == nullptr || n < 1 || N < 1) return SPTS_ERR_INVALID_ARG;
+  return launch_check_index_list(ctx, idx, n, N);
+}
+
+spts_status spts_selftest_wait_timeout(spts_ctx* ctx, uint32_t limit_us) {
+  TRY(check_ctx(ctx));
+  if (limit_us < 1 || limit_us > 100000) return SPTS_ERR_INVALID_ARG;
+  return launch_wait_selftest(ctx, limit_us);
+}
 
 spts_status spts_fold_norm_gain(spts_ctx* ctx, void* W, const float* g, int out_features, int in_features) {
   TRY(check_ctx(ctx));
@@ -512,7 +556,9 @@ spts_status spts_topk_select(spts_ctx* ctx, const float* scores, int N, int k, u
   TRY(check_ctx(ctx));
   if (scores == nullptr || idx_out == nullptr) return SPTS_ERR_INVALID_ARG;
   if (N < 1 || k < 1 || k > N) return SPTS_ERR_INVALID_ARG;
-  return launch_topk(ctx, scores, N, k, flags, idx_out, ctx->ws.topk_scratch);
+  TRY(launch_topk(ctx, scores, N, k, flags, idx_out, ctx->ws.topk_scratch));
+  if (ctx->debug_checks) TRY(launch_check_index_list(ctx, idx_out, k, N));
+  return SPTS_OK;
 }
 
 spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos, int N,
@@ -550,11 +596,28 @@ spts_status spts_layer_prefill_skip(spts_ctx* ctx, const spts_layer_weights* w, 
       s_ffn = ws.s_ffn;
     }
     OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * m_ffn, launch_topk(ctx, s_ffn, N, m_ffn, flags, jf, ws.topk_scratch));
+    if (ctx->debug_checks) TRY(launch_check_index_list(ctx, jf, m_ffn, N));
     idx_f = jf;
   } else if (idx_ffn_out) {
     TRY(launch_topk(ctx, S, N, N, flags, idx_ffn_out, ws.topk_scratch));
   }
   return ffn_gemms(ctx, w, X, N, idx_f, m_ffn);
+}
+
+spts_status spts_reduced_attention(spts_ctx* ctx, const void* Q, const void* K, const void* V, int m, void* O_out) {
+  TRY(check_ctx(ctx));
+  if (Q == nullptr || K == nullptr || V == nullptr || O_out == nullptr) return SPTS_ERR_INVALID_ARG;
+  if (m < 1 || m > ctx->max_seq) return SPTS_ERR_SHAPE;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O_out)) return SPTS_ERR_INVALID_ARG;
+  const auto& d = ctx->desc;
+  const double Ma = (double)m, HD = (double)d.n_q_heads * d.head_dim, KD = (double)d.n_kv_heads * d.head_dim;
+  ProfScope ps(ctx, SPTS_OP_ATTN, 2.0 * HD * Ma * (Ma + 1.0), (2.0 * Ma * HD + 2.0 * Ma * KD) * (double)elt_size(d));
+  if (!use_tc(ctx)) return launch_ref_attention(ctx, Q, K, V, m, O_out);
+  // the tensor-core kernel reads V through its transposed copy
+  const int ldvt = (int)align_up((size_t)m, 128);
+  TRY(launch_transpose_bf16(ctx, V, m, d.n_kv_heads * d.head_dim, ctx->ws.v_t, ldvt));
+  return launch_tc_attention(ctx, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)ctx->ws.v_t, ldvt, m,
+                             (bf16*)O_out);
 }
 
 spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos,
@@ -615,6 +678,7 @@ spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weight
     }
     off_f += mf;
   }
+  if (ctx->debug_checks && any_sel_f) TRY(launch_check_index_list(ctx, ws.idx_f, off_f, total));
   return ffn_gemms(ctx, w, X, total, any_sel_f ? ws.idx_f : nullptr, off_f);
 }
 
@@ -631,6 +695,7 @@ spts_status spts_msdp_compact(spts_ctx* ctx, const void* X_in, const int32_t* po
   if (!aligned16(X_in) || !aligned16(X_out)) return SPTS_ERR_INVALID_ARG;
   int32_t* idx = idx_out ? idx_out : ctx->ws.idx_p;
   OP(SPTS_OP_TOPK, 0.0, 4.0 * N + 4.0 * n_next, launch_topk(ctx, S_mha, N, n_next, flags, idx, ctx->ws.topk_scratch));
+  if (ctx->debug_checks) TRY(launch_check_index_list(ctx, idx, n_next, N));
   ProfScope ps_c(ctx, SPTS_OP_COMPACT, 0.0, 2.0 * n_next * (double)ctx->desc.hidden * (double)elt_size(ctx->desc) + 28.0 * n_next);
   TRY(launch_gather_rows(ctx, X_in, idx, n_next, (int)(ctx->desc.hidden * elt_size(ctx->desc)), X_out));
   TRY(launch_gather_i32(ctx, pos_in, idx, n_next, pos_out));
@@ -669,7 +734,7 @@ struct ProxyScratch {
   int32_t* order; unsigned int* offdiag;
 };
 size_t carve_proxy(const spts_model_desc& d, int n_cal, void* base, ProxyScratch* out) {
-  Carver c{reinterpret_cast<char*>(base), 0};
+  Carver c{reinterpret_cast<char*>(base), 0, nullptr};
   ProxyScratch p;
   p.ld = (int)align_up((size_t)n_cal, 32);
   p.rstd = c.take<float>((size_t)n_cal);
@@ -816,6 +881,9 @@ spts_status spts_decode_step(spts_ctx* ctx, const spts_model_weights* mw, spts_k
   // the residual is already rounded through the storage type; park it where the head can read it
   void* xo = x_out ? x_out : ctx->ws.xrow;
   TRY(launch_decode_store(ctx, xo));
+  // every layer is enqueued: only now do the caches grow on the host side, so a launch error in the middle of a
+  // step leaves all lengths as they were
+  for (int l = 0; l < d.n_layers; ++l) caches[l].len += 1;
   delete guard_d.p; guard_d.p = nullptr;
   if (logits_out != nullptr || token_out != nullptr) {
     if (mw->lm_head == nullptr) return SPTS_ERR_INVALID_ARG;

@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <vector>
+
 #include "spts.h"
 
 namespace spts {
@@ -93,6 +95,9 @@ struct spts_ctx {
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
   bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
   bool ffn_score_pap_only;   // T_f from S_mha alone (no proxy FFN)
+  bool debug_checks;        // every selected index list is checked on the device (SPTS_ERR_INDEX in the status word)
+  char* ws_base;            // the caller's workspace and the byte offsets of the guard bands that follow its slices
+  std::vector<size_t> guard_offsets;
   // set by spts_prefill between two layers: ws.rstd is current for the rows of rstd_x [rstd_n] except the listed ones
   const int32_t* rstd_rows; int rstd_nrows; const void* rstd_x; int rstd_n;
   // rotary table reuse inside spts_prefill: positions only change at a stage end, so the table computed for
@@ -123,6 +128,11 @@ spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* id
                                int row_bytes, void* dst);
 spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst);
 spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offset, int32_t* dst);
+spts_status launch_check_index_list(spts_ctx* ctx, const int32_t* idx, int n, int N);   // debug option only
+spts_status launch_wait_selftest(spts_ctx* ctx, uint32_t limit_us);
+
+static const int GUARD_BYTES = 256;           // band after every workspace slice
+static const int GUARD_PATTERN = 0xA5;
 
 // ---- kernels_probe.cu
 spts_status launch_rstd(spts_ctx* ctx, const void* X, int N, float* rstd);
@@ -136,6 +146,7 @@ spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld
                                       float* stats, float* S);
 spts_status launch_pap_regroup(spts_ctx* ctx, const void* q_win, int w, void* q_kv);
 spts_status launch_iota_from(spts_ctx* ctx, int32_t* out, int n, int first);
+spts_status launch_transpose_bf16(spts_ctx* ctx, const void* in, int rows, int cols, void* out_t, int ldt);
 spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
                              float* C_out, float* S_ffn);
 spts_status launch_fold_gain(spts_ctx* ctx, void* W, const float* g, int out_f, int in_f);
@@ -191,7 +202,7 @@ spts_status launch_proxy_factor(spts_ctx* ctx, const void* W, const int32_t* cha
 enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4 };
 struct TcGemmArgs {
   const bf16* A; int lda; int a_rows;   // A [a_rows, K]
-  const int32_t* idx;                   // optional gather list (TMA gather4)
+  const int32_t* idx;                   // optional gather list of A rows
   const int32_t* dst_idx;               // TC_RESID scatter rows
   const bf16* W; const bf16* W2;        // [Nout, K]
   int M, Nout, K;

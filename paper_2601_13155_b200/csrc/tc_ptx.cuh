@@ -66,13 +66,15 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;   // 2 s: far beyond any legitimate wait here
 
 // Returns false when the wait was abandoned (limit reached, or another thread raised abort).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t t0) {
+// `limit_ns` is WAIT_LIMIT_NS everywhere except in the self-test kernel, which shortens it.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t t0,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
   if (mbar_test_wait(bar, parity)) return true;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 0xFFu) == 0xFFu) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }

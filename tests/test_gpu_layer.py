@@ -23,6 +23,11 @@ ODD_GROUP_BF16 = replace(synth.LLAMA8B, hidden=384, n_q_heads=6, n_kv_heads=2, h
                          ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
 
 
+# a GQA group of 16 query heads per KV head: more than the eight probe logits the K-projection epilogue keeps in registers
+WIDE_GROUP_BF16 = replace(synth.LLAMA8B, hidden=512, n_q_heads=16, n_kv_heads=1, head_dim=128, ffn_dim=1024,
+                          ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
+
+
 def _mk(shape, max_seq, reference=None):
     from paper_2601_13155_b200 import binding
     lib = binding.Spts(shape, max_seq=max_seq)
@@ -49,6 +54,7 @@ def _modes():
         pytest.param(SMALL_BF16, 1024, 1024, 1024, False, id="small8b-bf16-tensorcore-dense"),
         pytest.param(SMALL_BF16, 640, 640, 200, False, id="small8b-bf16-tensorcore-attn-dense"),
         pytest.param(ODD_GROUP_BF16, 515, 259, 130, False, id="oddgroup-bf16-tensorcore"),
+        pytest.param(WIDE_GROUP_BF16, 333, 150, 101, False, id="group16-bf16-tensorcore"),
     ]
 
 
@@ -191,36 +197,57 @@ def test_prefill_and_decode_match_oracle(dtype, ref):
     lib.close()
 
 
-def test_attention_kernels_agree_under_large_score_jumps():
-    """The two tensor-core attention kernels (two heads per CTA with P in tensor memory; one tile per CTA with P
-    through shared memory) keep their running maximum lazily: O is rescaled only when the maximum grows by more
-    than 2^8.  Here W_q and W_k are scaled so that logits spread over ~45 octaves, which makes rows jump by tens
-    of octaves between key blocks, and the two kernels must agree on identical Q^, K^, V^.  (At this scale the
-    bf16 rounding of Q^ and K^ alone moves probabilities by tens of percent, so the oracle is not the yardstick
-    for this case; the oracle comparisons above cover the ordinary range.)"""
-    from paper_2601_13155_b200 import binding
-    shape = SMALL_BF16
-    N = 1024 + 77
-    W = synth.layer_weights(shape, 31, 0, std=0.05)
-    W["wq"] = synth.quantize(W["wq"] * 5.0, "bf16")
-    W["wk"] = synth.quantize(W["wk"] * 5.0, "bf16")
-    W["w_down"] = np.zeros_like(W["w_down"])          # expose the attention block alone
-    X, _ = synth.hidden_states(shape, N, 31, heavy=16)
-    Wd = binding.LayerWeights(W, "bf16")
-    pos = i32(np.arange(N))
-    outs = []
-    for one_tile in (False, True):
-        lib = _mk(shape, 2048, False)
-        lib.set_attention_one_tile(one_tile)
-        Xd = up(X, "bf16")
-        lib.layer_prefill_skip(Wd, Xd, pos, N, N, binding.KvCache(shape, 1, N))
-        assert lib.device_status() == 0
-        outs.append(host(Xd))
-        lib.close()
-    assert np.isfinite(outs[0]).all()
-    delta = outs[0] - host(up(X, "bf16"))
-    assert np.abs(delta).max() > 0.1                    # the attention block did something
-    check_output(outs[0], outs[1], "bf16")              # same rule as against the oracle
+def _attention_inputs(shape, m, kind, seed):
+    """Q [m,H,d], K, V [m,Hkv,d] as the attention step sees them, rounded to the storage type.
+    kind "normal": logits ~ N(0, 1).  "peaky": logits ~ N(0, 12^2), rows nearly one-hot, the row maximum moves by tens
+    of octaves from one key block to the next in either direction.  "ramp": the logit of key j grows by about half a
+    unit per key, so every row's running maximum rises by ~90 octaves per 128-key block and its mass sits on the
+    last few keys before the diagonal."""
+    rng = np.random.default_rng(seed)
+    H, Hkv, d = shape.n_q_heads, shape.n_kv_heads, shape.head_dim
+    Q = rng.standard_normal((m, H, d))
+    K = rng.standard_normal((m, Hkv, d))
+    V = rng.standard_normal((m, Hkv, d))
+    if kind == "peaky":
+        Q *= 12.0
+    elif kind == "ramp":
+        u = rng.standard_normal(d)
+        u /= np.linalg.norm(u)
+        Q = Q + 8.0 * u
+        K = K + (np.arange(m)[:, None, None] * (0.5 * np.sqrt(d) / 8.0)) * u
+    return tuple(synth.quantize(a.astype(np.float32), shape.dtype) for a in (Q, K, V))
+
+
+@pytest.mark.parametrize("kind", ["normal", "peaky", "ramp"])
+@pytest.mark.parametrize("shape,m,ref,one_tile", [
+    pytest.param(SMALL_BF16, 1101, False, False, id="pair-kernel-even-group"),
+    pytest.param(SMALL_BF16, 1101, False, True, id="one-tile-kernel"),
+    pytest.param(ODD_GROUP_BF16, 600, False, False, id="pair-kernel-odd-group"),
+    pytest.param(WIDE_GROUP_BF16, 385, False, False, id="pair-kernel-group16"),
+    pytest.param(SMALL_BF16, 129, False, False, id="pair-kernel-one-past-a-tile"),
+    pytest.param(SMALL_BF16, 1, False, False, id="pair-kernel-single-row"),
+    pytest.param(SMALL_BF16, 300, True, False, id="plain-kernels-bf16"),
+    pytest.param(synth.TINY, 389, None, False, id="plain-kernels-fp32"),
+])
+def test_reduced_attention_matches_oracle(shape, m, ref, one_tile, kind):
+    """spts_reduced_attention (Algorithm 1's F_MHA(Q^, K^, V^) on the active rows) on operands of the test's choosing
+    against the oracle's causal GQA attention on the very same Q, K, V.  The tensor-core kernels keep their running
+    row maximum lazily (O is rescaled only when the maximum has grown by more than 2^8); the "peaky" and "ramp"
+    operands make that happen at almost every key block, in the regime where a wrong rescale would show."""
+    lib = _mk(shape, 2048, ref)
+    if one_tile:
+        lib.set_attention_one_tile(True)
+    Q, K, V = _attention_inputs(shape, m, kind, 4000 + m)
+    got = lib.reduced_attention(up(Q, shape.dtype), up(K, shape.dtype), up(V, shape.dtype))
+    assert lib.device_status() == 0
+    want = O.causal_gqa_attention(Q.astype(np.float64), K.astype(np.float64), V.astype(np.float64))
+    if kind != "normal" and m >= 130:
+        # the cases are only worth their name if a row's logits really spread by more than the 2^8 threshold
+        z = (K[:, 0].astype(np.float64) @ Q[-1, 0].astype(np.float64)) / np.sqrt(shape.head_dim)
+        assert z.max() - np.sort(z)[-130] > 8.0 * np.log(2.0)
+    check_output(host(got), O.rounding("bf16" if shape.dtype == "bf16" else "exact")(want), shape.dtype, what=f"attention {kind}")
+    assert lib.check_guards() == 0
+    lib.close()
 
 
 @pytest.mark.parametrize("N,ma,mf", [(1, 1, 1), (2, 1, 2), (3, 2, 1), (17, 5, 17), (129, 128, 1), (257, 129, 130)])

@@ -105,9 +105,13 @@ def test_config2_bf16_layer_unforced_reports_selection_and_flip_counts():
     assert rep["max_rel_dist"] <= 2e-2
     # outputs: rows on which both sides took the same two decisions
     same = np.setdiff1d(np.arange(N), np.concatenate([np.setxor1d(ia, want["idx_attn"]), np.setxor1d(jf, want["idx_ffn"])]))
-    st = check_output(host(Xd)[same], want["X"][same], "bf16", what="X")
-    print(f"[parity] cfg2 bf16 unforced: X worst error {st['worst_rel']:.3e} of RMS, {st['flips']} one-ulp disagreements "
-          f"in {st.get('n_flip_rows', 0)} rows of {len(same)} compared rows ({st['flips'] / st['elements']:.2e} of the elements)")
+    # Unforced, an element of the output has been rounded to bf16 twice on each side (after the attention update and
+    # after the FFN update); a one-ulp disagreement after the first rounding can be joined by a second one, so the
+    # rare excursions beyond 2e-2 of the RMS are allowed two ulps here (one in every block-wise comparison).
+    st = check_output(host(Xd)[same], want["X"][same], "bf16", what="X", ulps=2)
+    print(f"[parity] cfg2 bf16 unforced: X worst error {st['worst_rel']:.3e} of RMS, {st['flips']} rounding disagreements "
+          f"beyond 2e-2 of the RMS ({st['flips_beyond_one_ulp']} of them two ulps) in {st.get('n_flip_rows', 0)} rows of "
+          f"{len(same)} compared rows ({st['flips'] / st['elements']:.2e} of the elements)")
     assert st["flips"] <= CFG2_MAX_FLIP_FRACTION * st["elements"]
     if swaps_a == 0:
         check_output(host(cache.k[0][:ma]), want["K"], "bf16", what="cache K")
