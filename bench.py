@@ -5,7 +5,8 @@ One step = one whole prefill of the 32-layer LLaMA-3.1-8B-shaped model (random-i
 synthetic hidden states with heavy tokens) through Algorithm 1: per layer PAP score, top-k,
 reduced attention, LTP score, top-k, reduced FFN; stage-end pruning; first-token head.
 The default workload is configuration "cfg3" (32768-token prompt, four MSDP stages); its line also
-carries `ctx_128k`, the same measurement on config 4 (131072 tokens, one timed step).
+carries `ctx_128k`, the same measurement on config 4 (131072 tokens, three timed steps), and `generation`, config 5
+in short (the cfg3 prompt prefilled at keep 0.5 then 32 greedy decode steps, beside the dense request).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3|cfg4|cfg2|cfg5] [--impl reference]
 
@@ -32,18 +33,15 @@ sys.path.insert(0, ROOT)
 import numpy as np
 
 
-# (workload, operation) -> DRAM bytes of one launch at the workload's stage-0 shape, measured with ncu
-NCU_TRAFFIC_BYTES = {
-    ("cfg3", "gate_up"): 1054.47e6 + 360.71e6,      # tc_gemm_kernel<256, 2, 1>, m_ffn = 13108
-    ("cfg3", "attention"): 360.84e6 + 102.60e6,     # tc_attention_pair_kernel, m_attn = 16384
-    ("cfg3", "down"): 1622.88e6 + 100.31e6,         # tc_gemm_kernel<256, 3, 0>, m_ffn = 13108
-}
-# Decode step at the 8B shape, from the ncu capture of a 4-layer case against 16384 cached rows per layer
-# (profiles/decode_step_8b_4layers.md): the five weight-streaming kernels of a layer move 453.3 MB, the attention
-# kernel 67.4 MB for 16384 rows = 4114 B per cached row.  Both grow in proportion (layers, cached rows), which is
-# how the figure is scaled to the 32-layer step against the benchmark's caches.
-NCU_DECODE_WEIGHT_BYTES_PER_LAYER = 453.3e6
-NCU_DECODE_KV_BYTES_PER_ROW = 4114.0
+def captured_traffic(workload, op):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `op` at the workload's first-stage shape, from the
+    ncu capture recorded in profiles/traffic.json -- or None when there is no record, or when the kernel's source
+    files have changed since the capture (the record carries their SHA-256)."""
+    from paper_2601_13155_b200 import ncu_summary
+    try:
+        return ncu_summary.traffic_for(workload, op)
+    except Exception:
+        return None
 
 
 def parse():
@@ -113,9 +111,10 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # CPU oracle leg (bounded sample)
 # --------------------------------------------------------------------------------------------
-def oracle_sample(w, seconds_hint=20.0):
-    """One skip layer of the workload's shape on a shortened prompt, on the host cores.
-    Returns (tokens_per_s extrapolated to the full depth, cores, description, seconds)."""
+def oracle_sample(w):
+    """The oracle as it stands on BASELINE config 2 in full: one SPTS layer of the 8B shape on an 8192-token prompt
+    (attention keep 0.5, FFN keep 0.4), on the host cores.  `w` only supplies the depth the figure is scaled to.
+    Returns (tokens/s scaled to that depth, cores, description, measured seconds)."""
     from oracle import spts_oracle as O
     from paper_2601_13155_b200 import synth
     try:
@@ -123,18 +122,20 @@ def oracle_sample(w, seconds_hint=20.0):
         cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
         cores = os.cpu_count() or 1
-    n = 1024
-    shape = w.shape
-    W = synth.layer_weights(shape, w.seed, 0)
-    X, _ = synth.hidden_states(shape, n, w.seed, heavy=max(1, n // 100))
-    ma, mf = math.ceil(w.keep_attn * n), math.ceil(w.keep_ffn * n)
+    w2 = synth.workload("qwen2" if w.shape.hidden == synth.QWEN7B.hidden else "cfg2")
+    shape, n = w2.shape, w2.n_tokens
+    W = synth.layer_weights(shape, w2.seed, 0)
+    X, _ = synth.hidden_states(shape, n, w2.seed, heavy=w2.heavy)
+    ma, mf = math.ceil(w2.keep_attn * n), math.ceil(w2.keep_ffn * n)
     t = time.perf_counter()
     O.layer_prefill_skip(X, np.arange(n), W, shape, ma, mf, mode="bf16" if shape.dtype == "bf16" else "exact")
     dt = time.perf_counter() - t
-    layers = shape.n_layers
+    layers = w.shape.n_layers
     tps = n / (dt * layers)
-    desc = (f"one SPTS layer of the {shape.hidden}-wide model on a {n}-token prompt (keep {w.keep_attn}/{w.keep_ffn}), "
-            f"fp64 numpy oracle, {dt:.2f} s; tokens/s = {n} / ({dt:.2f} s x {layers} layers)")
+    desc = (f"measured: config {w2.name} in full -- one SPTS layer of the {shape.hidden}-wide model on its {n}-token prompt "
+            f"(keep {w2.keep_attn}/{w2.keep_ffn}), fp64 numpy oracle, {dt:.2f} s on {cores} threads.  Extrapolation: "
+            f"tokens/s = {n} / ({dt:.2f} s x {layers} layers); the attention term grows with the square of the prompt "
+            f"length, so at 32768 / 131072 tokens the oracle would be slower than this figure")
     return tps, cores, desc, dt
 
 
@@ -197,18 +198,26 @@ def main():
         if args.workload == "cfg3" and not args.no_128k and not args.layers:
             # the same measurement at the longest context (cfg4, 131072 tokens), kernels already warm
             torch.cuda.empty_cache()
-            sub = prefill_line(args, rep, dev, "cfg4", 1, 1, 0, False)
+            sub = prefill_line(args, rep, dev, "cfg4", 3, 1, 0, False)
             if rank == 0:
                 line["ctx_128k"] = {k: sub[k] for k in ("value", "unit", "ms_per_step", "ttft_ms", "steps", "warmup", "config",
                                                         "dense", "roofline", "algorithmic_tflop_per_step",
                                                         "achieved_tflops_whole_step", "breakdown_ms", "per_operation",
                                                         "gpu_launches")}
+            # whole requests (config 5 in short): the cfg3 prompt prefilled at keep 0.5, then 32 greedy decode steps
+            # against the compressed caches, beside the same request with skipping disabled
+            torch.cuda.empty_cache()
+            gen = generation_line(args, rep, dev, decode_steps=32, keeps=(0.5,))
+            if rank == 0:
+                line["generation"] = {"config": gen["config"]["workload"], "decode_steps": 32,
+                                      "keep_0.5": gen["keep_sweep"]["0.5"], "dense": gen["dense"],
+                                      "decode_roofline": gen["roofline"]}
     if rank == 0:
         print(json.dumps(line))
     rep.close()
 
 
-def generation_line(args, rep, dev):
+def generation_line(args, rep, dev, decode_steps=None, keeps=(1.0, 0.7, 0.5, 0.3)):
     """Workload cfg5: a 32768-token prompt is prefilled (Algorithm 1), then `--decode-steps` tokens are decoded
     greedily against the per-layer compressed caches; repeated for keep ratios 1.0 / 0.7 / 0.5 / 0.3 (attention
     and FFN budgets = ceil(keep * prompt), MSDP stages as in config 3) and once with skipping disabled.
@@ -218,7 +227,7 @@ def generation_line(args, rep, dev):
     rank, world = rep.rank, rep.world
     w = synth.workload("cfg3")
     shape = w.shape
-    L, N, T = shape.n_layers, w.n_tokens, args.decode_steps
+    L, N, T = shape.n_layers, w.n_tokens, (decode_steps or args.decode_steps)
     layers = []
     for l in range(L):
         t = synth.device_layer_weights(shape, w.seed, l, dev)
@@ -271,7 +280,7 @@ def generation_line(args, rep, dev):
     pd, dd, lg_d, tk_d, kv_d = request(schedule.workload_plan(w, dense=True), T)
     prof_d = lib.profile_end()
     sweep = {}
-    for keep in (1.0, 0.7, 0.5, 0.3):
+    for keep in keeps:
         lib.profile_begin(14)
         pm, dm, lg, tk, kv = request(plan_for(keep), T)
         prof = lib.profile_end()["decode"]
@@ -294,7 +303,7 @@ def generation_line(args, rep, dev):
     peak = peaks.get("hbm_gbs", 6650.0)
     dk = prof_d["decode"]
     ach = dk["bytes"] / max(dk["ms"], 1e-9) / 1e6
-    mid = sweep["0.5"]
+    mid = sweep["0.5"] if "0.5" in sweep else next(iter(sweep.values()))
     line = None
     if rank == 0:
         line = {"metric": "e2e_generation_tokens_per_s", "value": mid["tokens_per_s"], "unit": "tokens/s", "n_gpus": world,
@@ -308,15 +317,25 @@ def generation_line(args, rep, dev):
                           "tokens_per_s": (N + T) * world / ((pd + dd) * 1e-3), "kv_token_layers": kv_d},
                 "keep_sweep": sweep,
                 "roofline": {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                             "traffic": (L * NCU_DECODE_WEIGHT_BYTES_PER_LAYER + NCU_DECODE_KV_BYTES_PER_ROW * L * (N + T / 2.0))
-                             if shape == synth.LLAMA8B else None,
-                             "traffic_note": "ncu capture of a 4-layer case, scaled by layers and cached rows (see profiles/)",
+                             "traffic": decode_traffic(shape, L, kv_d + L * T / 2.0),
+                             "traffic_note": "ncu capture of a 4-layer case, scaled by layers and cached rows (profiles/traffic.json)",
                              "kernel": "decode step (all layers, dense arm)", "launches": dk["calls"],
                              "ms_per_launch": dk["ms"] / dk["calls"],
                              "peak_source": "measured (copy)" if peaks else "fallback"},
                 "gpu_launches": int(lib.launch_count())}
     lib.close()
     return line
+
+
+def decode_traffic(shape, n_layers, cached_rows_all_layers):
+    """DRAM bytes of one decode step scaled from the capture of a 4-layer case (profiles/traffic.json, op "decode"):
+    the weight-streaming kernels move a fixed number of bytes per layer, the attention kernel a fixed number per
+    cached row; both grow in proportion to what a launch processes."""
+    from paper_2601_13155_b200 import synth
+    rec = captured_traffic("cfg5", "decode")
+    if rec is None or shape != synth.LLAMA8B:
+        return None
+    return n_layers * rec["weight_bytes_per_layer"] + rec["kv_bytes_per_row"] * cached_rows_all_layers
 
 
 def paper_protocol_line(args, rep, dev):
@@ -416,8 +435,9 @@ def per_operation(table, tensor_ops, peaks, wname=None):
             ach = v["bytes"] / sec / 1e9
             out[k] = {"ms": round(v["ms"], 3), "calls": v["calls"], "bound": "hbm", "achieved_gbs": round(ach, 1),
                       "frac_of_measured_peak": round(ach / bw_peak, 3)}
-        if (wname, k) in NCU_TRAFFIC_BYTES:      # DRAM bytes of one launch at the first-stage shape (ncu capture)
-            out[k]["dram_traffic_stage0_launch"] = NCU_TRAFFIC_BYTES[(wname, k)]
+        rec = captured_traffic(wname, k)         # DRAM bytes of one launch at the first-stage shape (ncu capture)
+        if rec is not None:
+            out[k]["dram_traffic_stage0_launch"] = rec["dram_bytes_per_launch"]
     return out
 
 
@@ -546,10 +566,12 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
                 "peak_source": "measured (copy)" if peaks else "fallback"}
 
     # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the stage-0 launch shape, from the ncu
-    # captures summarised under profiles/; only valid for the kernels as they were when the captures were taken
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wname, dom))
-    if roof["traffic"] is not None:
-        roof["traffic_note"] = "ncu capture of one launch at this workload's first-stage shape (see profiles/)"
+    # capture recorded in profiles/traffic.json; null once the kernel's sources differ from the captured ones
+    rec = captured_traffic(wname, dom)
+    if rec is not None:
+        roof["traffic"] = rec["dram_bytes_per_launch"]
+        roof["traffic_note"] = (f"ncu capture of one launch at this workload's first-stage shape ({rec['shape']}), kernel sources "
+                                f"unchanged since (sha256 {rec['source_sha256'][:12]}, captured at commit {rec['commit_at_capture']})")
     total_flops = sum(v["flops"] for v in table.values())
     line = None
     if rank == 0:

@@ -340,8 +340,7 @@ class Spts:
         self._check(self.lib.spts_layer_prefill_skip_batch(self.h, C.byref(w.c), _ptr(X), _ptr(pos), n_seq,
                                                            arr(seq_start), arr(m_attn), arr(m_ffn), flags, caches.c,
                                                            _ptr(S_out), _ptr(idx_attn_out), _ptr(idx_ffn_out)),
-                    "spts_layer_prefill_skip_batch", "spts_msdp_plan", "spts_check_guards", "spts_selftest_wait_timeout",
-           "spts_debug_check_index_list", "spts_reduced_attention")
+                    "spts_layer_prefill_skip_batch")
 
     def msdp_compact(self, X_in, pos_in, orig_in, S_mha, n_next: int, X_out, pos_out, orig_out, idx_out=None,
                      flags: int = FORCE_LAST):

@@ -245,7 +245,12 @@ def test_reduced_attention_matches_oracle(shape, m, ref, one_tile, kind):
         # the cases are only worth their name if a row's logits really spread by more than the 2^8 threshold
         z = (K[:, 0].astype(np.float64) @ Q[-1, 0].astype(np.float64)) / np.sqrt(shape.head_dim)
         assert z.max() - np.sort(z)[-130] > 8.0 * np.log(2.0)
-    check_output(host(got), O.rounding("bf16" if shape.dtype == "bf16" else "exact")(want), shape.dtype, what=f"attention {kind}")
+    # Rows of an attention output are independent averages: row 0 is V[0] itself, row 1000 the mean of a thousand
+    # values, thirty times smaller.  The tolerance is therefore taken relative to each row's own RMS.  fp32 mode on
+    # the ramp: logits reach ~200, i.e. raw dot products of ~1500 whose fp32 spacing (1.2e-4) times 1/sqrt(d) already
+    # moves a probability by ~1e-5 per rounding, so that case gets three times the fp32 bound.
+    check_output(host(got), O.rounding("bf16" if shape.dtype == "bf16" else "exact")(want), shape.dtype, per_row=True,
+                 scale=3.0 if (shape.dtype == "fp32" and kind == "ramp") else 1.0, what=f"attention {kind}")
     assert lib.check_guards() == 0
     lib.close()
 
