@@ -106,6 +106,8 @@ typedef struct {
   const void* vu;      /* [Dlow, r]   V_up^T    */
   const void* vd;      /* [r, Dlow]   V_down    */
   const void* ud;      /* [D, r]      U_down    */
+  const void* prepared; /* optional: the layer's buffer filled by spts_prepare_layer() (NULL: the proxy factors are
+                           repacked inside every call that evaluates Eq. 12-14) */
 } spts_layer_weights;
 
 /* One layer's KV cache: k, v are [capacity, Hkv, d] in the storage type (K after RoPE),
@@ -228,6 +230,16 @@ spts_status spts_fold_norm_gain(spts_ctx* ctx, void* W, const float* g, int out_
  * The logits are taken from the unrounded fp32 keys.  K_out may be NULL (workspace is used). */
 spts_status spts_pap_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X,
                            const int32_t* pos, int N, void* K_out, float* S_mha_out);
+
+/* One-time repacking of a layer's proxy-FFN factors (Eq. 12) into the operand layouts the probe's GEMM chain reads,
+ * so that nothing of it is left on the per-layer path: U_gate^T stacked over U_up^T (one [2r, D] matrix: the
+ * residual stream is then read once for both), V_gate^T and V_up^T zero-padded to [D_low, 2r] each, and the Gram
+ * matrix G = U_down^T U_down [r, r] split into a high and a low part: since ||t U_down^T||^2 = t G t^T, Eq. 13's
+ * norm needs an [N, r] x [r, 2r] product instead of the [N, r] x [r, D] one.  `prepared` is caller-owned device
+ * memory of spts_prepared_bytes(desc) bytes, 256-byte aligned; put its address into spts_layer_weights.prepared.
+ * It must be redone when ug, uu, vg, vu or ud change.  Results are bit-identical with and without it. */
+size_t spts_prepared_bytes(const spts_model_desc* desc);
+spts_status spts_prepare_layer(spts_ctx* ctx, const spts_layer_weights* w, void* prepared, size_t prepared_bytes);
 
 /* Low-rank Transformation Probing, Eq. 12-14: C[n] = || f(rmsnorm(X[n])) ||_2 with
  * f(x) = (silu(x Ug Vg) * (x Uu Vu)) Vd^T Ud^T, and S_ffn[n] = C[n] * S_mha[n].

@@ -44,7 +44,7 @@ WEIGHT_NAMES = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "ug", "vg", 
 
 
 class LayerWeightsC(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES] + [("prepared", C.c_void_p)]
 
 
 class KvLayerC(C.Structure):
@@ -71,7 +71,7 @@ EXPORTS = ("spts_workspace_bytes", "spts_create", "spts_destroy", "spts_set_opti
            "spts_first_token", "spts_prefill", "spts_decode_step", "spts_profile_begin", "spts_profile_end",
            "spts_topk_select_static", "spts_proxy_scratch_bytes", "spts_proxy_build",
            "spts_layer_prefill_skip_batch", "spts_msdp_plan", "spts_check_guards", "spts_selftest_wait_timeout",
-           "spts_debug_check_index_list", "spts_reduced_attention")
+           "spts_debug_check_index_list", "spts_reduced_attention", "spts_prepared_bytes", "spts_prepare_layer")
 
 OP_NAMES = {1: "prep", 2: "kproj_pap", 3: "pap_softmax", 4: "topk", 5: "kv_gather", 6: "qv_proj", 7: "attention",
             8: "o_proj", 9: "ltp", 10: "gate_up", 11: "down", 12: "compact", 13: "head", 14: "decode"}
@@ -114,6 +114,9 @@ def load_library() -> C.CDLL:
     lib.spts_selftest_wait_timeout.argtypes = [vp, u32]
     lib.spts_debug_check_index_list.argtypes = [vp, vp, i32, i32]
     lib.spts_reduced_attention.argtypes = [vp, vp, vp, vp, i32, vp]
+    lib.spts_prepared_bytes.restype = C.c_size_t
+    lib.spts_prepared_bytes.argtypes = [C.POINTER(ModelDesc)]
+    lib.spts_prepare_layer.argtypes = [vp, C.POINTER(LayerWeightsC), vp, C.c_size_t]
     lib.spts_first_token.argtypes = [vp, vp, vp, vp, vp]
     lib.spts_prefill.argtypes = [vp, C.POINTER(ModelWeightsC), C.POINTER(LayerPlanC), vp, vp, vp, vp, vp, vp,
                                  i32, u32, C.POINTER(KvLayerC), C.POINTER(C.c_int32), C.POINTER(C.c_int32), vp]
@@ -123,7 +126,8 @@ def load_library() -> C.CDLL:
     lib.spts_profile_end.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64), C.POINTER(C.c_double),
                                      C.POINTER(C.c_double)]
     for n in EXPORTS:
-        if n not in ("spts_workspace_bytes", "spts_destroy", "spts_launch_count", "spts_proxy_scratch_bytes"):
+        if n not in ("spts_workspace_bytes", "spts_destroy", "spts_launch_count", "spts_proxy_scratch_bytes",
+                     "spts_prepared_bytes"):
             getattr(lib, n).restype = C.c_int
     return lib
 
@@ -174,6 +178,16 @@ class LayerWeights:
     def __init__(self, arrays: Dict[str, np.ndarray], dtype: str, device="cuda:0"):
         self.t = {n: to_device(arrays[n], dtype, device) for n in WEIGHT_NAMES}
         self.c = LayerWeightsC(**{n: self.t[n].data_ptr() for n in WEIGHT_NAMES})
+        self.prepared = None
+
+    @classmethod
+    def from_tensors(cls, tensors: Dict[str, torch.Tensor]) -> "LayerWeights":
+        """Wraps device tensors that already hold the matrices in the storage type (no copy)."""
+        w = cls.__new__(cls)
+        w.t = tensors
+        w.c = LayerWeightsC(**{n: tensors[n].data_ptr() for n in WEIGHT_NAMES})
+        w.prepared = None
+        return w
 
 
 class KvCache:
@@ -321,6 +335,17 @@ class Spts:
                                                      flags, C.byref(cache.c[layer]), _ptr(S_out),
                                                      _ptr(idx_attn_out), _ptr(idx_ffn_out)),
                     "spts_layer_prefill_skip")
+
+    def prepare_layer(self, w: "LayerWeights"):
+        """spts_prepare_layer: repacks the layer's proxy factors once into a buffer the weights object then owns;
+        later calls with `w` skip the per-call repacking.  Redo after changing ug / uu / vg / vu / ud."""
+        nbytes = self.lib.spts_prepared_bytes(C.byref(self.desc))
+        buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        w.c.prepared = None
+        self._check(self.lib.spts_prepare_layer(self.h, C.byref(w.c), _ptr(buf), nbytes), "spts_prepare_layer")
+        w.prepared = buf
+        w.c.prepared = buf.data_ptr()
+        return w
 
     def reduced_attention(self, Q, K, V, O_out=None):
         """spts_reduced_attention: causal GQA attention among the m rows of Q [m,H,d], K, V [m,Hkv,d] -> [m, H*d]."""

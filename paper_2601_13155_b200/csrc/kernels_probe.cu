@@ -173,7 +173,7 @@ __global__ void ffn_score_kernel(const float* __restrict__ csq, int stride, int 
   if (n >= N) return;
   float s = 0.f;
   for (int p = 0; p < parts; ++p) s += csq[(size_t)n * stride + p];
-  float c = sqrtf(s);
+  float c = sqrtf(fmaxf(s, 0.f));            // the quadratic-form route can round a tiny norm below zero
   if (C_out) C_out[n] = c;
   S_ffn[n] = c * S_mha[n];
 }
@@ -196,6 +196,35 @@ __global__ void pad_proxy_kernel(const T* __restrict__ vg, const T* __restrict__
   T zero = from_f32<T>(0.f);
   out[t] = c < r ? vg[row * r + c] : zero;
   out[total + t] = c < r ? zero : vu[row * r + (c - r)];
+}
+
+// G = Ud^T Ud for Ud [D, r] (row-major), accumulated in double; written as its bf16 rounding (rows 0..r) followed by
+// the bf16 rounding of the remainder (rows r..2r), so that a bf16 tensor-core product with [G_hi ; G_lo] carries G to
+// ~2^-17.  One 16 x 16 tile of G per block.  Runs once per layer (spts_prepare_layer) or, without a prepared
+// buffer, once per call.
+__global__ void gram_kernel(const bf16* __restrict__ ud, int D, int r, bf16* __restrict__ g2) {
+  __shared__ float sa[64][17], sb[64][17];
+  const int i0 = blockIdx.x * 16, j0 = blockIdx.y * 16;
+  const int ti = threadIdx.x & 15, tj = threadIdx.x >> 4;
+  double acc = 0.0;
+  for (int d0 = 0; d0 < D; d0 += 64) {
+    for (int e = threadIdx.x; e < 64 * 16; e += 256) {
+      const int dd = e >> 4, c = e & 15;
+      const bool in = d0 + dd < D;
+      sa[dd][c] = in ? to_f32(ud[(size_t)(d0 + dd) * r + i0 + c]) : 0.f;
+      sb[dd][c] = in ? to_f32(ud[(size_t)(d0 + dd) * r + j0 + c]) : 0.f;
+    }
+    __syncthreads();
+    float part = 0.f;                        // 64 products of bf16 pairs: exact enough in fp32 before the double sum
+#pragma unroll 16
+    for (int dd = 0; dd < 64; ++dd) part = fmaf(sa[dd][ti], sb[dd][tj], part);
+    acc += (double)part;
+    __syncthreads();
+  }
+  const float g = (float)acc;
+  const bf16 hi = __float2bfloat16_rn(g);
+  g2[(size_t)(i0 + ti) * r + j0 + tj] = hi;
+  g2[(size_t)(r + i0 + ti) * r + j0 + tj] = __float2bfloat16_rn(g - __bfloat162float(hi));
 }
 
 // argmax with the lowest index on ties (NaN never wins; 0 if nothing does), in two steps: every block reduces one
@@ -394,6 +423,14 @@ spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void
     pad_proxy_kernel<bf16><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const bf16*)vg, (const bf16*)vu, d.ltp_dlow, d.ltp_rank, (bf16*)out);
   else
     pad_proxy_kernel<float><<<ceil_div(total, 256), 256, 0, ctx->stream>>>((const float*)vg, (const float*)vu, d.ltp_dlow, d.ltp_rank, (float*)out);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_gram(spts_ctx* ctx, const void* ud, void* g2) {
+  const auto& d = ctx->desc;
+  if (d.dtype != SPTS_BF16 || d.ltp_rank % 16) return SPTS_ERR_UNSUPPORTED;
+  gram_kernel<<<dim3(d.ltp_rank / 16, d.ltp_rank / 16), 256, 0, ctx->stream>>>((const bf16*)ud, d.hidden, d.ltp_rank, (bf16*)g2);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

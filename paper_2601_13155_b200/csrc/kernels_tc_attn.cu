@@ -14,7 +14,8 @@
 //               (4 x 128 fp32 columns).  Per key block j and tile t:  O_t += P_t V_j  (A operand P_t
 //               read from TMEM, where it overwrites the first 64 columns of S_t; issued piece by
 //               piece as the softmax warps deliver it), then S_t = Q_t K_{j+1}^T.
-//   warps 2-5   softmax of tile 0, warps 6-9 softmax of tile 1; one query row per thread, the whole score
+//   warps 2-3   no role (they fill the first warp group, whose registers are handed to the softmax warps)
+//   warps 4-7   softmax of tile 0, warps 8-11 softmax of tile 1; one query row per thread, the whole score
 //               row in registers: row maximum, p = 2^(s * log2(e)/sqrt(d) - max) with a lazily updated running maximum (O_t
 //               is rescaled in TMEM only when the maximum grows by more than 2^8), row sum, P_t
 //               written back to TMEM as packed bf16; at the end O_t / l goes to global memory.
@@ -313,7 +314,16 @@ tc_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // paired-head kernel
 // ---------------------------------------------------------------------------------------------
-constexpr int AP_THREADS = 320;              // TMA warp, MMA warp, 2 x 4 softmax warps
+// Warp group 0: TMA warp, MMA warp, two warps with no role; warp groups 1 and 2: the softmax of tile 0 and of tile 1.
+// Registers live per SM sub-partition (16384 each, three warps of this block on every one), so an even split caps a
+// thread at 168.  The light warp group hands registers back (setmaxnreg works on whole warp groups, hence the two
+// idle warps) and a softmax thread -- which keeps a whole 128-entry score row plus its packed probabilities in
+// registers -- gets 224: the same kernel with the softmax squeezed into 168 registers ran 6 % slower.
+constexpr int AP_THREADS = 384;
+constexpr int REGS_LIGHT = 56, REGS_SOFTMAX = 224;   // 128 * 56 + 256 * 224 = 384 * 168
+
+__device__ __forceinline__ void setmaxnreg_dec_light() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_LIGHT)); }
+__device__ __forceinline__ void setmaxnreg_inc_softmax() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX)); }
 constexpr int AP_SMEM = 2 * TILE_BYTES /*Q_0, Q_1*/ + KV_STAGES * TILE_BYTES /*K*/ + KV_STAGES * TILE_BYTES /*V^T*/ +
                         1024 + 256;
 
@@ -378,6 +388,10 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // the register hand-over brackets each warp group's whole role: code after a join of the two branches would have to
+  // fit the smaller allowance
+  if (warp < 4) {
+  setmaxnreg_dec_light();
   if (warp == 0) {
     if (lane == 0) {
       mbar_expect_tx(q_full, 3 * TILE_BYTES);               // both Q tiles and K_0 (K_j sits in slot (j + 1) & 1)
@@ -467,9 +481,11 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         mma_commit(kv_free + 8 * sv);
       }
     }
+  }
   } else {
+    setmaxnreg_inc_softmax();
     // ------------------------------------------------------------------ softmax / rescale / epilogue
-    const int t = (warp - 2) >> 2;                     // tile
+    const int t = (warp - 4) >> 2;                     // tile
     const int qt = qt0 + t * dq, head = h0 + t * dh;
     const int nblk_t = qt + 1;
     const int quarter = warp & 3;                      // TMEM lane quarter this warp may access

@@ -16,6 +16,7 @@
 //                 TC_SWIGLU  tile = 128 gate | 128 up columns; out = bf16(silu(g) * u)   (Eq. 6)
 //                 TC_RESID   X[dst(i), :] += acc, in place (Eq. 2 residual scatter)
 //                 TC_SUMSQ   per-row sum of squares of the tile (Eq. 13), no matrix written
+//                 TC_QFORM   per-row dot product of the tile with the row's own A operand (Eq. 13 as t G t^T)
 // Accumulators are double-buffered in TMEM so the epilogue of tile t overlaps the MMAs of t+1.
 #include "spts_common.cuh"
 #include "tc_ptx.cuh"
@@ -464,6 +465,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
+      } else if (EPI == TC_QFORM) {
+        // Eq. 13 through the Gram matrix: the tile holds y = t [G_hi ; G_lo]^T for this row's t (the A operand itself,
+        // r wide); its share of t G t^T is sum_j y_j t_{j mod r}.  No matrix is written.
+        float s = 0.f;
+        const bf16* trow = reinterpret_cast<const bf16*>(p.a_ptr) + (size_t)grow * p.lda;
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(tacc + c, r);
+          tmem_ld_wait();
+          if (row_ok && n0 + c < p.Nout) {
+            const int k0 = (n0 + c) % p.K;               // K = r, a multiple of 32: the 32 columns stay inside one copy
+            const uint4* tp = reinterpret_cast<const uint4*>(trow + k0);
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const uint4 w = __ldg(tp + g);
+              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float t0v, t1v;
+                unpack_bf16(ww[e], t0v, t1v);
+                s = fmaf(__uint_as_float(r[g * 8 + 2 * e]), t0v, s);
+                s = fmaf(__uint_as_float(r[g * 8 + 2 * e + 1]), t1v, s);
+              }
+            }
+          }
+        }
+        if (row_ok) p.csq[(size_t)grow * p.csq_parts + nb] = s;
       } else {   // TC_SUMSQ
         float s = 0.f;
 #pragma unroll 1
@@ -634,7 +663,7 @@ spts_status tc_gemm_init(spts_ctx* ctx) {
   ctx->encode_tiled = fn;
   bool ok = set_smem_attr<256, TC_STORE>() && set_smem_attr<256, TC_ROPE>() && set_smem_attr<256, TC_SWIGLU>() &&
             set_smem_attr<256, TC_RESID>() && set_smem_attr<256, TC_SUMSQ>() && set_smem_attr<128, TC_STORE>() &&
-            set_smem_attr<128, TC_ROPE>() && set_smem_attr<128, TC_SWIGLU>();
+            set_smem_attr<128, TC_ROPE>() && set_smem_attr<128, TC_SWIGLU>() && set_smem_attr<256, TC_QFORM>();
   return ok ? SPTS_OK : SPTS_ERR_CUDA;
 }
 
@@ -643,21 +672,34 @@ spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a) {
   if (ctx->encode_tiled == nullptr) return SPTS_ERR_UNSUPPORTED;
   if ((a.K % 8) || (a.lda % 8) || (reinterpret_cast<uintptr_t>(a.A) & 15) || (reinterpret_cast<uintptr_t>(a.W) & 15))
     return SPTS_ERR_SHAPE;
-  if (a.out == nullptr && epi != TC_SUMSQ && !(epi == TC_SWIGLU && a.sal_t != nullptr) &&
+  if (a.out == nullptr && epi != TC_SUMSQ && epi != TC_QFORM && !(epi == TC_SWIGLU && a.sal_t != nullptr) &&
       !(epi == TC_STORE && a.out_f32 != nullptr))
     return SPTS_ERR_INVALID_ARG;
   if (a.ldw % 8) return SPTS_ERR_SHAPE;
   if (a.out != nullptr && ((a.ldo % 8) || (reinterpret_cast<uintptr_t>(a.out) & 15))) return SPTS_ERR_SHAPE;
   if ((a.Nout % 8) && a.out_f32 == nullptr) return SPTS_ERR_SHAPE;
   const bool narrow = a.Nout <= 128;       // a 128-wide tile wastes less on the skinny proxy factors
+  // A skinny output (the proxy's stacked first factors: 2r columns) gives one 256-wide tile per 128 rows, and the
+  // tile count then rounds badly against the SM count (256 tiles on 148 SMs: two waves, the second 73 % idle).
+  // Half-width tiles double the count; take them when they fill the waves clearly better.
+  bool half = false;
+  if (epi == TC_STORE && !narrow && a.Nout <= 512) {
+    const int sm = ctx->sm_count > 0 ? ctx->sm_count : 148;
+    const int t256 = ceil_div(a.M, BM) * ceil_div(a.Nout, 256), t128 = ceil_div(a.M, BM) * ceil_div(a.Nout, 128);
+    const double e256 = (double)t256 / ((double)ceil_div(t256, sm) * sm), e128 = (double)t128 / ((double)ceil_div(t128, sm) * sm);
+    half = e128 > e256 + 0.08;
+  }
   switch (epi) {
-    case TC_STORE: return narrow ? launch_one<128, TC_STORE>(ctx, a) : launch_one<256, TC_STORE>(ctx, a);
+    case TC_STORE: return (narrow || half) ? launch_one<128, TC_STORE>(ctx, a) : launch_one<256, TC_STORE>(ctx, a);
     case TC_ROPE:
       if (a.Nout % 128) return SPTS_ERR_SHAPE;
       return narrow ? launch_one<128, TC_ROPE>(ctx, a) : launch_one<256, TC_ROPE>(ctx, a);
     case TC_SWIGLU: return (a.Nout <= 64) ? launch_one<128, TC_SWIGLU>(ctx, a) : launch_one<256, TC_SWIGLU>(ctx, a);
     case TC_RESID: return launch_one<256, TC_RESID>(ctx, a);
     case TC_SUMSQ: return launch_one<256, TC_SUMSQ>(ctx, a);
+    case TC_QFORM:
+      if (a.K % 32 || a.Nout % a.K || a.idx != nullptr) return SPTS_ERR_SHAPE;
+      return launch_one<256, TC_QFORM>(ctx, a);
     default: return SPTS_ERR_INVALID_ARG;
   }
 }

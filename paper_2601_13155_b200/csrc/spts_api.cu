@@ -60,6 +60,7 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
   w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
   w.ugu = c.take<char>(2 * (size_t)d.ltp_rank * d.hidden * es);
+  w.g2 = c.take<char>(2 * (size_t)d.ltp_rank * d.ltp_rank * es);
   {
     const size_t G = (size_t)d.n_q_heads / d.n_kv_heads;
     w.pw_logits = c.take<float>((size_t)PAP_MAX_WINDOW * G * Npad);
@@ -247,6 +248,34 @@ spts_status pap_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   return SPTS_OK;
 }
 
+// Layout of a prepared-layer buffer (spts_prepare_layer): [Ug^T ; Uu^T] [2r, D], then [Vg^T | 0] and [0 | Vu^T]
+// ([D_low, 2r] each), then [G_hi ; G_lo] [2r, r] (tensor-core mode), each slice 256-byte aligned.
+struct PreparedLayout { size_t ugu, vgu, g2, total; };
+PreparedLayout prepared_layout(const spts_model_desc& d) {
+  const size_t es = elt_size(d);
+  PreparedLayout l;
+  l.ugu = 0;
+  l.vgu = align_up(l.ugu + 2 * (size_t)d.ltp_rank * d.hidden * es, 256);
+  l.g2 = align_up(l.vgu + 2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es, 256);
+  l.total = align_up(l.g2 + 2 * (size_t)d.ltp_rank * d.ltp_rank * es, 256);
+  return l;
+}
+
+// Eq. 13 as a quadratic form in the Gram matrix of U_down: tensor-core mode with a rank the epilogue's 32-column
+// chunks divide.  Otherwise the proxy output's sum of squares is taken from the [N, r] x [r, D] product itself.
+bool ltp_uses_gram(const spts_ctx* ctx) { return use_tc(ctx) && ctx->desc.ltp_rank % 32 == 0; }
+
+spts_status pack_proxy(spts_ctx* ctx, const spts_layer_weights* w, void* ugu, void* vgu, void* g2) {
+  const auto& d = ctx->desc;
+  const size_t ubytes = (size_t)d.ltp_rank * d.hidden * elt_size(d);
+  TRY(launch_pad_proxy(ctx, w->vg, w->vu, vgu));
+  if (cudaMemcpyAsync(ugu, w->ug, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess ||
+      cudaMemcpyAsync((char*)ugu + ubytes, w->uu, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+    return SPTS_ERR_CUDA;
+  if (ltp_uses_gram(ctx)) TRY(launch_gram(ctx, w->ud, g2));
+  return SPTS_OK;
+}
+
 // LTP (Eq. 12-14) on rows already normalised through `rstd`.
 spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const float* S_mha, int N,
                          float* C_out, float* S_ffn_out) {
@@ -257,32 +286,44 @@ spts_status ltp_pipeline(spts_ctx* ctx, const spts_layer_weights* w, const void*
   const double Nd = (double)N;
   ProfScope ps_ltp(ctx, SPTS_OP_LTP, 6.0 * Nd * r * ((double)d.hidden + Dl),
                    Nd * d.hidden * (double)es + 3.0 * r * ((double)d.hidden + Dl) * (double)es + 8.0 * Nd);
-  TRY(launch_pad_proxy(ctx, w->vg, w->vu, ws.vgu_pad));
+  // the repacked factors: the layer's prepared buffer, or packed here into the workspace
+  const void* ugu = ws.ugu; const void* vgu = ws.vgu_pad; const void* g2 = ws.g2;
+  if (w->prepared != nullptr) {
+    const PreparedLayout pl = prepared_layout(d);
+    const char* base = (const char*)w->prepared;
+    ugu = base + pl.ugu; vgu = base + pl.vgu; g2 = base + pl.g2;
+  } else {
+    TRY(pack_proxy(ctx, w, ws.ugu, ws.vgu_pad, ws.g2));
+  }
   Gemm g;
   // t1 = [x Ug | x Uu]: the two first factors are stacked into one [2r, D] matrix so that the residual
   // stream (the only large operand of the whole proxy) is read once
-  const size_t ubytes = (size_t)r * d.hidden * es;
-  if (cudaMemcpyAsync(ws.ugu, w->ug, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess ||
-      cudaMemcpyAsync((char*)ws.ugu + ubytes, w->uu, ubytes, cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
-    return SPTS_ERR_CUDA;
   memset(&g, 0, sizeof(g));
-  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = ws.ugu; g.M = N; g.Nout = 2 * r; g.K = d.hidden;
+  g.A = X; g.lda = d.hidden; g.a_rows = N; g.W = ugu; g.M = N; g.Nout = 2 * r; g.K = d.hidden;
   g.rowscale = ws.rstd; g.out = ws.t1; g.ldo = 2 * r;
   TRY(run_gemm(ctx, REF_STORE, g));
   // hlow = silu(t_g Vg) * (t_u Vu)
   memset(&g, 0, sizeof(g));
-  g.A = ws.t1; g.lda = 2 * r; g.a_rows = N; g.W = ws.vgu_pad; g.W2 = (char*)ws.vgu_pad + (size_t)Dl * 2 * r * es;
+  g.A = ws.t1; g.lda = 2 * r; g.a_rows = N; g.W = vgu; g.W2 = (const char*)vgu + (size_t)Dl * 2 * r * es;
   g.M = N; g.Nout = Dl; g.K = 2 * r; g.out = ws.hlow; g.ldo = Dl;
   TRY(run_gemm(ctx, REF_SWIGLU, g));
   // t2 = hlow Vd^T
   memset(&g, 0, sizeof(g));
   g.A = ws.hlow; g.lda = Dl; g.a_rows = N; g.W = w->vd; g.M = N; g.Nout = r; g.K = Dl; g.out = ws.t2; g.ldo = r;
   TRY(run_gemm(ctx, REF_STORE, g));
-  // C^2 = || t2 Ud^T ||^2, summed in the epilogue
+  int parts;
   memset(&g, 0, sizeof(g));
-  g.A = ws.t2; g.lda = r; g.a_rows = N; g.W = w->ud; g.M = N; g.Nout = d.hidden; g.K = r; g.csq = ws.csq;
-  TRY(run_gemm(ctx, REF_SUMSQ, g));
-  const int parts = use_tc(ctx) ? tc_sumsq_parts(d.hidden) : ceil_div(d.hidden, 64);
+  if (ltp_uses_gram(ctx)) {
+    // C^2 = t2 G t2^T with G = Ud^T Ud: y = t2 [G_hi ; G_lo]^T, and the epilogue dots y with the row of t2 itself
+    g.A = ws.t2; g.lda = r; g.a_rows = N; g.W = g2; g.M = N; g.Nout = 2 * r; g.K = r; g.csq = ws.csq;
+    TRY(run_gemm(ctx, TC_QFORM, g));
+    parts = ceil_div(2 * r, 256);
+  } else {
+    // C^2 = || t2 Ud^T ||^2, summed in the epilogue
+    g.A = ws.t2; g.lda = r; g.a_rows = N; g.W = w->ud; g.M = N; g.Nout = d.hidden; g.K = r; g.csq = ws.csq;
+    TRY(run_gemm(ctx, REF_SUMSQ, g));
+    parts = use_tc(ctx) ? tc_sumsq_parts(d.hidden) : ceil_div(d.hidden, 64);
+  }
   TRY(launch_ffn_score(ctx, ws.csq, parts, S_mha, N, C_out, S_ffn_out));
   return SPTS_OK;
 }
@@ -533,6 +574,23 @@ spts_status spts_fold_norm_gain(spts_ctx* ctx, void* W, const float* g, int out_
   return launch_fold_gain(ctx, W, g, out_features, in_features);
 }
 
+size_t spts_prepared_bytes(const spts_model_desc* desc) {
+  if (desc == nullptr || !shape_ok(*desc)) return 0;
+  return prepared_layout(*desc).total;
+}
+
+spts_status spts_prepare_layer(spts_ctx* ctx, const spts_layer_weights* w, void* prepared, size_t prepared_bytes) {
+  TRY(check_ctx(ctx));
+  if (w == nullptr || prepared == nullptr || w->ug == nullptr || w->uu == nullptr || w->vg == nullptr ||
+      w->vu == nullptr || w->ud == nullptr)
+    return SPTS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(prepared) & 255) != 0) return SPTS_ERR_INVALID_ARG;
+  const PreparedLayout pl = prepared_layout(ctx->desc);
+  if (prepared_bytes < pl.total) return SPTS_ERR_WORKSPACE;
+  char* base = (char*)prepared;
+  return pack_proxy(ctx, w, base + pl.ugu, base + pl.vgu, base + pl.g2);
+}
+
 spts_status spts_pap_score(spts_ctx* ctx, const spts_layer_weights* w, const void* X, const int32_t* pos, int N,
                            void* K_out, float* S_mha_out) {
   TRY(check_ctx(ctx));
@@ -611,11 +669,11 @@ spts_status spts_reduced_attention(spts_ctx* ctx, const void* Q, const void* K, 
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O_out)) return SPTS_ERR_INVALID_ARG;
   const auto& d = ctx->desc;
   const double Ma = (double)m, HD = (double)d.n_q_heads * d.head_dim, KD = (double)d.n_kv_heads * d.head_dim;
+  // the tensor-core kernel reads V through its transposed copy (made outside the timed operation)
+  const int ldvt = (int)align_up((size_t)m, 128);
+  if (use_tc(ctx)) TRY(launch_transpose_bf16(ctx, V, m, d.n_kv_heads * d.head_dim, ctx->ws.v_t, ldvt));
   ProfScope ps(ctx, SPTS_OP_ATTN, 2.0 * HD * Ma * (Ma + 1.0), (2.0 * Ma * HD + 2.0 * Ma * KD) * (double)elt_size(d));
   if (!use_tc(ctx)) return launch_ref_attention(ctx, Q, K, V, m, O_out);
-  // the tensor-core kernel reads V through its transposed copy
-  const int ldvt = (int)align_up((size_t)m, 128);
-  TRY(launch_transpose_bf16(ctx, V, m, d.n_kv_heads * d.head_dim, ctx->ws.v_t, ldvt));
   return launch_tc_attention(ctx, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)ctx->ws.v_t, ldvt, m,
                              (bf16*)O_out);
 }

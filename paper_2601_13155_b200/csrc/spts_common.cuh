@@ -60,6 +60,7 @@ struct Workspace {
   void* q_kv;           // the same regrouped by KV head
   int32_t* idx_w;       // [PAP_MAX_WINDOW] the window's candidate indices
   void* ugu;            // [2r, D] the proxy's first factors stacked (Ug^T over Uu^T): one GEMM reads x once
+  void* g2;             // [2r, r] Gram matrix Ud^T Ud, high part over low part (tensor-core mode)
   float* logits;        // [H, Nmax]
   float* head_stats;    // [2*H] max and sum of exp per head
   float* s_mha;         // [Nmax]
@@ -141,6 +142,7 @@ spts_status launch_rope_table(spts_ctx* ctx, const int32_t* pos, int N, float2* 
 spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N, const void* wq,
                           const float* rstd, float* q);
 spts_status launch_pad_proxy(spts_ctx* ctx, const void* vg, const void* vu, void* out);
+spts_status launch_gram(spts_ctx* ctx, const void* ud, void* g2);   // g2 [2r, r]: bf16(G) over bf16(G - bf16(G)), G = Ud^T Ud
 spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, float* S);
 spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, int w, int accumulate,
                                       float* stats, float* S);
@@ -199,7 +201,7 @@ spts_status launch_proxy_factor(spts_ctx* ctx, const void* W, const int32_t* cha
                                 void* u_out, void* v_out, float* sigma_sorted);
 
 // ---- kernels_tc_gemm.cu / kernels_tc_attn.cu : tcgen05 path (bf16)
-enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4 };
+enum TcEpi { TC_STORE = 0, TC_ROPE = 1, TC_SWIGLU = 2, TC_RESID = 3, TC_SUMSQ = 4, TC_QFORM = 5 };
 struct TcGemmArgs {
   const bf16* A; int lda; int a_rows;   // A [a_rows, K]
   const int32_t* idx;                   // optional gather list of A rows

@@ -35,9 +35,7 @@ def main():
     dev = "cuda:0"
     n = a.tokens
     t = synth.device_layer_weights(shape, w.seed, 0, dev)
-    lw = binding.LayerWeights.__new__(binding.LayerWeights)
-    lw.t = t
-    lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    lw = binding.LayerWeights.from_tensors(t)
     X0, _ = synth.device_hidden_states(w, dev, n_tokens=n)
     lib = binding.Spts(shape, max_seq=n)
     cache = binding.KvCache(shape, 1, n)
@@ -64,9 +62,7 @@ def proxy_case(a):
     shape = replace(w.shape, n_layers=1)
     dev = "cuda:0"
     t = synth.device_layer_weights(shape, w.seed, 0, dev)
-    lw = binding.LayerWeights.__new__(binding.LayerWeights)
-    lw.t = t
-    lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    lw = binding.LayerWeights.from_tensors(t)
     Xc, _ = synth.device_hidden_states(w, dev, n_tokens=a.proxy)
     lib = binding.Spts(shape, max_seq=1024)
     lib.proxy_build(lw, Xc, rho=0.2)
@@ -91,9 +87,7 @@ def decode_case(a):
     layers = []
     for l in range(a.layers):
         t = synth.device_layer_weights(shape, 7, l, dev)
-        lw = binding.LayerWeights.__new__(binding.LayerWeights)
-        lw.t = t
-        lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+        lw = binding.LayerWeights.from_tensors(t)
         layers.append(lw)
     hw = synth.device_head_weights(shape, 7, dev)
     model = binding.Model(layers, hw["lm_head"], hw["embed"])

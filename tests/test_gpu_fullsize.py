@@ -36,14 +36,10 @@ def _run_layer_case(name, N, ma, mf, n_rows):
     w = synth.workload(name)
     shape = replace(w.shape, n_layers=1)
     wt = synth.device_layer_weights(shape, w.seed, 0, dev())
-    lw = binding.LayerWeights.__new__(binding.LayerWeights)
-    lw.t = wt
-    lw.c = binding.LayerWeightsC(**{k: wt[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    lw = binding.LayerWeights.from_tensors(wt)
     wz = dict(wt)
     wz["w_down"] = torch.zeros_like(wt["w_down"])
-    lz = binding.LayerWeights.__new__(binding.LayerWeights)
-    lz.t = wz
-    lz.c = binding.LayerWeightsC(**{k: wz[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    lz = binding.LayerWeights.from_tensors(wz)
     X0, _ = synth.device_hidden_states(w, dev(), n_tokens=N)
     pos_h = np.arange(N, dtype=np.int32) * 2 + 3          # original positions need not be 0..N-1
     pos = torch.from_numpy(pos_h).to(dev())
@@ -164,9 +160,7 @@ def test_proxy_build_at_the_8b_layer_shape():
     from paper_2601_13155_b200 import binding
     shape = replace(synth.LLAMA8B, n_layers=1)
     wt = synth.device_layer_weights(shape, 1002, 0, dev())
-    lw = binding.LayerWeights.__new__(binding.LayerWeights)
-    lw.t = wt
-    lw.c = binding.LayerWeightsC(**{k: wt[k].data_ptr() for k in binding.WEIGHT_NAMES})
+    lw = binding.LayerWeights.from_tensors(wt)
     w = synth.workload("cfg2")
     Xc, _ = synth.device_hidden_states(w, dev(), n_tokens=2048)
     lib = binding.Spts(shape, max_seq=1024)
@@ -199,9 +193,7 @@ def test_decode_steps_at_the_8b_shape():
     layers, hostW = [], []
     for l in range(L):
         t = synth.device_layer_weights(shape, 1005, l, dev())
-        lw = binding.LayerWeights.__new__(binding.LayerWeights)
-        lw.t = t
-        lw.c = binding.LayerWeightsC(**{k: t[k].data_ptr() for k in binding.WEIGHT_NAMES})
+        lw = binding.LayerWeights.from_tensors(t)
         layers.append(lw)
         hostW.append(_host_weights(t))
     hw = synth.device_head_weights(shape, 1005, dev())

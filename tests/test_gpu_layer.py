@@ -83,6 +83,33 @@ def test_probes_match_oracle(shape, N, ma, mf, ref):
     lib.close()
 
 
+@pytest.mark.parametrize("shape,ref", [(SMALL_BF16, False), (SMALL_BF16, True), (synth.TINY, None),
+                                       (replace(SMALL_BF16, ltp_rank=48), False)])
+def test_prepared_layer_gives_the_same_bits(shape, ref):
+    """spts_prepare_layer moves the repacking of the proxy factors out of the calls; scores and layer outputs must
+    not change by a bit.  (The rank-48 shape takes the route without the Gram matrix in tensor-core mode.)"""
+    from paper_2601_13155_b200 import binding
+    lib = _mk(shape, 1024, ref)
+    N, ma, mf = 700, 300, 222
+    W, X, Wd = _layer_case(shape, N, 909, 16, std=0.05)
+    Wp = lib.prepare_layer(binding.LayerWeights(W, shape.dtype))
+    assert Wp.c.prepared and not Wd.c.prepared
+    pos = i32(np.arange(N))
+    outs = []
+    for lw in (Wd, Wp):
+        Xd = up(X, shape.dtype)
+        S = lib.pap_score(lw, Xd, pos)
+        Cd = torch.empty(N, dtype=torch.float32, device=dev())
+        Sf = lib.ltp_score(lw, Xd, S, C_out=Cd)
+        jf = torch.empty(mf, dtype=torch.int32, device=dev())
+        lib.layer_prefill_skip(lw, Xd, pos, ma, mf, binding.KvCache(shape, 1, N), idx_ffn_out=jf)
+        outs.append((Cd, Sf, jf, Xd))
+    assert lib.device_status() == 0
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    lib.close()
+
+
 @pytest.mark.parametrize("shape,N,ma,mf,ref", _modes())
 def test_layer_matches_oracle(shape, N, ma, mf, ref):
     from paper_2601_13155_b200 import binding

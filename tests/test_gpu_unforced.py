@@ -77,7 +77,7 @@ def test_config1_fp32_layer_unforced():
 # Bounds asserted for the unforced 8B-shaped layer (measured values are printed by the test; the design doc records them).
 CFG2_MAX_TF_DIFF_OUTSIDE_BAND = 8       # tokens of T_f (of 3277) on which GPU and oracle may disagree beyond the band (measured: 0)
 CFG2_MAX_FRACTION_BEYOND_TOL = 1e-3     # elements of the layer output beyond 2e-2 of the RMS (measured: 1.5e-4)
-CFG2_MAX_ERROR = 5e-2                   # largest error of any element, relative to the RMS (measured: 3.9e-2)
+CFG2_MAX_ERROR = 5e-2                   # largest error relative to the RMS, single rounding steps of large entries aside (measured: 3.9e-2)
 
 
 def test_config2_bf16_layer_unforced_reports_selection_and_flip_counts():
@@ -122,7 +122,12 @@ def test_config2_bf16_layer_unforced_reports_selection_and_flip_counts():
           f"({over.mean():.2e}) beyond 2e-2 of the RMS, in {len(rows_over)} of {len(same)} compared rows, first rows "
           f"{[int(same[r]) for r in rows_over[:12]]}")
     assert over.mean() <= CFG2_MAX_FRACTION_BEYOND_TOL
-    assert err.max() <= CFG2_MAX_ERROR * rms
+    # beyond the second bound only single rounding steps of large entries may remain (the x8 rows hold values up to
+    # ~30, where one bf16 step is 0.125 = 6e-2 of the RMS)
+    from parity_utils import bf16_ulp
+    step = bf16_ulp(np.maximum(np.maximum(np.abs(got), np.abs(ref)), np.abs(X[same])))
+    beyond = (err > CFG2_MAX_ERROR * rms) & (err > 1.001 * step)
+    assert not beyond.any(), f"{int(beyond.sum())} elements beyond {CFG2_MAX_ERROR} of the RMS and beyond one rounding step"
     if swaps_a == 0:
         check_output(host(cache.k[0][:ma]), want["K"], "bf16", what="cache K")
         check_output(host(cache.v[0][:ma]), want["V"], "bf16", what="cache V")
