@@ -29,6 +29,11 @@ struct Carver {
 
 size_t elt_size(const spts_model_desc& d) { return d.dtype == SPTS_BF16 ? 2 : 4; }
 
+// The SwiGLU intermediate [rows, Dff] is the widest buffer of a layer (28 KiB per row at the 8B shape).  The FFN block
+// therefore runs over chunks of this many selected rows: per chunk the weights stream once more (a few hundred MB
+// against ~6 TFLOP of work), and the workspace holds one chunk's intermediate instead of one row per candidate.
+constexpr int FFN_CHUNK_ROWS = 16384;
+
 bool shape_ok(const spts_model_desc& d) {
   if (d.hidden <= 0 || d.n_q_heads <= 0 || d.n_kv_heads <= 0 || d.ffn_dim <= 0) return false;
   if (d.n_q_heads % d.n_kv_heads != 0) return false;
@@ -83,7 +88,7 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   w.q_act = c.take<char>(Npad * HD * es);
   w.v_t = c.take<char>(KD * Npad * es);
   w.o_att = c.take<char>(Npad * HD * es);
-  w.hm = c.take<char>(Npad * (size_t)d.ffn_dim * es);
+  w.hm = c.take<char>((Npad < (size_t)FFN_CHUNK_ROWS ? Npad : (size_t)FFN_CHUNK_ROWS) * (size_t)d.ffn_dim * es);
   w.t1 = c.take<char>(Npad * 2 * (size_t)d.ltp_rank * es);
   w.hlow = c.take<char>(Npad * (size_t)d.ltp_dlow * es);
   w.t2 = c.take<char>(Npad * (size_t)d.ltp_rank * es);
@@ -390,18 +395,26 @@ spts_status ffn_gemms(spts_ctx* ctx, const spts_layer_weights* w, void* X, int N
   const auto& d = ctx->desc;
   Workspace& ws = ctx->ws;
   const int D = d.hidden;
-  const double Mf = (double)m_ffn, Dd = (double)D, esd = (double)elt_size(d);
-  Gemm g;
-  memset(&g, 0, sizeof(g));
-  g.A = X; g.lda = D; g.a_rows = N; g.idx = idx_f; g.W = w->w_gate; g.W2 = w->w_up; g.M = m_ffn; g.Nout = d.ffn_dim;
-  g.K = D; g.rowscale = ws.rstd; g.out = ws.hm; g.ldo = d.ffn_dim;
-  OP(SPTS_OP_GATEUP, 4.0 * Mf * Dd * d.ffn_dim, (Mf * Dd + Mf * d.ffn_dim + 2.0 * Dd * d.ffn_dim) * esd,
-     run_gemm(ctx, REF_SWIGLU, g));
-  memset(&g, 0, sizeof(g));
-  g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = m_ffn; g.dst_idx = idx_f; g.W = w->w_down; g.M = m_ffn; g.Nout = D;
-  g.K = d.ffn_dim; g.out = X; g.ldo = D;
-  OP(SPTS_OP_DOWN, 2.0 * Mf * Dd * d.ffn_dim, (Mf * d.ffn_dim + 2.0 * Mf * Dd + Dd * d.ffn_dim) * esd,
-     run_gemm(ctx, REF_RESID, g));
+  const double Dd = (double)D, esd = (double)elt_size(d);
+  const size_t row_bytes = (size_t)D * elt_size(d);
+  for (int c0 = 0; c0 < m_ffn; c0 += FFN_CHUNK_ROWS) {
+    const int mc = m_ffn - c0 < FFN_CHUNK_ROWS ? m_ffn - c0 : FFN_CHUNK_ROWS;
+    const double Mf = (double)mc;
+    // without an index list the chunk is rows [c0, c0 + mc) of X itself
+    char* xc = idx_f ? (char*)X : (char*)X + (size_t)c0 * row_bytes;
+    const int32_t* ic = idx_f ? idx_f + c0 : nullptr;
+    Gemm g;
+    memset(&g, 0, sizeof(g));
+    g.A = xc; g.lda = D; g.a_rows = idx_f ? N : mc; g.idx = ic; g.W = w->w_gate; g.W2 = w->w_up; g.M = mc; g.Nout = d.ffn_dim;
+    g.K = D; g.rowscale = idx_f ? ws.rstd : ws.rstd + c0; g.out = ws.hm; g.ldo = d.ffn_dim;
+    OP(SPTS_OP_GATEUP, 4.0 * Mf * Dd * d.ffn_dim, (Mf * Dd + Mf * d.ffn_dim + 2.0 * Dd * d.ffn_dim) * esd,
+       run_gemm(ctx, REF_SWIGLU, g));
+    memset(&g, 0, sizeof(g));
+    g.A = ws.hm; g.lda = d.ffn_dim; g.a_rows = mc; g.dst_idx = ic; g.W = w->w_down; g.M = mc; g.Nout = D;
+    g.K = d.ffn_dim; g.out = xc; g.ldo = D;
+    OP(SPTS_OP_DOWN, 2.0 * Mf * Dd * d.ffn_dim, (Mf * d.ffn_dim + 2.0 * Mf * Dd + Dd * d.ffn_dim) * esd,
+       run_gemm(ctx, REF_RESID, g));
+  }
   return SPTS_OK;
 }
 

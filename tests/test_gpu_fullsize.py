@@ -154,6 +154,12 @@ def test_bench_last_stage_dense_ragged_layer():
     _run_layer_case("cfg3", 11469, 11469, 11469, 256)
 
 
+def test_dense_layer_across_ffn_row_chunks():
+    """A dense layer a little longer than one FFN row chunk (16384 rows): the second chunk is a ragged tail of 300
+    rows, addressed without an index list."""
+    _run_layer_case("cfg3", 16384 + 300, 16384 + 300, 16384 + 300, 64)
+
+
 def test_proxy_build_at_the_8b_layer_shape():
     """spts_proxy_build at the LLaMA-3.1-8B layer shape ((D_low, r) = (512, 128), 14336 channels) on 2048 synthetic
     calibration tokens: importance in full, channel set, singular values and the rank-r products."""
