@@ -67,8 +67,6 @@ enum {
   SPTS_PAP_WINDOW = 8u,        /* spts_set_option: value = number of trailing queries the probe score averages over
                                   (1..64; 1 = last token only, Eq. 4; larger windows are the query-length ablation of
                                   Appendix C: every query attends causally, K and the queries are taken as stored) */
-  SPTS_ATTENTION_ONE_TILE = 4u, /* spts_set_option: tensor-core attention with one query tile per CTA (an older,
-                                  slower kernel kept as a cross-check of the two-tile kernel) */
   SPTS_DEBUG_CHECKS = 32u,     /* spts_set_option: after every selection a small kernel checks the index list
                                   (0 <= idx < N, strictly ascending) and records SPTS_ERR_INDEX in the device status
                                   word; nothing traps.  Off by default (one extra launch per selection) */
@@ -180,7 +178,7 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
                         size_t workspace_bytes, void* cuda_stream, spts_ctx** out);
 void spts_destroy(spts_ctx* ctx);
 
-/* Sets SPTS_REFERENCE_KERNELS, SPTS_ATTENTION_ONE_TILE, SPTS_FFN_SCORE_PAP_ONLY or SPTS_DEBUG_CHECKS on/off
+/* Sets SPTS_REFERENCE_KERNELS, SPTS_FFN_SCORE_PAP_ONLY or SPTS_DEBUG_CHECKS on/off
  * (value 0/1), or SPTS_PAP_WINDOW (value 1..64). */
 spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value);
 

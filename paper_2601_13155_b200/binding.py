@@ -14,12 +14,11 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libspts.so")
+LIB_PATH = os.environ.get("SPTS_LIBRARY") or os.path.join(_PKG, "libspts.so")     # SPTS_LIBRARY: another build of the library
 
 SPTS_BF16, SPTS_FP32 = 0, 1
 FORCE_LAST = 1
 OPT_REFERENCE_KERNELS = 2
-OPT_ATTENTION_ONE_TILE = 4
 OPT_PAP_WINDOW = 8
 OPT_FFN_SCORE_PAP_ONLY = 16
 OPT_DEBUG_CHECKS = 32
@@ -261,9 +260,6 @@ class Spts:
     def set_ffn_score_pap_only(self, on: bool):
         """T_f = TopK(S_mha, m_ffn): the FFN criterion without the proxy network (Table 4's baseline row)."""
         self._check(self.lib.spts_set_option(self.h, OPT_FFN_SCORE_PAP_ONLY, 1 if on else 0), "spts_set_option")
-
-    def set_attention_one_tile(self, on: bool):
-        self._check(self.lib.spts_set_option(self.h, OPT_ATTENTION_ONE_TILE, 1 if on else 0), "spts_set_option")
 
     def set_debug_checks(self, on: bool):
         """Every selected index list is checked on the device (range, strictly ascending); SPTS_ERR_INDEX otherwise."""

@@ -19,10 +19,6 @@
 //               row in registers: row maximum, p = 2^(s * log2(e)/sqrt(d) - max) with a lazily updated running maximum (O_t
 //               is rescaled in TMEM only when the maximum grows by more than 2^8), row sum, P_t
 //               written back to TMEM as packed bf16; at the end O_t / l goes to global memory.
-//
-// tc_attention_kernel (kept as a cross-check, option SPTS_ATTENTION_ONE_TILE): one CTA = 128 queries of
-// one head, P_j staged through shared memory; QK^T of block j+1 is issued before P_j V_j so the tensor
-// core works on S_{j+1} while the softmax warps process S_j.
 #include "spts_common.cuh"
 #include "tc_ptx.cuh"
 
@@ -34,19 +30,16 @@ namespace {
 
 using namespace ptx;
 
-constexpr int AT_THREADS = 192;
 constexpr int TILE = 128;                    // queries per CTA, keys per block, head dim
 constexpr int SLAB_BYTES = TILE * 128;       // [128 rows x 64 bf16] swizzled slab = 16 KiB
 constexpr int TILE_BYTES = 2 * SLAB_BYTES;   // 32 KiB
 constexpr int KV_STAGES = 2;
-constexpr int AT_SMEM = TILE_BYTES /*Q*/ + KV_STAGES * TILE_BYTES /*K*/ + KV_STAGES * TILE_BYTES /*V^T*/ +
-                        TILE_BYTES /*P*/ + 1024 + 256;
 constexpr int AT_TMEM_COLS = 512;
 constexpr float RESCALE_THRESHOLD = 8.0f;    // log2 units
 
 struct AttnParams {
   int m, H, Hkv;
-  int pair_tiles;   // paired kernel: 0 = the CTA's two tiles are two heads of one KV head, 1 = two query tiles of one head
+  int pair_tiles;   // 0 = the CTA's two tiles are two heads of one KV head, 1 = two query tiles of one head
   bf16* O;          // [m, H*128]
   int* status;
 };
@@ -62,258 +55,6 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__global__ void __launch_bounds__(AT_THREADS, 1)
-tc_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                    const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = base;
-  const uint32_t sK = sQ + TILE_BYTES;
-  const uint32_t sV = sK + KV_STAGES * TILE_BYTES;
-  const uint32_t sP = sV + KV_STAGES * TILE_BYTES;
-  const uint32_t bars = sP + TILE_BYTES;
-  // barrier block (8 bytes each)
-  const uint32_t q_full = bars;
-  const uint32_t k_full = bars + 8;          // [2]
-  const uint32_t k_free = bars + 24;         // [2]
-  const uint32_t v_full = bars + 40;         // [2]
-  const uint32_t v_free = bars + 56;         // [2]
-  const uint32_t s_full = bars + 72;         // [2]
-  const uint32_t s_free = bars + 88;         // [2]
-  const uint32_t p_full = bars + 104;
-  const uint32_t p_free = bars + 112;        // completes when P_j V_j is done
-  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  uint8_t* genP = gen + (sP - base);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + (bars - base) + 128);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.x;
-  const int qt = (int)gridDim.y - 1 - (int)blockIdx.y;      // longest tiles first
-  const int kvh = h / (p.H / p.Hkv);
-  const int nblk = qt + 1;
-  const uint64_t t0 = globaltimer_ns();
-
-  if (threadIdx.x == 0) {
-    *abort_flag = 0;
-    mbar_init(q_full, 1);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(k_full + 8 * s, 1); mbar_init(k_free + 8 * s, 1);
-      mbar_init(v_full + 8 * s, 1); mbar_init(v_free + 8 * s, 1);
-      mbar_init(s_full + 8 * s, 1); mbar_init(s_free + 8 * s, 128);
-    }
-    mbar_init(p_full, 128);
-    mbar_init(p_free, 1);
-    fence_mbar_init();
-    prefetch_tensormap(&tmQ); prefetch_tensormap(&tmK); prefetch_tensormap(&tmV);
-  }
-  if (warp == 1) {
-    tmem_alloc(smem_u32((const void*)tmem_slot), AT_TMEM_COLS);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tS = tmem_base;            // S buffers at columns [0,128) and [128,256)
-  const uint32_t tO = tmem_base + 256;      // O at columns [256,384)
-
-  if (warp == 0) {
-    if (lane == 0) {
-      mbar_expect_tx(q_full, TILE_BYTES);
-      tma_load_2d(sQ, &tmQ, q_full, h * TILE, qt * TILE);
-      tma_load_2d(sQ + SLAB_BYTES, &tmQ, q_full, h * TILE + 64, qt * TILE);
-      bool ok = true;
-      for (int j = 0; j < nblk && ok; ++j) {
-        const int s = j & 1;
-        const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-        ok = mbar_wait(k_free + 8 * s, ph ^ 1, abort_flag, t0);
-        if (!ok) break;
-        mbar_expect_tx(k_full + 8 * s, TILE_BYTES);
-        tma_load_2d(sK + s * TILE_BYTES, &tmK, k_full + 8 * s, kvh * TILE, j * TILE);
-        tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, k_full + 8 * s, kvh * TILE + 64, j * TILE);
-        ok = mbar_wait(v_free + 8 * s, ph ^ 1, abort_flag, t0);
-        if (!ok) break;
-        mbar_expect_tx(v_full + 8 * s, TILE_BYTES);
-        tma_load_2d(sV + s * TILE_BYTES, &tmV, v_full + 8 * s, j * TILE, kvh * TILE);
-        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, v_full + 8 * s, j * TILE + 64, kvh * TILE);
-      }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16(TILE, TILE);
-      bool ok = mbar_wait(q_full, 0, abort_flag, t0);
-      for (int j = 0; j <= nblk && ok; ++j) {
-        if (j < nblk) {      // S_j = Q K_j^T
-          const int s = j & 1;
-          const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-          ok = mbar_wait(k_full + 8 * s, ph, abort_flag, t0);
-          if (!ok) break;
-          ok = mbar_wait(s_free + 8 * s, ph ^ 1, abort_flag, t0);
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
-            mma_bf16(tS + s * TILE, smem_desc_sw128(sQ + off), smem_desc_sw128(sK + s * TILE_BYTES + off), idesc,
-                     k > 0 ? 1u : 0u);
-          }
-          mma_commit(s_full + 8 * s);
-          mma_commit(k_free + 8 * s);
-        }
-        if (j >= 1) {        // O += P_{j-1} V_{j-1}
-          const int jj = j - 1;
-          const int s = jj & 1;
-          ok = mbar_wait(v_full + 8 * s, (uint32_t)(jj >> 1) & 1u, abort_flag, t0);
-          if (!ok) break;
-          ok = mbar_wait(p_full, (uint32_t)jj & 1u, abort_flag, t0);
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t off = (k >> 2) * SLAB_BYTES + (k & 3) * 32;
-            mma_bf16(tO, smem_desc_sw128(sP + off), smem_desc_sw128(sV + s * TILE_BYTES + off), idesc,
-                     (jj > 0 || k > 0) ? 1u : 0u);
-          }
-          mma_commit(p_free);
-          mma_commit(v_free + 8 * s);
-        }
-      }
-    }
-  } else {
-    // ------------------------------------------------------------------ softmax / correction / epilogue
-    const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;               // row inside the tile
-    const int qi = qt * TILE + row;                    // compact query index
-    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const float sc = 0.08838834764831845f * 1.4426950408889634f;   // log2(e) / sqrt(128)
-    float m_used = -INFINITY, l = 0.f;
-    bool ok = true;
-    for (int j = 0; j < nblk && ok; ++j) {
-      const int s = j & 1;
-      ok = mbar_wait(s_full + 8 * s, (uint32_t)(j >> 1) & 1u, abort_flag, t0);
-      if (!ok) break;
-      tc_fence_after();
-      const uint32_t tSj = tS + s * TILE + lane_off;
-      const bool diag = (j == qt);
-      const int key0 = j * TILE;
-      // pass 1: row maximum
-      float bmax = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < TILE; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(tSj + c, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          float x = __uint_as_float(r[i]) * sc;
-          if (diag && key0 + c + i > qi) x = -INFINITY;
-          bmax = fmaxf(bmax, x);
-        }
-      }
-      float alpha = 1.0f;      // factor applied to O and l when the running maximum is replaced
-      if (bmax > m_used + RESCALE_THRESHOLD || m_used == -INFINITY) {
-        alpha = (m_used == -INFINITY) ? 0.0f : ex2(m_used - bmax);
-        m_used = bmax;
-      }
-      // pass 2: p = 2^(x - m), row sum, bf16 pack
-      uint32_t pk[64];
-      float psum = 0.f;
-#pragma unroll
-      for (int c = 0; c < TILE; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(tSj + c, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float x0 = __uint_as_float(r[i]) * sc - m_used;
-          float x1 = __uint_as_float(r[i + 1]) * sc - m_used;
-          if (diag && key0 + c + i > qi) x0 = -INFINITY;
-          if (diag && key0 + c + i + 1 > qi) x1 = -INFINITY;
-          float p0 = ex2(x0), p1 = ex2(x1);
-          psum += p0 + p1;
-          pk[(c + i) >> 1] = pack2(p0, p1);
-        }
-      }
-      l = l * alpha + psum;
-      tc_fence_before();
-      mbar_arrive(s_free + 8 * s);                     // S_j fully read
-      // P buffer and O are free once P_{j-1} V_{j-1} has completed
-      if (j >= 1) {
-        ok = mbar_wait(p_free, (uint32_t)(j - 1) & 1u, abort_flag, t0);
-        if (!ok) break;
-        tc_fence_after();
-        const bool need = __any_sync(0xffffffffu, alpha != 1.0f);
-        if (need) {
-#pragma unroll 1
-          for (int c = 0; c < TILE; c += 32) {
-            uint32_t r[32];
-            tmem_ld32(tO + lane_off + c, r);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            tmem_st32(tO + lane_off + c, r);
-          }
-          tmem_st_wait();
-        }
-      }
-      // write P_j (row `row`) into the 128B-swizzled K-major layout: two slabs of 64 keys
-      {
-        uint8_t* prow = genP + row * 128;
-#pragma unroll
-        for (int ch = 0; ch < 16; ++ch) {              // 16 chunks of 8 keys (16 bytes)
-          const int slab = ch >> 3, cc = ch & 7;
-          uint4 w = make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
-          *reinterpret_cast<uint4*>(prow + slab * SLAB_BYTES + ((cc ^ (row & 7)) << 4)) = w;
-        }
-      }
-      fence_proxy_async_smem();
-      tc_fence_before();
-      mbar_arrive(p_full);
-    }
-    // ---- epilogue: O / l
-    if (ok) ok = mbar_wait(p_free, (uint32_t)(nblk - 1) & 1u, abort_flag, t0);
-    if (ok) {
-      tc_fence_after();
-      const float inv = 1.0f / l;
-      bf16* orow = p.O + ((size_t)qi * p.H + h) * TILE;
-#pragma unroll 1
-      for (int c = 0; c < TILE; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(tO + lane_off + c, r);
-        tmem_ld_wait();
-        if (qi < p.m) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 w;
-            w.x = pack2(__uint_as_float(r[g * 8 + 0]) * inv, __uint_as_float(r[g * 8 + 1]) * inv);
-            w.y = pack2(__uint_as_float(r[g * 8 + 2]) * inv, __uint_as_float(r[g * 8 + 3]) * inv);
-            w.z = pack2(__uint_as_float(r[g * 8 + 4]) * inv, __uint_as_float(r[g * 8 + 5]) * inv);
-            w.w = pack2(__uint_as_float(r[g * 8 + 6]) * inv, __uint_as_float(r[g * 8 + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + c + g * 8) = w;
-          }
-        }
-      }
-    }
-  }
-
-  tc_fence_before();
-  __syncthreads();
-  if (*abort_flag) {
-    if (threadIdx.x == 0) set_status(p.status, SPTS_ERR_TIMEOUT);
-    const uint64_t t1 = globaltimer_ns();
-    while (globaltimer_ns() - t1 < 200000ull) { }
-    __syncthreads();
-  }
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem_base, AT_TMEM_COLS);
-  }
-}
-
-// ---------------------------------------------------------------------------------------------
-// paired-head kernel
-// ---------------------------------------------------------------------------------------------
 // Warp group 0: TMA warp, MMA warp, two warps with no role; warp groups 1 and 2: the softmax of tile 0 and of tile 1.
 // Registers live per SM sub-partition (16384 each, three warps of this block on every one), so an even split caps a
 // thread at 168.  The light warp group hands registers back (setmaxnreg works on whole warp groups, hence the two
@@ -627,8 +368,6 @@ bool make_map(spts_ctx* ctx, CUtensorMap* tm, const void* base, uint64_t rows, u
 spts_status tc_init(spts_ctx* ctx) {
   spts_status s = tc_gemm_init(ctx);
   if (s != SPTS_OK) return s;
-  if (cudaFuncSetAttribute(tc_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM) != cudaSuccess)
-    return SPTS_ERR_CUDA;
   if (cudaFuncSetAttribute(tc_attention_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AP_SMEM) != cudaSuccess)
     return SPTS_ERR_CUDA;
   return SPTS_OK;
@@ -648,16 +387,11 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
   if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)m, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
   AttnParams p;
   p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.pair_tiles = 0; p.O = O; p.status = ctx->ws.status;
-  if (!ctx->attn_one_tile) {
-    // two score tiles per CTA: two heads of one KV head when the GQA group is even, else two query tiles of a head
-    p.pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 0 : 1;
-    dim3 grid(p.pair_tiles ? d.n_q_heads : d.n_q_heads / 2,
-              p.pair_tiles ? ceil_div(ceil_div(m, TILE), 2) : ceil_div(m, TILE));
-    tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
-  } else {
-    dim3 grid(d.n_q_heads, ceil_div(m, TILE));
-    tc_attention_kernel<<<grid, AT_THREADS, AT_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
-  }
+  // two score tiles per CTA: two heads of one KV head when the GQA group is even, else two query tiles of a head
+  p.pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 0 : 1;
+  dim3 grid(p.pair_tiles ? d.n_q_heads : d.n_q_heads / 2,
+            p.pair_tiles ? ceil_div(ceil_div(m, TILE), 2) : ceil_div(m, TILE));
+  tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

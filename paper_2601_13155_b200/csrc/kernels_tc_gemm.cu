@@ -119,8 +119,7 @@ constexpr int GATHER_LAG = 2;        // k-blocks a gather thread keeps in flight
 
 // GATHER: the A rows are X[idx[i], :].  Warps 6..9 fetch them with 16-byte cp.async copies --
 // eight lanes per 128-byte row slice, written straight into the swizzled operand layout -- while
-// warp 0 keeps feeding W through TMA.  (A tile::gather4 TMA load does the same job in one
-// instruction per four rows, but was measured at a third of the tiled-load rate on this part.)
+// warp 0 keeps feeding W through TMA.
 template <int BN, int EPI, bool GATHER>
 __global__ void __launch_bounds__(GATHER ? GEMM_THREADS + 32 * GATHER_WARPS : GEMM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,

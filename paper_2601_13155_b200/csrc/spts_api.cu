@@ -448,7 +448,6 @@ spts_status spts_create(const spts_model_desc* desc, int max_seq, void* workspac
   ctx->launches = 0;
   ctx->sm_count = prop.multiProcessorCount;
   ctx->encode_tiled = nullptr;
-  ctx->attn_one_tile = false;
   ctx->ffn_score_pap_only = false;
   ctx->rstd_rows = nullptr;
   ctx->rope_trust = false;
@@ -525,10 +524,6 @@ spts_status spts_set_option(spts_ctx* ctx, uint32_t option, int value) {
   if (option == SPTS_PAP_WINDOW) {
     if (value < 1 || value > PAP_MAX_WINDOW) return SPTS_ERR_INVALID_ARG;
     ctx->pap_window = value;
-    return SPTS_OK;
-  }
-  if (option == SPTS_ATTENTION_ONE_TILE) {
-    ctx->attn_one_tile = value != 0;
     return SPTS_OK;
   }
   if (option == SPTS_DEBUG_CHECKS) {

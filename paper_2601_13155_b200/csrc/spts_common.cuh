@@ -94,7 +94,6 @@ struct spts_ctx {
   cudaStream_t stream;
   spts::Workspace ws;
   bool reference_kernels;   // plain CUDA-core kernels (always true in fp32 mode)
-  bool attn_one_tile;       // tensor-core attention: force the one-tile-per-CTA kernel
   bool ffn_score_pap_only;   // T_f from S_mha alone (no proxy FFN)
   bool debug_checks;        // every selected index list is checked on the device (SPTS_ERR_INDEX in the status word)
   char* ws_base;            // the caller's workspace and the byte offsets of the guard bands that follow its slices

@@ -18,7 +18,7 @@ SMALL_BF16 = replace(synth.LLAMA8B, hidden=512, n_q_heads=8, n_kv_heads=2, head_
                      ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
 
 
-# an odd GQA group (3 query heads per KV head): takes the one-tile attention kernel and the per-head decode attention
+# an odd GQA group (3 query heads per KV head): the attention kernel pairs two query tiles of one head; per-head decode attention
 ODD_GROUP_BF16 = replace(synth.LLAMA8B, hidden=384, n_q_heads=6, n_kv_heads=2, head_dim=128, ffn_dim=768,
                          ltp_dlow=128, ltp_rank=32, n_layers=1, vocab=1024)
 
@@ -246,24 +246,21 @@ def _attention_inputs(shape, m, kind, seed):
 
 
 @pytest.mark.parametrize("kind", ["normal", "peaky", "ramp"])
-@pytest.mark.parametrize("shape,m,ref,one_tile", [
-    pytest.param(SMALL_BF16, 1101, False, False, id="pair-kernel-even-group"),
-    pytest.param(SMALL_BF16, 1101, False, True, id="one-tile-kernel"),
-    pytest.param(ODD_GROUP_BF16, 600, False, False, id="pair-kernel-odd-group"),
-    pytest.param(WIDE_GROUP_BF16, 385, False, False, id="pair-kernel-group16"),
-    pytest.param(SMALL_BF16, 129, False, False, id="pair-kernel-one-past-a-tile"),
-    pytest.param(SMALL_BF16, 1, False, False, id="pair-kernel-single-row"),
-    pytest.param(SMALL_BF16, 300, True, False, id="plain-kernels-bf16"),
-    pytest.param(synth.TINY, 389, None, False, id="plain-kernels-fp32"),
+@pytest.mark.parametrize("shape,m,ref", [
+    pytest.param(SMALL_BF16, 1101, False, id="pair-kernel-even-group"),
+    pytest.param(ODD_GROUP_BF16, 600, False, id="pair-kernel-odd-group"),
+    pytest.param(WIDE_GROUP_BF16, 385, False, id="pair-kernel-group16"),
+    pytest.param(SMALL_BF16, 129, False, id="pair-kernel-one-past-a-tile"),
+    pytest.param(SMALL_BF16, 1, False, id="pair-kernel-single-row"),
+    pytest.param(SMALL_BF16, 300, True, id="plain-kernels-bf16"),
+    pytest.param(synth.TINY, 389, None, id="plain-kernels-fp32"),
 ])
-def test_reduced_attention_matches_oracle(shape, m, ref, one_tile, kind):
+def test_reduced_attention_matches_oracle(shape, m, ref, kind):
     """spts_reduced_attention (Algorithm 1's F_MHA(Q^, K^, V^) on the active rows) on operands of the test's choosing
-    against the oracle's causal GQA attention on the very same Q, K, V.  The tensor-core kernels keep their running
+    against the oracle's causal GQA attention on the very same Q, K, V.  The tensor-core kernel keeps its running
     row maximum lazily (O is rescaled only when the maximum has grown by more than 2^8); the "peaky" and "ramp"
     operands make that happen at almost every key block, in the regime where a wrong rescale would show."""
     lib = _mk(shape, 2048, ref)
-    if one_tile:
-        lib.set_attention_one_tile(True)
     Q, K, V = _attention_inputs(shape, m, kind, 4000 + m)
     got = lib.reduced_attention(up(Q, shape.dtype), up(K, shape.dtype), up(V, shape.dtype))
     assert lib.device_status() == 0
