@@ -5,6 +5,10 @@ records bench.py reports (profiles/traffic.json).  Runs where the report is read
       prints one line per captured launch: duration, DRAM bytes read / written, DRAM and tensor-pipe utilisation,
       registers per thread.
 
+  python -m paper_2601_13155_b200.ncu_summary --launch-list LAUNCHES.csv
+      the launch list of a whole run (the CSV log of `ncu --metrics gpu__time_duration.sum --csv --log-file ...`):
+      launches, total time and share per kernel.
+
   python -m paper_2601_13155_b200.ncu_summary REPORT.ncu-rep --traffic OP=KERNEL_REGEX[@INDEX] ... \
          --workload cfg3 --shape "m_ffn = 13108" --command "<the command that was profiled>"
       additionally records, for every OP given, dram__bytes_read.sum + dram__bytes_write.sum of the INDEX-th (default
@@ -100,7 +104,32 @@ def read_report(path):
     return launches
 
 
+def launch_list(path):
+    import collections
+    lines = [l for l in open(path) if l.startswith('"')]
+    agg = collections.OrderedDict()
+    for row in csv.DictReader(lines):
+        short = re.sub(r"^void ", "", row["Kernel Name"])
+        short = re.sub(r"spts::<unnamed>::", "", short)
+        short = re.sub(r"\(.*$", "", short)
+        if len(short) > 70:
+            short = short[:67] + "..."
+        a = agg.setdefault(short, [0, 0.0])
+        a[0] += 1
+        a[1] += float(row["Metric Value"].replace(",", ""))
+    tot = sum(v[1] for v in agg.values())
+    mine = {k: v for k, v in agg.items() if not k.startswith("at::") and "elementwise" not in k}
+    tm = sum(v[1] for v in mine.values())
+    print(f"all kernels: {sum(v[0] for v in agg.values())} launches, {tot / 1e6:.1f} ms; library kernels: "
+          f"{sum(v[0] for v in mine.values())} launches, {tm / 1e6:.1f} ms")
+    print(f"{'kernel':70s} {'launches':>8s} {'total ms':>10s} {'avg us':>9s} {'share':>7s}")
+    for k, v in sorted(mine.items(), key=lambda kv: -kv[1][1]):
+        print(f"{k:70s} {v[0]:8d} {v[1] / 1e6:10.3f} {v[1] / v[0] / 1e3:9.1f} {100 * v[1] / tm:6.2f}%")
+
+
 def main():
+    if len(sys.argv) == 3 and sys.argv[1] == "--launch-list":
+        return launch_list(sys.argv[2])
     ap = argparse.ArgumentParser()
     ap.add_argument("report")
     ap.add_argument("extra", nargs="*", help="further metric names to print")
