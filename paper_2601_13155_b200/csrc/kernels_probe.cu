@@ -66,14 +66,24 @@ __global__ void rope_table_kernel(const int32_t* __restrict__ pos, int N, int ha
 }
 
 // q[h, :] = RoPE(rstd * x_last . Wq[h*d + :, :]); one warp per rotary pair (j, j + d/2).
+// With `last_rows` (packed batch) block row y serves sequence y: x, rstd_last and cs_last then point at row 0 of the
+// packed arrays and the sequence's last row is looked up; q gets HD floats per sequence.
 template <typename T>
 __global__ void q_last_kernel(const T* __restrict__ x, const T* __restrict__ wq, int D, int d, int HD,
                               float rs_scale_dummy, const float* __restrict__ rstd_last,
-                              const float2* __restrict__ cs_last, float* __restrict__ q) {
+                              const float2* __restrict__ cs_last, float* __restrict__ q,
+                              const int32_t* __restrict__ seq_start) {
   constexpr int V = Vec16<T>::N;
   int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   int half = d >> 1;
   if (pair >= HD / 2) return;
+  if (seq_start != nullptr) {
+    const int last = seq_start[blockIdx.y + 1] - 1;
+    x += (size_t)last * D;
+    rstd_last += last;
+    cs_last += (size_t)last * half;
+    q += (size_t)blockIdx.y * HD;
+  }
   int lane = threadIdx.x & 31;
   int h = pair / half, i = pair - h * half;
   const T* w1 = wq + (size_t)(h * d + i) * D;
@@ -103,13 +113,10 @@ __global__ void q_last_kernel(const T* __restrict__ x, const T* __restrict__ wq,
 // token only); that query sees the keys n < N - w + 1 + query (causal).  `scale` multiplies the raw logits.
 __device__ __forceinline__ int pap_row_keys(int r, int N, int w, int G) { return N - w + 1 + (r % (w * G)) / G; }
 
-__global__ void __launch_bounds__(1024)
-pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N_all, int w, int G, float scale,
-                      float* __restrict__ stats) {
+// max and sum of exp of l[0..N) * scale -> out[0], out[1]; the whole block takes part
+__device__ __forceinline__ void head_stats_body(const float* __restrict__ l, int N, float scale, float* __restrict__ out) {
   __shared__ float red[32];
   __shared__ float bcast;
-  const float* l = logits + (size_t)blockIdx.x * ld;
-  const int N = pap_row_keys(blockIdx.x, N_all, w, G);
   int tid = threadIdx.x;
   float m = -INFINITY;
   for (int n = tid; n < N; n += blockDim.x) m = fmaxf(m, l[n] * scale);
@@ -132,7 +139,85 @@ pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N_all, int w
   if (tid < 32) {
     float v = tid < (blockDim.x >> 5) ? red[tid] : 0.f;
     v = warp_sum(v);
-    if (tid == 0) { stats[2 * blockIdx.x] = m; stats[2 * blockIdx.x + 1] = v; }
+    if (tid == 0) { out[0] = m; out[1] = v; }
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+pap_head_stats_kernel(const float* __restrict__ logits, int ld, int N_all, int w, int G, float scale,
+                      float* __restrict__ stats) {
+  head_stats_body(logits + (size_t)blockIdx.x * ld, pap_row_keys(blockIdx.x, N_all, w, G), scale, stats + 2 * blockIdx.x);
+}
+
+// Packed batch: block (h, b) takes head h over the rows of sequence b; stats [n_seq][H][2].  The same reduction, thread
+// for thread, as the single-sequence kernel runs on that sequence alone.
+__global__ void __launch_bounds__(1024)
+pap_head_stats_batch_kernel(const float* __restrict__ logits, int ld, const int32_t* __restrict__ seq_start,
+                            float* __restrict__ stats) {
+  const int s0 = seq_start[blockIdx.y];
+  head_stats_body(logits + (size_t)blockIdx.x * ld + s0, seq_start[blockIdx.y + 1] - s0, 1.0f,
+                  stats + 2 * ((size_t)blockIdx.y * gridDim.x + blockIdx.x));
+}
+
+// S[n] = (1/H) sum_h exp(l[h, n] - max_{b,h}) / sum_{b,h} with b the sequence of row n (Eq. 4 per prompt)
+__global__ void pap_mean_batch_kernel(const float* __restrict__ logits, int ld, int total, int H,
+                                      const int32_t* __restrict__ row_seq, const float* __restrict__ stats,
+                                      float* __restrict__ S) {
+  int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= total) return;
+  const float* st = stats + 2 * (size_t)row_seq[n] * H;
+  float acc = 0.f;
+  for (int r = 0; r < H; ++r) acc += expf(logits[(size_t)r * ld + n] * 1.0f - st[2 * r]) / st[2 * r + 1];
+  S[n] = acc * (1.0f / (float)H);
+}
+
+// row_seq[n] = the sequence that owns packed row n (seq_start ascending, n_seq + 1 entries)
+__global__ void batch_row_seq_kernel(const int32_t* __restrict__ seq_start, int n_seq, int total, int32_t* __restrict__ row_seq) {
+  int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= total) return;
+  int lo = 0, hi = n_seq;                     // seq_start[lo] <= n < seq_start[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (seq_start[mid] <= n) lo = mid; else hi = mid;
+  }
+  row_seq[n] = lo;
+}
+
+// vt_col[a] = column of the transposed V copy that active row a goes to: sequence b's columns start at vt0[b] (a
+// multiple of 8, so that a TMA box of that sequence starts on a 16-byte boundary)
+__global__ void batch_vt_col_kernel(const int32_t* __restrict__ act_off, const int32_t* __restrict__ vt0, int n_seq,
+                                    int n_act, int32_t* __restrict__ vt_col) {
+  int a = blockIdx.x * blockDim.x + threadIdx.x;
+  if (a >= n_act) return;
+  int lo = 0, hi = n_seq;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (act_off[mid] <= a) lo = mid; else hi = mid;
+  }
+  vt_col[a] = vt0[lo] + (a - act_off[lo]);
+}
+
+// The selected rows of every sequence go to that sequence's cache: K^ = K[T_a] and the positions by the (global)
+// index list, V^ from the packed projection output.  Active row a of the batch belongs to the sequence b with
+// act_off[b] <= a < act_off[b + 1] and is that cache's row a - act_off[b].  16 bytes per thread.
+struct BatchCachePtrs { void* const* k; void* const* v; int32_t* const* pos; };
+__global__ void batch_cache_fill_kernel(const uint4* __restrict__ k_all, const uint4* __restrict__ v_act,
+                                        const int32_t* __restrict__ pos, const int32_t* __restrict__ idx_global,
+                                        const int32_t* __restrict__ act_off, int n_seq, int n_act, int row_vec,
+                                        BatchCachePtrs c) {
+  const size_t total = (size_t)n_act * row_vec;
+  for (size_t t = (size_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (size_t)gridDim.x * blockDim.x) {
+    const int a = (int)(t / row_vec), e = (int)(t - (size_t)a * row_vec);
+    int lo = 0, hi = n_seq;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (act_off[mid] <= a) lo = mid; else hi = mid;
+    }
+    const int i = a - act_off[lo];
+    const int src = idx_global[a];
+    reinterpret_cast<uint4*>(c.k[lo])[(size_t)i * row_vec + e] = k_all[(size_t)src * row_vec + e];
+    reinterpret_cast<uint4*>(c.v[lo])[(size_t)i * row_vec + e] = v_act[(size_t)a * row_vec + e];
+    if (e == 0) c.pos[lo][i] = pos[src];
   }
 }
 
@@ -322,10 +407,10 @@ spts_status launch_q_last(spts_ctx* ctx, const void* X, const float2* cs, int N,
   dim3 grid(ceil_div(HD / 2, wpb));
   if (d.dtype == SPTS_BF16)
     q_last_kernel<bf16><<<grid, wpb * 32, 0, ctx->stream>>>((const bf16*)X + (size_t)(N - 1) * d.hidden,
-        (const bf16*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q);
+        (const bf16*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q, nullptr);
   else
     q_last_kernel<float><<<grid, wpb * 32, 0, ctx->stream>>>((const float*)X + (size_t)(N - 1) * d.hidden,
-        (const float*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q);
+        (const float*)wq, d.hidden, d.head_dim, HD, 0.f, rstd + (N - 1), cs + (size_t)(N - 1) * half, q, nullptr);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }
@@ -375,6 +460,59 @@ spts_status launch_transpose_bf16(spts_ctx* ctx, const void* in, int rows, int c
   if (rows <= 0 || cols <= 0) return SPTS_OK;
   transpose_bf16_kernel<<<dim3(ceil_div(cols, 32), ceil_div(rows, 32)), dim3(32, 8), 0, ctx->stream>>>(
       (const bf16*)in, rows, cols, (bf16*)out_t, ldt);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+// ---- packed batches (tensor-core mode): one launch per step over all sequences
+spts_status launch_batch_row_seq(spts_ctx* ctx, const int32_t* seq_start, int n_seq, int total, int32_t* row_seq) {
+  batch_row_seq_kernel<<<ceil_div(total, 256), 256, 0, ctx->stream>>>(seq_start, n_seq, total, row_seq);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_batch_vt_col(spts_ctx* ctx, const int32_t* act_off, const int32_t* vt0, int n_seq, int n_act, int32_t* vt_col) {
+  if (n_act <= 0) return SPTS_OK;
+  batch_vt_col_kernel<<<ceil_div(n_act, 256), 256, 0, ctx->stream>>>(act_off, vt0, n_seq, n_act, vt_col);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_q_last_batch(spts_ctx* ctx, const void* X, const float2* cs, const int32_t* seq_start, int n_seq,
+                                const void* wq, const float* rstd, float* q) {
+  const auto& d = ctx->desc;
+  if (d.dtype != SPTS_BF16) return SPTS_ERR_UNSUPPORTED;
+  const int HD = d.n_q_heads * d.head_dim;
+  const int wpb = 8;
+  dim3 grid(ceil_div(HD / 2, wpb), n_seq);
+  q_last_kernel<bf16><<<grid, wpb * 32, 0, ctx->stream>>>((const bf16*)X, (const bf16*)wq, d.hidden, d.head_dim, HD, 0.f,
+                                                          rstd, cs, q, seq_start);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_pap_softmax_batch(spts_ctx* ctx, const float* logits, int ld_logits, const int32_t* seq_start,
+                                     int n_seq, int total, const int32_t* row_seq, float* stats, float* S) {
+  const int H = ctx->desc.n_q_heads;
+  pap_head_stats_batch_kernel<<<dim3(H, n_seq), 1024, 0, ctx->stream>>>(logits, ld_logits, seq_start, stats);
+  SPTS_CUDA_OK(ctx);
+  pap_mean_batch_kernel<<<ceil_div(total, 256), 256, 0, ctx->stream>>>(logits, ld_logits, total, H, row_seq, stats, S);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
+spts_status launch_batch_cache_fill(spts_ctx* ctx, const void* k_all, const void* v_act, const int32_t* pos,
+                                    const int32_t* idx_global, const int32_t* act_off, int n_seq, int n_act,
+                                    void* const* k_ptrs, void* const* v_ptrs, int32_t* const* pos_ptrs) {
+  const auto& d = ctx->desc;
+  const int row_vec = d.n_kv_heads * d.head_dim * 2 / 16;
+  if (n_act <= 0) return SPTS_OK;
+  size_t total = (size_t)n_act * row_vec;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+  BatchCachePtrs c{k_ptrs, v_ptrs, pos_ptrs};
+  batch_cache_fill_kernel<<<blocks, 256, 0, ctx->stream>>>((const uint4*)k_all, (const uint4*)v_act, pos, idx_global, act_off,
+                                                           n_seq, n_act, row_vec, c);
   SPTS_CUDA_OK(ctx);
   return SPTS_OK;
 }

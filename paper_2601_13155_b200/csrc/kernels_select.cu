@@ -268,7 +268,119 @@ __global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t
   if (i < n) dst[i] = src[idx[i]];
 }
 
+// ---- one selection per sequence of a packed batch, one CTA each (sequences of up to TOPK_SEG_MAX scores: the keys
+// sit in shared memory).  Same rule as the kernels above: 8-bit radix select on the order-preserving keys finds the
+// k-th largest key and how many of the keys equal to it are taken (the ones with the lowest indices), then the
+// selected indices are written in ascending order -- numbered from the sequence's own first row into out_local
+// (optional) and from the batch's first row into out_global (optional), at out_off[b].
+constexpr int SEG_THREADS = 512;
+__global__ void __launch_bounds__(SEG_THREADS)
+topk_segmented_kernel(const float* __restrict__ scores, const int32_t* __restrict__ seq_start,
+                      const int32_t* __restrict__ k_arr, const int32_t* __restrict__ out_off, int force_last,
+                      int32_t* __restrict__ out_local, int32_t* __restrict__ out_global, int* status) {
+  extern __shared__ uint32_t seg_keys[];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t scan[256];
+  __shared__ uint32_t s_prefix, s_krem;
+  __shared__ uint32_t wsum_gt[SEG_THREADS / 32], wsum_eq[SEG_THREADS / 32];
+  __shared__ uint32_t carry_gt, carry_eq;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int b = blockIdx.x;
+  const int s0 = seq_start[b];
+  const int N = seq_start[b + 1] - s0;
+  const int k = k_arr[b];
+  const int o0 = out_off[b];
+  const float* sc = scores + s0;
+  if (k >= N) {                                  // TopK of everything: the identity list
+    for (int i = tid; i < N; i += SEG_THREADS) {
+      if (out_local) out_local[o0 + i] = i;
+      if (out_global) out_global[o0 + i] = s0 + i;
+    }
+    return;
+  }
+  bool nonfinite = false;
+  for (int i = tid; i < N; i += SEG_THREADS) seg_keys[i] = load_key(sc, i, N, force_last != 0, &nonfinite);
+  if (nonfinite) set_status(status, SPTS_ERR_NONFINITE);
+  if (tid == 0) { s_prefix = 0u; s_krem = (uint32_t)k; }
+  __syncthreads();
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    const uint32_t mask = pass == 0 ? 0u : (0xFFFFFFFFu << (32 - 8 * pass));
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    for (int i = tid; i < N; i += SEG_THREADS) {
+      const uint32_t key = seg_keys[i];
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFFu], 1u);
+    }
+    __syncthreads();
+    // inclusive scan from the top digit downwards: scan[t] = sum of hist[255 - t .. 255]
+    uint32_t mine = 0u;
+    if (tid < 256) { mine = hist[255 - tid]; scan[tid] = mine; }
+    __syncthreads();
+    for (int o = 1; o < 256; o <<= 1) {
+      uint32_t v = (tid < 256 && tid >= o) ? scan[tid - o] : 0u;
+      __syncthreads();
+      if (tid < 256) scan[tid] += v;
+      __syncthreads();
+    }
+    const uint32_t krem = s_krem;
+    __syncthreads();
+    if (tid < 256) {
+      const uint32_t above = scan[tid] - mine;    // keys in strictly higher buckets
+      if (above < krem && krem <= scan[tid]) {    // exactly one thread
+        s_prefix = prefix | ((uint32_t)(255 - tid) << shift);
+        s_krem = krem - above;
+      }
+    }
+    __syncthreads();
+  }
+  const uint32_t thr = s_prefix, take_eq = s_krem;
+  if (tid == 0) { carry_gt = 0u; carry_eq = 0u; }
+  __syncthreads();
+  // ascending emit: element i goes to (keys above the threshold before it) + (taken equals before it)
+  for (int base = 0; base < N; base += SEG_THREADS) {
+    const int i = base + tid;
+    const uint32_t key = i < N ? seg_keys[i] : 0u;
+    const bool gt = i < N && key > thr, eq = i < N && key == thr;
+    const uint32_t bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) { wsum_gt[wid] = __popc(bg); wsum_eq[wid] = __popc(be); }
+    __syncthreads();
+    uint32_t pre_gt = carry_gt, pre_eq = carry_eq;
+    for (int w = 0; w < wid; ++w) { pre_gt += wsum_gt[w]; pre_eq += wsum_eq[w]; }
+    const uint32_t lt = (1u << lane) - 1u;
+    pre_gt += __popc(bg & lt);
+    pre_eq += __popc(be & lt);
+    if (gt || (eq && pre_eq < take_eq)) {
+      const uint32_t pos = pre_gt + (pre_eq < take_eq ? pre_eq : take_eq);
+      if (out_local) out_local[o0 + pos] = i;
+      if (out_global) out_global[o0 + pos] = s0 + i;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t g = 0u, e = 0u;
+      for (int w = 0; w < SEG_THREADS / 32; ++w) { g += wsum_gt[w]; e += wsum_eq[w]; }
+      carry_gt += g;
+      carry_eq += e;
+    }
+    __syncthreads();
+  }
+}
+
 }  // namespace
+
+spts_status launch_topk_segmented(spts_ctx* ctx, const float* scores, const int32_t* seq_start, const int32_t* k_arr,
+                                  const int32_t* out_off, int n_seq, int max_len, uint32_t flags, int32_t* out_local,
+                                  int32_t* out_global) {
+  if (n_seq <= 0) return SPTS_OK;
+  if (max_len > TOPK_SEG_MAX) return SPTS_ERR_SHAPE;
+  const size_t smem = (size_t)max_len * sizeof(uint32_t);
+  topk_segmented_kernel<<<n_seq, SEG_THREADS, smem, ctx->stream>>>(scores, seq_start, k_arr, out_off,
+                                                                  (flags & SPTS_FORCE_LAST) ? 1 : 0, out_local, out_global,
+                                                                  ctx->ws.status);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
 
 spts_status launch_topk(spts_ctx* ctx, const float* scores, int N, int k, uint32_t flags,
                         int32_t* idx_out, uint32_t* scratch) {

@@ -56,6 +56,8 @@ struct TcParams {
   bf16* out_t; int ldt;
   const float2* cs;             // rotary table [rows, 64]
   const float* q; float* logits; int ld_logits; int group;
+  const int32_t* row_seq; int q_stride;   // packed batch: row -> sequence, and the distance between two sequences' q
+  const int32_t* out_t_col;     // TC_STORE: column of out_t a row goes to (nullptr: the row's own number)
   float* csq; int csq_parts;
   float* out_f32;               // TC_STORE: write fp32 [M, ldo] instead of the bf16 tile
   float* sal_t; int ld_sal;     // TC_SWIGLU: write |silu(g) u| as fp32 [column, row] instead of the bf16 tile
@@ -311,9 +313,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             store32_bf16(p.out + (size_t)grow * p.ldo + n0 + c, v, n0 + c, p.Nout);
             if (p.out_t != nullptr) {
+              const int tcol = p.out_t_col ? p.out_t_col[grow] : grow;
 #pragma unroll
               for (int i = 0; i < 32; ++i)
-                if (n0 + c + i < p.Nout) p.out_t[(size_t)(n0 + c + i) * p.ldt + grow] = __float2bfloat16_rn(v[i]);
+                if (n0 + c + i < p.Nout) p.out_t[(size_t)(n0 + c + i) * p.ldt + tcol] = __float2bfloat16_rn(v[i]);
             }
           }
         }
@@ -378,10 +381,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               store32_bf16(o + 64, b, 0, 32);
               if (p.logits != nullptr) {
                 const int kvh = hcol >> 7;
+                // packed batch: every sequence is probed with its own last token's query
+                const float* qseq = p.q + (p.row_seq ? (size_t)p.row_seq[src] * p.q_stride : 0);
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
                   if (g < p.group) {
-                    const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
+                    const float* qh = qseq + (size_t)(kvh * p.group + g) * 128 + jj * 32;
                     float d = dots[hh][g];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
@@ -391,7 +396,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 // query heads beyond the eight kept in registers (GQA groups larger than 8): their partial sums
                 // over this half of the frequencies go through the logits row itself (same thread, same address)
                 for (int g = 8; g < p.group; ++g) {
-                  const float* qh = p.q + (size_t)(kvh * p.group + g) * 128 + jj * 32;
+                  const float* qh = qseq + (size_t)(kvh * p.group + g) * 128 + jj * 32;
                   float d = 0.f;
 #pragma unroll
                   for (int i = 0; i < 32; ++i) d = fmaf(a[i], __ldg(qh + i), fmaf(b[i], __ldg(qh + 64 + i), d));
@@ -590,6 +595,7 @@ spts_status launch_one_g(spts_ctx* ctx, const TcGemmArgs& a) {
   p.cs = ctx->ws.rope_cs; p.q = a.q; p.logits = a.logits; p.ld_logits = a.ld_logits; p.group = a.group;
   p.csq = a.csq; p.csq_parts = a.csq_parts; p.status = ctx->ws.status;
   p.sal_t = a.sal_t; p.ld_sal = a.ld_sal; p.out_f32 = a.out_f32;
+  p.row_seq = a.row_seq; p.q_stride = a.q_stride; p.out_t_col = a.out_t_col;
   p.num_m = ceil_div(a.M, BM);
   p.num_n = ceil_div(a.Nout, NT);
   {

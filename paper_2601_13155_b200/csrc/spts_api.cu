@@ -61,7 +61,11 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   const size_t Npad = align_up(N, 128);
   w.status = c.take<int>(64);
   w.rstd = c.take<float>(N);
-  w.q = c.take<float>(HD);
+  w.q = c.take<float>(HD * (size_t)BATCH_MAX_SEQ);          // one probe query per sequence of a packed batch
+  w.batch_i32 = c.take<int32_t>(6 * (size_t)(BATCH_MAX_SEQ + 1));
+  w.batch_ptr = c.take<void*>(3 * (size_t)BATCH_MAX_SEQ);
+  w.row_seq = c.take<int32_t>(N);
+  w.vt_col = c.take<int32_t>(Npad);
   w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
   w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
   w.ugu = c.take<char>(2 * (size_t)d.ltp_rank * d.hidden * es);
@@ -75,7 +79,7 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
     w.idx_w = c.take<int32_t>(PAP_MAX_WINDOW);
   }
   w.logits = c.take<float>((size_t)d.n_q_heads * Npad);
-  w.head_stats = c.take<float>(2 * (size_t)d.n_q_heads);
+  w.head_stats = c.take<float>(2 * (size_t)d.n_q_heads * BATCH_MAX_SEQ);
   w.s_mha = c.take<float>(N);
   w.s_ffn = c.take<float>(N);
   w.csq_parts = ceil_div(d.hidden, 64);
@@ -86,7 +90,8 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   w.topk_scratch = c.take<uint32_t>(TOPK_SCRATCH_WORDS);
   w.k_all = c.take<char>(N * KD * es);
   w.q_act = c.take<char>(Npad * HD * es);
-  w.v_t = c.take<char>(KD * Npad * es);
+  w.vt_ld_max = (int)(Npad + 8 * (size_t)BATCH_MAX_SEQ);     // a packed batch starts every sequence's columns on a multiple of 8
+  w.v_t = c.take<char>(KD * (size_t)w.vt_ld_max * es);
   w.o_att = c.take<char>(Npad * HD * es);
   w.hm = c.take<char>((Npad < (size_t)FFN_CHUNK_ROWS ? Npad : (size_t)FFN_CHUNK_ROWS) * (size_t)d.ffn_dim * es);
   w.t1 = c.take<char>(Npad * 2 * (size_t)d.ltp_rank * es);
@@ -418,6 +423,105 @@ spts_status ffn_gemms(spts_ctx* ctx, const spts_layer_weights* w, void* X, int N
   return SPTS_OK;
 }
 
+// The attention blocks of a packed batch with one launch per step instead of one per step and sequence (tensor-core
+// mode, probe window 1, at most BATCH_MAX_SEQ sequences of at most TOPK_SEG_MAX rows): the row statistics, the
+// rotary table, every sequence's last-token query, the K projection with each row probed by its own sequence's
+// query, the per-sequence softmax of Eq. 4 and TopK of Eq. 5, the Q / V projections of all selected rows and the O
+// projection run once over the packed rows; only the causal attention itself is launched per sequence.  Every row
+// gets the bits the single-sequence call gives it.
+spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos, int n_seq,
+                                   const int32_t* seq_start, const int32_t* m_attn, uint32_t flags, spts_kv_layer* caches,
+                                   float* S, int32_t* idx_attn_out) {
+  const auto& d = ctx->desc;
+  Workspace& ws = ctx->ws;
+  const int D = d.hidden, HD = d.n_q_heads * d.head_dim, KD = d.n_kv_heads * d.head_dim;
+  const int total = seq_start[n_seq];
+  const size_t es = elt_size(d);
+  // host tables: seq_start | m_attn | act_off | vt0, and the caches' pointers
+  std::vector<int32_t> tab((size_t)4 * (n_seq + 1), 0);
+  int32_t* h_start = tab.data();
+  int32_t* h_m = h_start + (n_seq + 1);
+  int32_t* h_off = h_m + (n_seq + 1);
+  int32_t* h_vt0 = h_off + (n_seq + 1);
+  std::vector<void*> ptrs((size_t)3 * n_seq);
+  int A = 0, vt = 0, max_len = 0;
+  for (int b = 0; b < n_seq; ++b) {
+    h_start[b] = seq_start[b]; h_m[b] = m_attn[b]; h_off[b] = A; h_vt0[b] = vt;
+    A += m_attn[b];
+    vt += (m_attn[b] + 7) & ~7;
+    const int len = seq_start[b + 1] - seq_start[b];
+    max_len = len > max_len ? len : max_len;
+    ptrs[b] = caches[b].k; ptrs[n_seq + b] = caches[b].v; ptrs[2 * n_seq + b] = caches[b].pos;
+  }
+  h_start[n_seq] = total; h_off[n_seq] = A;
+  const int ldvt = (int)align_up((size_t)vt, 128);
+  if (ldvt > ws.vt_ld_max) return SPTS_ERR_WORKSPACE;
+  int32_t* d_start = ws.batch_i32;
+  int32_t* d_m = d_start + (n_seq + 1);
+  int32_t* d_off = d_m + (n_seq + 1);
+  int32_t* d_vt0 = d_off + (n_seq + 1);
+  if (cudaMemcpyAsync(d_start, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess ||
+      cudaMemcpyAsync(ws.batch_ptr, ptrs.data(), ptrs.size() * sizeof(void*), cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
+    return SPTS_ERR_CUDA;
+  const double Nd = (double)total, Dd = (double)D, esd = (double)es, Ad = (double)A;
+  const int ld = (int)align_up((size_t)total, 128);
+  // ---- probe (Eq. 4), per sequence
+  OP(SPTS_OP_PREP, 0.0, Nd * Dd * esd + 4.0 * Nd, launch_rstd(ctx, X, total, ws.rstd));
+  ctx->rope_trust = false;
+  OP(SPTS_OP_PREP, 0.0, Nd * (4.0 + 4.0 * d.head_dim), launch_rope_table(ctx, pos, total, ws.rope_cs));
+  TRY(launch_batch_row_seq(ctx, d_start, n_seq, total, ws.row_seq));
+  OP(SPTS_OP_PREP, 2.0 * n_seq * Dd * HD, Dd * HD * esd, launch_q_last_batch(ctx, X, ws.rope_cs, d_start, n_seq, w->wq, ws.rstd, ws.q));
+  {
+    TcGemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = (const bf16*)X; a.lda = D; a.a_rows = total; a.W = (const bf16*)w->wk; a.M = total; a.Nout = KD; a.K = D;
+    a.rowscale = ws.rstd; a.out = (bf16*)ws.k_all; a.ldo = KD; a.q = ws.q; a.logits = ws.logits; a.ld_logits = ld;
+    a.group = d.n_q_heads / d.n_kv_heads; a.row_seq = ws.row_seq; a.q_stride = HD; a.csq_parts = ws.csq_parts;
+    OP(SPTS_OP_KPROJ, 2.0 * Nd * Dd * KD, (Nd * Dd + Nd * KD + Dd * KD) * esd, launch_tc_gemm(ctx, TC_ROPE, a));
+  }
+  OP(SPTS_OP_PAP_SOFTMAX, 0.0, Nd * 4.0 * (2.0 * d.n_q_heads + 1.0),
+     launch_pap_softmax_batch(ctx, ws.logits, ld, d_start, n_seq, total, ws.row_seq, ws.head_stats, S));
+  // ---- TopK (Eq. 5) per sequence: lists numbered within the sequence for the caller, within the batch for the gathers
+  OP(SPTS_OP_TOPK, 0.0, 4.0 * Nd + 4.0 * Ad,
+     launch_topk_segmented(ctx, S, d_start, d_m, d_off, n_seq, max_len, flags, idx_attn_out, ws.idx_a));
+  if (ctx->debug_checks) TRY(launch_check_index_list(ctx, ws.idx_a, A, total));
+  TRY(launch_batch_vt_col(ctx, d_off, d_vt0, n_seq, A, ws.vt_col));
+  // ---- Q and V of the selected rows; V goes through the (still unused) attention-output buffer to the caches
+  {
+    TcGemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = (const bf16*)X; a.lda = D; a.a_rows = total; a.idx = ws.idx_a; a.W = (const bf16*)w->wq; a.M = A; a.Nout = HD; a.K = D;
+    a.rowscale = ws.rstd; a.out = (bf16*)ws.q_act; a.ldo = HD; a.group = d.n_q_heads / d.n_kv_heads; a.csq_parts = ws.csq_parts;
+    OP(SPTS_OP_QVPROJ, 2.0 * Ad * Dd * HD, (Ad * Dd + Ad * HD + Dd * HD) * esd, launch_tc_gemm(ctx, TC_ROPE, a));
+    a.W = (const bf16*)w->wv; a.Nout = KD; a.out = (bf16*)ws.o_att; a.ldo = KD;
+    a.out_t = (bf16*)ws.v_t; a.ldt = ldvt; a.out_t_col = ws.vt_col;
+    OP(SPTS_OP_QVPROJ, 2.0 * Ad * Dd * KD, (Ad * Dd + 2.0 * Ad * KD + Dd * KD) * esd, launch_tc_gemm(ctx, TC_STORE, a));
+  }
+  OP(SPTS_OP_KV_GATHER, 0.0, 4.0 * Ad * (double)KD * esd + 12.0 * Ad,
+     launch_batch_cache_fill(ctx, ws.k_all, ws.o_att, pos, ws.idx_a, d_off, n_seq, A, ws.batch_ptr, ws.batch_ptr + n_seq,
+                             (int32_t* const*)(ws.batch_ptr + 2 * n_seq)));
+  // ---- causal attention, one launch per sequence (Algorithm 1: F_MHA on each prompt's own active rows)
+  {
+    double fl = 0.0;
+    for (int b = 0; b < n_seq; ++b) fl += 2.0 * HD * (double)m_attn[b] * (m_attn[b] + 1.0);
+    ProfScope ps(ctx, SPTS_OP_ATTN, fl, (2.0 * Ad * HD + 2.0 * Ad * KD) * esd);
+    for (int b = 0; b < n_seq; ++b) {
+      TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act + (size_t)h_off[b] * HD, (const bf16*)caches[b].k,
+                              (const bf16*)caches[b].v, (const bf16*)ws.v_t + h_vt0[b], ldvt, m_attn[b],
+                              (bf16*)ws.o_att + (size_t)h_off[b] * HD));
+      caches[b].len = m_attn[b];
+    }
+  }
+  {
+    TcGemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.A = (const bf16*)ws.o_att; a.lda = HD; a.a_rows = A; a.dst_idx = ws.idx_a; a.W = (const bf16*)w->wo; a.M = A; a.Nout = D; a.K = HD;
+    a.out = (bf16*)X; a.ldo = D; a.csq_parts = ws.csq_parts;
+    OP(SPTS_OP_OPROJ, 2.0 * Ad * Dd * HD, (Ad * HD + 2.0 * Ad * Dd + Dd * HD) * esd, launch_tc_gemm(ctx, TC_RESID, a));
+  }
+  return SPTS_OK;
+}
+
 spts_status check_ctx(const spts_ctx* ctx) { return ctx == nullptr ? SPTS_ERR_INVALID_ARG : SPTS_OK; }
 
 }  // namespace
@@ -713,6 +817,33 @@ spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weight
   Workspace& ws = ctx->ws;
   const size_t row_bytes = (size_t)d.hidden * elt_size(d);
   float* S = S_mha_out ? S_mha_out : ws.s_mha;
+  int max_len = 0;
+  for (int b = 0; b < n_seq; ++b) max_len = seq_start[b + 1] - seq_start[b] > max_len ? seq_start[b + 1] - seq_start[b] : max_len;
+  const bool one_launch_per_step = use_tc(ctx) && n_seq <= BATCH_MAX_SEQ && max_len <= TOPK_SEG_MAX && ctx->pap_window < 2;
+  if (one_launch_per_step) {
+    TRY(batch_attention_blocks(ctx, w, X, pos, n_seq, seq_start, m_attn, flags, caches, S, idx_attn_out));
+    OP(SPTS_OP_PREP, 0.0, (double)total * (double)row_bytes + 4.0 * total, launch_rstd(ctx, X, total, ws.rstd));
+    const float* s_sel = S;
+    if (any_sel_f && !ctx->ffn_score_pap_only) {
+      TRY(ltp_pipeline(ctx, w, X, S, total, nullptr, ws.s_ffn));
+      s_sel = ws.s_ffn;
+    }
+    // TopK of Eq. 15 per sequence in one launch; the tables of budgets and offsets follow the attention block's
+    std::vector<int32_t> tab((size_t)2 * (n_seq + 1), 0);
+    int F = 0;
+    for (int b = 0; b < n_seq; ++b) { tab[b] = m_ffn[b]; tab[n_seq + 1 + b] = F; F += m_ffn[b]; }
+    tab[2 * n_seq + 1] = F;
+    int32_t* d_mf = ws.batch_i32 + 4 * (n_seq + 1);
+    int32_t* d_foff = d_mf + (n_seq + 1);
+    if (any_sel_f || idx_ffn_out != nullptr) {
+      if (cudaMemcpyAsync(d_mf, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
+        return SPTS_ERR_CUDA;
+      OP(SPTS_OP_TOPK, 0.0, 4.0 * total + 4.0 * F,
+         launch_topk_segmented(ctx, s_sel, ws.batch_i32, d_mf, d_foff, n_seq, max_len, flags, idx_ffn_out, ws.idx_f));
+      if (ctx->debug_checks && any_sel_f) TRY(launch_check_index_list(ctx, ws.idx_f, F, total));
+    }
+    return ffn_gemms(ctx, w, X, total, any_sel_f ? ws.idx_f : nullptr, F);
+  }
   // ---- attention blocks, one sequence after the other: the probe's softmax, the selection and the causal mask
   //      are per sequence.  The rotary table is rebuilt for every slice.
   int off_a = 0;

@@ -84,6 +84,12 @@ struct Workspace {
   float* logits_v;      // [vocab]
   void* xrow;           // [D] one hidden row in the storage type
   int csq_parts;
+  // packed batches: host tables copied in per call, row -> sequence map, V^T column of every active row
+  int32_t* batch_i32;   // [6 * (BATCH_MAX_SEQ + 1)]
+  void** batch_ptr;     // [3 * BATCH_MAX_SEQ] cache pointers (k, v, pos)
+  int32_t* row_seq;     // [Nmax]
+  int32_t* vt_col;      // [Nmax]
+  int vt_ld_max;        // columns of v_t
 };
 
 }  // namespace spts
@@ -114,6 +120,7 @@ struct spts_ctx {
 
 namespace spts {
 
+static const int BATCH_MAX_SEQ = 1024;        // sequences per packed batch that take the one-launch-per-step route
 static const int PAP_MAX_WINDOW = 64;         // largest query window of the probe (the paper ablates 1, 4 and 64)
 
 // top-k scratch size in uint32 words
@@ -128,6 +135,10 @@ spts_status launch_gather_rows(spts_ctx* ctx, const void* src, const int32_t* id
                                int row_bytes, void* dst);
 spts_status launch_gather_i32(spts_ctx* ctx, const int32_t* src, const int32_t* idx, int n, int32_t* dst);
 spts_status launch_offset_i32(spts_ctx* ctx, const int32_t* src, int n, int offset, int32_t* dst);
+static const int TOPK_SEG_MAX = 8192;         // longest sequence the one-CTA-per-sequence selection takes
+spts_status launch_topk_segmented(spts_ctx* ctx, const float* scores, const int32_t* seq_start, const int32_t* k_arr,
+                                  const int32_t* out_off, int n_seq, int max_len, uint32_t flags, int32_t* out_local,
+                                  int32_t* out_global);
 spts_status launch_check_index_list(spts_ctx* ctx, const int32_t* idx, int n, int N);   // debug option only
 spts_status launch_wait_selftest(spts_ctx* ctx, uint32_t limit_us);
 
@@ -146,6 +157,15 @@ spts_status launch_pap_softmax(spts_ctx* ctx, const float* logits, int ld_logits
 spts_status launch_pap_window_softmax(spts_ctx* ctx, const float* logits, int ld_logits, int N, int w, int accumulate,
                                       float* stats, float* S);
 spts_status launch_pap_regroup(spts_ctx* ctx, const void* q_win, int w, void* q_kv);
+spts_status launch_batch_vt_col(spts_ctx* ctx, const int32_t* act_off, const int32_t* vt0, int n_seq, int n_act, int32_t* vt_col);
+spts_status launch_batch_row_seq(spts_ctx* ctx, const int32_t* seq_start, int n_seq, int total, int32_t* row_seq);
+spts_status launch_q_last_batch(spts_ctx* ctx, const void* X, const float2* cs, const int32_t* seq_start, int n_seq,
+                                const void* wq, const float* rstd, float* q);
+spts_status launch_pap_softmax_batch(spts_ctx* ctx, const float* logits, int ld_logits, const int32_t* seq_start,
+                                     int n_seq, int total, const int32_t* row_seq, float* stats, float* S);
+spts_status launch_batch_cache_fill(spts_ctx* ctx, const void* k_all, const void* v_act, const int32_t* pos,
+                                    const int32_t* idx_global, const int32_t* act_off, int n_seq, int n_act,
+                                    void* const* k_ptrs, void* const* v_ptrs, int32_t* const* pos_ptrs);
 spts_status launch_iota_from(spts_ctx* ctx, int32_t* out, int n, int first);
 spts_status launch_transpose_bf16(spts_ctx* ctx, const void* in, int rows, int cols, void* out_t, int ldt);
 spts_status launch_ffn_score(spts_ctx* ctx, const float* csq, int parts, const float* S_mha, int N,
@@ -215,6 +235,8 @@ struct TcGemmArgs {
   float* sal_t; int ld_sal;             // TC_SWIGLU: saliency output (proxy construction)
   int ldw;                              // row stride of W in elements (0: K)
   float* out_f32;                       // TC_STORE: fp32 output [M, ldo] instead of `out`
+  const int32_t* row_seq; int q_stride; // TC_ROPE + PAP over a packed batch: row -> sequence, stride between the q's
+  const int32_t* out_t_col;             // TC_STORE: column of out_t per row (nullptr: the row number)
 };
 spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
 spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,

@@ -160,6 +160,54 @@ def test_dense_layer_across_ffn_row_chunks():
     _run_layer_case("cfg3", 16384 + 300, 16384 + 300, 16384 + 300, 64)
 
 
+@pytest.mark.parametrize("lens", [[256] * 40 + [1, 7, 300, 129], [9000, 500, 128]])
+def test_packed_batch_at_the_8b_layer_shape(lens):
+    """spts_layer_prefill_skip_batch at the 8B layer shape against one call per prompt, bit for bit: 44 short prompts
+    (the route with one launch per step over all prompts: per-sequence probe queries, softmax and TopK in single
+    launches, projections over the packed rows), and a batch with a 9000-token prompt, which is longer than the
+    one-CTA-per-sequence selection takes and sends the whole batch through the per-prompt loop."""
+    from paper_2601_13155_b200 import binding
+    w = synth.workload("cfg2")
+    shape = replace(w.shape, n_layers=1)
+    lw = binding.LayerWeights.from_tensors(synth.device_layer_weights(shape, w.seed, 0, dev()))
+    total = sum(lens)
+    start = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    ma = [max(1, math.ceil(0.5 * n)) for n in lens]
+    mf = [max(1, math.ceil(0.4 * n)) for n in lens]
+    ma[2], mf[1] = lens[2], lens[1]                      # one prompt dense in attention, one dense in the FFN
+    X0, _ = synth.device_hidden_states(w, dev(), n_tokens=total)
+    pos = torch.cat([torch.arange(n, dtype=torch.int32, device=dev()) * 2 + b for b, n in enumerate(lens)])
+    lib = binding.Spts(shape, max_seq=total)
+    lib.set_debug_checks(True)
+    Xs, Ss = X0.clone(), torch.zeros(total, dtype=torch.float32, device=dev())
+    single = binding.KvCache(shape, len(lens), ma)
+    ia_s, jf_s = [], []
+    for b, n in enumerate(lens):
+        s0 = int(start[b])
+        ia = torch.empty(ma[b], dtype=torch.int32, device=dev())
+        jf = torch.empty(mf[b], dtype=torch.int32, device=dev())
+        lib.layer_prefill_skip(lw, Xs[s0:s0 + n], pos[s0:s0 + n], ma[b], mf[b], single, layer=b, S_out=Ss[s0:s0 + n],
+                               idx_attn_out=ia, idx_ffn_out=jf)
+        ia_s.append(ia)
+        jf_s.append(jf)
+    Xb, Sb = X0.clone(), torch.zeros(total, dtype=torch.float32, device=dev())
+    packed = binding.KvCache(shape, len(lens), ma)
+    ia_b = torch.empty(sum(ma), dtype=torch.int32, device=dev())
+    jf_b = torch.empty(sum(mf), dtype=torch.int32, device=dev())
+    lib.layer_prefill_skip_batch(lw, Xb, pos, start, ma, mf, packed, S_out=Sb, idx_attn_out=ia_b, idx_ffn_out=jf_b)
+    assert lib.device_status() == 0 and lib.check_guards() == 0
+    assert torch.equal(ia_b, torch.cat(ia_s)) and torch.equal(jf_b, torch.cat(jf_s))
+    assert torch.equal(Xb, Xs)
+    for b, n in enumerate(lens):
+        s0 = int(start[b])
+        if ma[b] < n or mf[b] < n:
+            assert torch.equal(Sb[s0:s0 + n], Ss[s0:s0 + n])
+        assert packed.length(b) == ma[b]
+        assert torch.equal(packed.k[b][:ma[b]], single.k[b][:ma[b]]) and torch.equal(packed.v[b][:ma[b]], single.v[b][:ma[b]])
+        assert torch.equal(packed.pos[b][:ma[b]], single.pos[b][:ma[b]])
+    lib.close()
+
+
 def test_proxy_build_at_the_8b_layer_shape():
     """spts_proxy_build at the LLaMA-3.1-8B layer shape ((D_low, r) = (512, 128), 14336 channels) on 2048 synthetic
     calibration tokens: importance in full, channel set, singular values and the rank-r products."""

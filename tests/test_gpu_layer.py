@@ -447,14 +447,15 @@ def test_ffn_selection_by_the_attention_score_alone(dtype, ref):
     lib.close()
 
 
-@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", False)])
+@pytest.mark.parametrize("dtype,ref", [("fp32", None), ("bf16", False), ("bf16", True), ("bf16-oddgroup", False),
+                                       ("bf16-group16", False)])
 def test_packed_batch_equals_one_call_per_sequence(dtype, ref):
     """spts_layer_prefill_skip_batch on four ragged prompts (one of them dense in the FFN, one dense in attention, one a
     single token) against spts_layer_prefill_skip on each prompt alone: hidden states, scores, both index lists and the
     caches must agree bit for bit -- the packed FFN GEMMs compute every row exactly as the per-sequence ones do -- and
     the single-sequence call is what the oracle comparisons above cover."""
     from paper_2601_13155_b200 import binding
-    shape = SMALL_BF16 if dtype == "bf16" else synth.TINY
+    shape = {"bf16": SMALL_BF16, "fp32": synth.TINY, "bf16-oddgroup": ODD_GROUP_BF16, "bf16-group16": WIDE_GROUP_BF16}[dtype]
     lens = [300, 1, 517, 130]
     ma = [150, 1, 517, 70]
     mf = [120, 1, 200, 130]
