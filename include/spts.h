@@ -306,9 +306,10 @@ spts_status spts_reduced_attention(spts_ctx* ctx, const void* Q, const void* K, 
  * each sequence's last row), attention is causal within the sequence.  The row normalisation, the K projection
  * (every row probed with its own sequence's last-token query), the per-sequence softmax and TopK, the Q / V / O
  * projections of all selected rows, the proxy FFN of Eq. 12-14 and the selected rows' SwiGLU FFN (Eq. 6) each run once
- * over the packed rows -- gathered GEMMs with ragged index lists -- and only the causal attention itself is launched
- * per sequence (tensor-core mode, up to 1024 sequences of up to 8192 rows each, probe window 1; other batches run the
- * attention blocks one sequence after the other).  Every row gets the bits the single-sequence call gives it.
+ * over the packed rows -- gathered GEMMs with ragged index lists, the attention kernel over a table of all
+ * sequences' query tiles (tensor-core mode, up to 1024 sequences of up to 8192 rows each, probe window 1; other
+ * batches run the attention blocks one sequence after the other).  Every row gets the bits the single-sequence call
+ * gives it.
  * Optional outputs: S_mha_out [total]; idx_attn_out [sum m_attn] and idx_ffn_out [sum m_ffn], sequence after
  * sequence, each numbered from the sequence's own first row. */
 spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos,

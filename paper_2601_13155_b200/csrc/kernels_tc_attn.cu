@@ -42,6 +42,10 @@ struct AttnParams {
   int pair_tiles;   // 0 = the CTA's two tiles are two heads of one KV head, 1 = two query tiles of one head
   bf16* O;          // [m, H*128]
   int* status;
+  // Packed batch (nullptr: one sequence of m rows starting at row 0).  Entry blockIdx.y = (first row of the sequence in
+  // the packed Q / K^ / O buffers, its first column in the packed V^T, its row count, the query tile (or tile pair) of
+  // that sequence this CTA takes); longest tiles first.
+  const int4* tiles;
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -101,7 +105,12 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
   // Tile t of the CTA is (head_t, query tile qt_t).  Even GQA groups: two heads that share a KV head, same query
   // tile (both tiles see the same key blocks).  Otherwise: two consecutive query tiles of one head; tile 0 then has
   // one key block fewer than tile 1 and sits out the last block.
-  const int yy = (int)gridDim.y - 1 - (int)blockIdx.y;        // longest tiles first
+  int yy = (int)gridDim.y - 1 - (int)blockIdx.y;              // longest tiles first
+  int row0 = 0, vcol0 = 0, m_rows = p.m;
+  if (p.tiles != nullptr) {
+    const int4 e = p.tiles[blockIdx.y];
+    row0 = e.x; vcol0 = e.y; m_rows = e.z; yy = e.w;
+  }
   const int h0 = p.pair_tiles ? (int)blockIdx.x : 2 * (int)blockIdx.x;
   const int qt0 = p.pair_tiles ? 2 * yy : yy;
   const int dh = p.pair_tiles ? 0 : 1, dq = p.pair_tiles ? 1 : 0;   // head / query-tile step from tile 0 to tile 1
@@ -138,11 +147,11 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
       mbar_expect_tx(q_full, 3 * TILE_BYTES);               // both Q tiles and K_0 (K_j sits in slot (j + 1) & 1)
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
-        tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE, (qt0 + t * dq) * TILE);
-        tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE + 64, (qt0 + t * dq) * TILE);
+        tma_load_2d(sQ + t * TILE_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE, row0 + (qt0 + t * dq) * TILE);
+        tma_load_2d(sQ + t * TILE_BYTES + SLAB_BYTES, &tmQ, q_full, (h0 + t * dh) * TILE + 64, row0 + (qt0 + t * dq) * TILE);
       }
-      tma_load_2d(sK + TILE_BYTES, &tmK, q_full, kvh * TILE, 0);
-      tma_load_2d(sK + TILE_BYTES + SLAB_BYTES, &tmK, q_full, kvh * TILE + 64, 0);
+      tma_load_2d(sK + TILE_BYTES, &tmK, q_full, kvh * TILE, row0);
+      tma_load_2d(sK + TILE_BYTES + SLAB_BYTES, &tmK, q_full, kvh * TILE + 64, row0);
       bool ok = true;
       for (int j = 0; j < nblk && ok; ++j) {
         const int s = j & 1;
@@ -152,11 +161,11 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
         ok = mbar_wait(kv_free + 8 * s, ((uint32_t)(j >> 1) & 1u) ^ (uint32_t)(s ^ 1), abort_flag, t0);
         if (!ok) break;
         mbar_expect_tx(kv_full + 8 * s, more ? 2 * TILE_BYTES : TILE_BYTES);
-        tma_load_2d(sV + s * TILE_BYTES, &tmV, kv_full + 8 * s, j * TILE, kvh * TILE);
-        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, kv_full + 8 * s, j * TILE + 64, kvh * TILE);
+        tma_load_2d(sV + s * TILE_BYTES, &tmV, kv_full + 8 * s, vcol0 + j * TILE, kvh * TILE);
+        tma_load_2d(sV + s * TILE_BYTES + SLAB_BYTES, &tmV, kv_full + 8 * s, vcol0 + j * TILE + 64, kvh * TILE);
         if (more) {
-          tma_load_2d(sK + s * TILE_BYTES, &tmK, kv_full + 8 * s, kvh * TILE, (j + 1) * TILE);
-          tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, kv_full + 8 * s, kvh * TILE + 64, (j + 1) * TILE);
+          tma_load_2d(sK + s * TILE_BYTES, &tmK, kv_full + 8 * s, kvh * TILE, row0 + (j + 1) * TILE);
+          tma_load_2d(sK + s * TILE_BYTES + SLAB_BYTES, &tmK, kv_full + 8 * s, kvh * TILE + 64, row0 + (j + 1) * TILE);
         }
       }
     }
@@ -313,13 +322,13 @@ tc_attention_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_c
     if (ok) {
       tc_fence_after();
       const float inv = 1.0f / l;
-      bf16* orow = p.O + ((size_t)qi * p.H + head) * TILE;
+      bf16* orow = p.O + ((size_t)(row0 + qi) * p.H + head) * TILE;
 #pragma unroll 1
       for (int c = 0; c < TILE; c += 32) {
         uint32_t r[32];
         tmem_ld32(tOt + c, r);
         tmem_ld_wait();
-        if (qi < p.m) {
+        if (qi < m_rows) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             uint4 w;
@@ -373,6 +382,29 @@ spts_status tc_init(spts_ctx* ctx) {
   return SPTS_OK;
 }
 
+// The same kernel over a packed batch: Q [n_act, H*128], K [n_act, Hkv*128] and O hold the sequences' active rows one
+// after the other, Vt [Hkv*128, ldvt] their transposed values with every sequence starting on a multiple of 8
+// columns; `tiles` (device, n_tiles entries) lists every sequence's query tiles (tile pairs for odd GQA groups).
+spts_status launch_tc_attention_packed(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* Vt, int ldvt, int n_act,
+                                       int vt_cols, const int4* tiles, int n_tiles, bf16* O) {
+  if (n_tiles <= 0) return SPTS_OK;
+  const auto& d = ctx->desc;
+  if (d.head_dim != TILE || ctx->encode_tiled == nullptr) return SPTS_ERR_UNSUPPORTED;
+  if (ldvt % 8) return SPTS_ERR_SHAPE;
+  const int HD = d.n_q_heads * TILE, KD = d.n_kv_heads * TILE;
+  CUtensorMap tmQ, tmK, tmV;
+  if (!make_map(ctx, &tmQ, Q, (uint64_t)n_act, (uint64_t)HD, (uint64_t)HD)) return SPTS_ERR_CUDA;
+  if (!make_map(ctx, &tmK, K, (uint64_t)n_act, (uint64_t)KD, (uint64_t)KD)) return SPTS_ERR_CUDA;
+  if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)vt_cols, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
+  AttnParams p;
+  p.m = 0; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.O = O; p.status = ctx->ws.status; p.tiles = tiles;
+  p.pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 0 : 1;
+  dim3 grid(p.pair_tiles ? d.n_q_heads : d.n_q_heads / 2, n_tiles);
+  tc_attention_pair_kernel<<<grid, AP_THREADS, AP_SMEM, ctx->stream>>>(tmQ, tmK, tmV, p);
+  SPTS_CUDA_OK(ctx);
+  return SPTS_OK;
+}
+
 spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,
                                 int m, bf16* O) {
   (void)V;
@@ -386,7 +418,7 @@ spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, con
   if (!make_map(ctx, &tmK, K, (uint64_t)m, (uint64_t)KD, (uint64_t)KD)) return SPTS_ERR_CUDA;
   if (!make_map(ctx, &tmV, Vt, (uint64_t)KD, (uint64_t)m, (uint64_t)ldvt)) return SPTS_ERR_CUDA;
   AttnParams p;
-  p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.pair_tiles = 0; p.O = O; p.status = ctx->ws.status;
+  p.m = m; p.H = d.n_q_heads; p.Hkv = d.n_kv_heads; p.pair_tiles = 0; p.O = O; p.status = ctx->ws.status; p.tiles = nullptr;
   // two score tiles per CTA: two heads of one KV head when the GQA group is even, else two query tiles of a head
   p.pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 == 0 ? 0 : 1;
   dim3 grid(p.pair_tiles ? d.n_q_heads : d.n_q_heads / 2,

@@ -4,6 +4,7 @@
 #include <new>
 #include <cmath>
 #include <cstring>
+#include <algorithm>
 #include <vector>
 
 #include "spts_common.cuh"
@@ -66,6 +67,7 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   w.batch_ptr = c.take<void*>(3 * (size_t)BATCH_MAX_SEQ);
   w.row_seq = c.take<int32_t>(N);
   w.vt_col = c.take<int32_t>(Npad);
+  w.attn_tiles = c.take<int4>(Npad / 128 + (size_t)BATCH_MAX_SEQ);
   w.rope_cs = c.take<float2>(N * (d.head_dim / 2));
   w.vgu_pad = c.take<char>(2 * (size_t)d.ltp_dlow * 2 * d.ltp_rank * es);
   w.ugu = c.take<char>(2 * (size_t)d.ltp_rank * d.hidden * es);
@@ -427,8 +429,8 @@ spts_status ffn_gemms(spts_ctx* ctx, const spts_layer_weights* w, void* X, int N
 // mode, probe window 1, at most BATCH_MAX_SEQ sequences of at most TOPK_SEG_MAX rows): the row statistics, the
 // rotary table, every sequence's last-token query, the K projection with each row probed by its own sequence's
 // query, the per-sequence softmax of Eq. 4 and TopK of Eq. 5, the Q / V projections of all selected rows and the O
-// projection run once over the packed rows; only the causal attention itself is launched per sequence.  Every row
-// gets the bits the single-sequence call gives it.
+// projection run once over the packed rows, and the causal attention of all sequences is one launch over a table
+// of their query tiles.  Every row gets the bits the single-sequence call gives it.
 spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, void* X, const int32_t* pos, int n_seq,
                                    const int32_t* seq_start, const int32_t* m_attn, uint32_t flags, spts_kv_layer* caches,
                                    float* S, int32_t* idx_attn_out) {
@@ -493,6 +495,9 @@ spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, v
     a.A = (const bf16*)X; a.lda = D; a.a_rows = total; a.idx = ws.idx_a; a.W = (const bf16*)w->wq; a.M = A; a.Nout = HD; a.K = D;
     a.rowscale = ws.rstd; a.out = (bf16*)ws.q_act; a.ldo = HD; a.group = d.n_q_heads / d.n_kv_heads; a.csq_parts = ws.csq_parts;
     OP(SPTS_OP_QVPROJ, 2.0 * Ad * Dd * HD, (Ad * Dd + Ad * HD + Dd * HD) * esd, launch_tc_gemm(ctx, TC_ROPE, a));
+    // a prompt's last key block reaches into the columns after its own: the up to seven pad columns before the next
+    // prompt's start must hold finite values (they meet probabilities that are exactly zero)
+    if (cudaMemsetAsync(ws.v_t, 0, (size_t)KD * ldvt * es, ctx->stream) != cudaSuccess) return SPTS_ERR_CUDA;
     a.W = (const bf16*)w->wv; a.Nout = KD; a.out = (bf16*)ws.o_att; a.ldo = KD;
     a.out_t = (bf16*)ws.v_t; a.ldt = ldvt; a.out_t_col = ws.vt_col;
     OP(SPTS_OP_QVPROJ, 2.0 * Ad * Dd * KD, (Ad * Dd + 2.0 * Ad * KD + Dd * KD) * esd, launch_tc_gemm(ctx, TC_STORE, a));
@@ -500,17 +505,26 @@ spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, v
   OP(SPTS_OP_KV_GATHER, 0.0, 4.0 * Ad * (double)KD * esd + 12.0 * Ad,
      launch_batch_cache_fill(ctx, ws.k_all, ws.o_att, pos, ws.idx_a, d_off, n_seq, A, ws.batch_ptr, ws.batch_ptr + n_seq,
                              (int32_t* const*)(ws.batch_ptr + 2 * n_seq)));
-  // ---- causal attention, one launch per sequence (Algorithm 1: F_MHA on each prompt's own active rows)
+  // ---- causal attention of every prompt among its own active rows (Algorithm 1: F_MHA(Q^, K^, V^)) in one launch:
+  //      K^ packed like Q^ (in the FFN intermediate's buffer, idle during the attention block), a table of the
+  //      prompts' query tiles, longest first
   {
-    double fl = 0.0;
-    for (int b = 0; b < n_seq; ++b) fl += 2.0 * HD * (double)m_attn[b] * (m_attn[b] + 1.0);
-    ProfScope ps(ctx, SPTS_OP_ATTN, fl, (2.0 * Ad * HD + 2.0 * Ad * KD) * esd);
+    const bool pair_tiles = (d.n_q_heads / d.n_kv_heads) % 2 != 0;
+    std::vector<int4> tiles;
     for (int b = 0; b < n_seq; ++b) {
-      TRY(launch_tc_attention(ctx, (const bf16*)ws.q_act + (size_t)h_off[b] * HD, (const bf16*)caches[b].k,
-                              (const bf16*)caches[b].v, (const bf16*)ws.v_t + h_vt0[b], ldvt, m_attn[b],
-                              (bf16*)ws.o_att + (size_t)h_off[b] * HD));
+      const int nqt = ceil_div(m_attn[b], 128), ny = pair_tiles ? ceil_div(nqt, 2) : nqt;
+      for (int y = 0; y < ny; ++y) tiles.push_back(make_int4(h_off[b], h_vt0[b], m_attn[b], y));
       caches[b].len = m_attn[b];
     }
+    std::stable_sort(tiles.begin(), tiles.end(), [](const int4& a, const int4& b) { return a.w > b.w; });
+    if (cudaMemcpyAsync(ws.attn_tiles, tiles.data(), tiles.size() * sizeof(int4), cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
+      return SPTS_ERR_CUDA;
+    OP(SPTS_OP_KV_GATHER, 0.0, 2.0 * Ad * (double)KD * esd, launch_gather_rows(ctx, ws.k_all, ws.idx_a, A, (int)(KD * es), ws.hm));
+    double fl = 0.0;
+    for (int b = 0; b < n_seq; ++b) fl += 2.0 * HD * (double)m_attn[b] * (m_attn[b] + 1.0);
+    OP(SPTS_OP_ATTN, fl, (2.0 * Ad * HD + 2.0 * Ad * KD) * esd,
+       launch_tc_attention_packed(ctx, (const bf16*)ws.q_act, (const bf16*)ws.hm, (const bf16*)ws.v_t, ldvt, A, vt,
+                                  ws.attn_tiles, (int)tiles.size(), (bf16*)ws.o_att));
   }
   {
     TcGemmArgs a;
@@ -819,7 +833,10 @@ spts_status spts_layer_prefill_skip_batch(spts_ctx* ctx, const spts_layer_weight
   float* S = S_mha_out ? S_mha_out : ws.s_mha;
   int max_len = 0;
   for (int b = 0; b < n_seq; ++b) max_len = seq_start[b + 1] - seq_start[b] > max_len ? seq_start[b + 1] - seq_start[b] : max_len;
-  const bool one_launch_per_step = use_tc(ctx) && n_seq <= BATCH_MAX_SEQ && max_len <= TOPK_SEG_MAX && ctx->pap_window < 2;
+  const bool one_launch_per_step = use_tc(ctx) && n_seq <= BATCH_MAX_SEQ && max_len <= TOPK_SEG_MAX && ctx->pap_window < 2 &&
+                                   // K^ is packed in the FFN intermediate's buffer: it has to fit there
+                                   (size_t)total * d.n_kv_heads * d.head_dim <=
+                                       std::min(align_up((size_t)ctx->max_seq, 128), (size_t)FFN_CHUNK_ROWS) * (size_t)d.ffn_dim;
   if (one_launch_per_step) {
     TRY(batch_attention_blocks(ctx, w, X, pos, n_seq, seq_start, m_attn, flags, caches, S, idx_attn_out));
     OP(SPTS_OP_PREP, 0.0, (double)total * (double)row_bytes + 4.0 * total, launch_rstd(ctx, X, total, ws.rstd));

@@ -90,6 +90,7 @@ struct Workspace {
   int32_t* row_seq;     // [Nmax]
   int32_t* vt_col;      // [Nmax]
   int vt_ld_max;        // columns of v_t
+  int4* attn_tiles;     // [Nmax / 128 + BATCH_MAX_SEQ] query tiles of a packed batch's attention launch
 };
 
 }  // namespace spts
@@ -241,6 +242,8 @@ struct TcGemmArgs {
 spts_status launch_tc_gemm(spts_ctx* ctx, int epi, const TcGemmArgs& a);
 spts_status launch_tc_attention(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* V, const bf16* Vt, int ldvt,
                                 int m, bf16* O);
+spts_status launch_tc_attention_packed(spts_ctx* ctx, const bf16* Q, const bf16* K, const bf16* Vt, int ldvt, int n_act,
+                                       int vt_cols, const int4* tiles, int n_tiles, bf16* O);
 spts_status tc_init(spts_ctx* ctx);          // resolves the tensor-map encoder, sets kernel attributes
 int tc_sumsq_parts(int n_out);               // partial sums per row written by TC_SUMSQ
 
