@@ -134,6 +134,9 @@ def main():
     ap.add_argument("report")
     ap.add_argument("extra", nargs="*", help="further metric names to print")
     ap.add_argument("--traffic", nargs="*", default=[], metavar="OP=REGEX[@INDEX]")
+    ap.add_argument("--decode-rows", type=int, default=0, metavar="CACHED_ROWS",
+                    help="the report holds decode kernels against caches of this many rows: record the bytes one layer's "
+                         "weight-streaming kernels move and the bytes per cached row of the attention kernel (op 'decode')")
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--shape", default="")
     ap.add_argument("--command", default="")
@@ -145,6 +148,28 @@ def main():
         print(f"{l['name'][:40]:40s} {l['grid']:>14s} {l['us']:8.1f} {l['read'] / 1e6:9.2f} {l['write'] / 1e6:9.2f} "
               f"{(l['read'] + l['write']) / l['us'] / 1e3:7.0f} {l['dram_pct']:6.1f} {l['tensor_pct']:7.1f} {l['regs']:>4s}"
               + "".join(f" {l['get'](e):>28s}" for e in a.extra))
+    if a.decode_rows:
+        first = next(i for i, l in enumerate(launches) if "dec_qkv_kernel" in l["name"])
+        second = next(i for i, l in enumerate(launches[first + 1:], first + 1) if "dec_qkv_kernel" in l["name"])
+        layer = launches[first:second]
+        attn = sum(l["read"] + l["write"] for l in layer if "dec_attn_mma" in l["name"] or "dec_attn_partial" in l["name"])
+        rest = sum(l["read"] + l["write"] for l in layer) - attn
+        try:
+            commit = subprocess.run(["git", "-C", ROOT, "rev-parse", "--short", "HEAD"], capture_output=True, text=True).stdout.strip()
+        except Exception:
+            commit = ""
+        rec = {"workload": "cfg5", "op": "decode", "kernel": "decode step, one layer", "shape": f"{a.decode_rows} cached rows per layer",
+               "weight_bytes_per_layer": rest, "kv_bytes_per_row": attn / (a.decode_rows + 3.0),
+               "dram_bytes_per_launch": rest + attn, "source_files": OP_SOURCES["decode"], "source_sha256": source_digest("decode"),
+               "commit_at_capture": commit, "command": a.command}
+        data = load_traffic()
+        data["records"] = [r for r in data["records"] if r["op"] != "decode"] + [rec]
+        data["records"].sort(key=lambda r: (r["workload"], r["op"]))
+        with open(TRAFFIC_JSON, "w") as f:
+            json.dump(data, f, indent=1)
+            f.write("\n")
+        print(f"recorded decode: {rest / 1e6:.1f} MB per layer of weight-streaming kernels, {rec['kv_bytes_per_row']:.0f} B per cached row")
+        return
     if not a.traffic:
         return
     try:
