@@ -112,7 +112,7 @@ class ClockSampler:
 # CPU oracle leg (bounded sample)
 # --------------------------------------------------------------------------------------------
 def oracle_sample(w):
-    """The oracle as it stands on BASELINE config 2 in full: one SPTS layer of the 8B shape on an 8192-token prompt
+    """The oracle as it stands on configuration cfg2 in full: one SPTS layer of the 8B shape on an 8192-token prompt
     (attention keep 0.5, FFN keep 0.4), on the host cores.  `w` only supplies the depth the figure is scaled to.
     Returns (tokens/s scaled to that depth, cores, description, measured seconds)."""
     from oracle import spts_oracle as O

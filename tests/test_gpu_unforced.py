@@ -5,9 +5,9 @@ a clipped budget and the trailing segment.
 of the library's own intermediate state is handed to it: the FFN selection T_f is then compared against the
 oracle's own post-attention residual, which the block-wise tests do not do.
 
-* BASELINE config 1 in fp32 verification mode: every output element within 1e-4 of the output RMS, both index sets
+* Configuration cfg1 (the tiny fp32 layer) in fp32 verification mode: every output element within 1e-4 of the output RMS, both index sets
   by the 1e-3 band rule (no one-ulp allowance exists in fp32).
-* BASELINE config 2 (one 8B-shaped bf16 layer, 8192 tokens): the oracle runs the layer in full; the test reports
+* Configuration cfg2 (one 8B-shaped bf16 layer, 8192 tokens): the oracle runs the layer in full; the test reports
   and bounds the T_f symmetric difference (with and without the band) and the one-bf16-ulp disagreements of the
   output, and checks every row on which both sides took the same decisions.
 * A mixed plan in the paper's form (Section 4.1: dense shallow layers, stages with fixed budgets, candidates pruned
@@ -47,7 +47,7 @@ def _unforced_layer(shape, W, X, pos, ma, mf, lw, lib):
 
 
 def test_config1_fp32_layer_unforced():
-    """BASELINE config 1 end to end in fp32 mode: X, S_mha, T_a, T_f and the cache against the oracle's whole layer."""
+    """Configuration cfg1 (the tiny fp32 layer) end to end in fp32 mode: X, S_mha, T_a, T_f and the cache against the oracle's whole layer."""
     from paper_2601_13155_b200 import binding
     w = synth.workload("cfg1")
     shape = w.shape
@@ -74,14 +74,14 @@ def test_config1_fp32_layer_unforced():
     lib.close()
 
 
-# Bounds asserted for the unforced 8B-shaped layer (measured values are printed by the test; the design doc records them).
+# Bounds asserted for the unforced 8B-shaped layer (the measured values are printed by the test).
 CFG2_MAX_TF_DIFF_OUTSIDE_BAND = 8       # tokens of T_f (of 3277) on which GPU and oracle may disagree beyond the band (measured: 0)
 CFG2_MAX_FRACTION_BEYOND_TOL = 1e-3     # elements of the layer output beyond 2e-2 of the RMS (measured: 1.5e-4)
 CFG2_MAX_ERROR = 5e-2                   # largest error relative to the RMS, single rounding steps of large entries aside (measured: 3.9e-2)
 
 
 def test_config2_bf16_layer_unforced_reports_selection_and_flip_counts():
-    """BASELINE config 2 with the oracle run in full from the same input.  T_a must obey the band rule outright.  For
+    """Configuration cfg2 with the oracle run in full from the same input.  T_a must obey the band rule outright.  For
     T_f the oracle's LTP score is computed on the oracle's own post-attention residual: where the library's bf16
     residual differs from it by one ulp in elements of a row, that row's proxy norm moves a little, so tokens next to
     the k-th score can change sides; their number is reported and bounded (measured: 3 tokens of 3277, all inside the
