@@ -276,9 +276,11 @@ def test_decode_steps_at_the_8b_shape():
         assert lib.device_status() == 0
         x, lgo, _ = O.decode_step(emb_host[token], 40000 + step, hostW, shape, oc, np.ones(shape.hidden), lm_host,
                                   mode="bf16")
-        check_output(host(xo), x, "bf16", scale=3)         # the same bounds as the small decode cases
+        check_output(host(xo), x, "bf16", scale=2, what="decode hidden state")   # the same bounds as the small decode cases
         lgh = host(lg)
-        assert rel_rms_err(lgh, lgo) <= 3 * TOL["bf16"]
+        lg_err = rel_rms_err(lgh, lgo)
+        print(f"[parity] decode step {step} at the 8B shape: logits max-abs error {lg_err:.3e} of their RMS")
+        assert lg_err <= 2 * TOL["bf16"]
         assert int(tok.item()) == int(np.argmax(lgh))
         for l, n in enumerate(lens):
             assert cache.length(l) == n + step + 1

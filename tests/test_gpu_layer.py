@@ -216,8 +216,10 @@ def test_prefill_and_decode_match_oracle(dtype, ref):
         lib.decode_step(model, cache2, N + step, token_in=token, x_out=xo, logits_out=lgd, token_out=tok)
         x, lg, tk = O.decode_step(emb[token], N + step, layers, shape, ocaches, np.ones(shape.hidden),
                                   hw["lm_head"], mode=mode)
-        check_output(host(xo), x, dtype, scale=3)
-        assert rel_rms_err(host(lgd), lg) <= 3 * TOL[dtype]
+        check_output(host(xo), x, dtype, scale=2, what="decode hidden state")
+        lg_err = rel_rms_err(host(lgd), lg)
+        print(f"[parity] decode step {step}: logits max-abs error {lg_err:.3e} of their RMS")
+        assert lg_err <= 2 * TOL[dtype]
         assert all(cache2.length(l) == len(ocaches[l]["pos"]) for l in range(L))
         assert int(tok.item()) == int(np.argmax(host(lgd)))
     assert lib.device_status() == 0
