@@ -99,8 +99,11 @@ size_t carve(const spts_model_desc& d, int Nmax, void* base, Workspace* ws, std:
   w.t1 = c.take<char>(Npad * 2 * (size_t)d.ltp_rank * es);
   w.hlow = c.take<char>(Npad * (size_t)d.ltp_dlow * es);
   w.t2 = c.take<char>(Npad * (size_t)d.ltp_rank * es);
+  // The fp32 keys of the plain-kernel K projection live only between that GEMM and the logits kernel behind it, when
+  // the attention output buffer of the block is still unused: they share its storage whenever it is large enough.
   w.acc32_elems = N * KD;
-  w.acc32 = c.take<float>(w.acc32_elems);
+  if (Npad * HD * es >= w.acc32_elems * sizeof(float)) w.acc32 = reinterpret_cast<float*>(w.o_att);
+  else w.acc32 = c.take<float>(w.acc32_elems);
   w.dec = c.take<float>(decode_scratch_floats(d));
   w.logits_v = c.take<float>((size_t)(d.vocab > 0 ? d.vocab : 1));
   w.xrow = c.take<char>((size_t)d.hidden * es);
@@ -514,7 +517,6 @@ spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, v
     for (int b = 0; b < n_seq; ++b) {
       const int nqt = ceil_div(m_attn[b], 128), ny = pair_tiles ? ceil_div(nqt, 2) : nqt;
       for (int y = 0; y < ny; ++y) tiles.push_back(make_int4(h_off[b], h_vt0[b], m_attn[b], y));
-      caches[b].len = m_attn[b];
     }
     std::stable_sort(tiles.begin(), tiles.end(), [](const int4& a, const int4& b) { return a.w > b.w; });
     if (cudaMemcpyAsync(ws.attn_tiles, tiles.data(), tiles.size() * sizeof(int4), cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
@@ -533,6 +535,7 @@ spts_status batch_attention_blocks(spts_ctx* ctx, const spts_layer_weights* w, v
     a.out = (bf16*)X; a.ldo = D; a.csq_parts = ws.csq_parts;
     OP(SPTS_OP_OPROJ, 2.0 * Ad * Dd * HD, (Ad * HD + 2.0 * Ad * Dd + Dd * HD) * esd, launch_tc_gemm(ctx, TC_RESID, a));
   }
+  for (int b = 0; b < n_seq; ++b) caches[b].len = m_attn[b];      // only once everything is enqueued
   return SPTS_OK;
 }
 

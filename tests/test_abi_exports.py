@@ -54,6 +54,41 @@ def test_host_argument_checks_need_no_gpu(lib_path):
     # a call without a context is refused before anything is touched
     assert lib.spts_layer_prefill_skip_batch(None, None, None, None, 2, None, None, None, 0, None, None, None, None) == 1
     assert lib.spts_set_option(None, 16, 1) == 1
+    assert lib.spts_reduced_attention(None, None, None, None, 4, None) == 1
+    assert lib.spts_prepare_layer(None, None, None, 0) == 1
+    assert lib.spts_check_guards(None, None) == 1
+    assert lib.spts_selftest_wait_timeout(None, 1000) == 1
+    assert lib.spts_debug_check_index_list(None, None, 4, 8) == 1
+    assert lib.spts_prepared_bytes(None) == 0
+
+
+def test_workspace_at_the_longest_context_stays_below_four_gigabytes(lib_path):
+    """The SwiGLU intermediate is held for one chunk of 16384 rows, not per candidate: 131072 candidates of the 8B shape
+    need less than 4 GB of workspace, and the prepared proxy factors of a layer a few MB."""
+    from paper_2601_13155_b200 import binding, synth
+    lib = binding.load_library()
+    s = synth.LLAMA8B
+    d = binding.ModelDesc(s.hidden, s.n_q_heads, s.n_kv_heads, s.head_dim, s.ffn_dim, s.ltp_dlow, s.ltp_rank,
+                          s.n_layers, s.vocab, s.rms_eps, s.rope_theta, 0)
+    assert lib.spts_workspace_bytes(ctypes.byref(d), 131072) < 4 * 10 ** 9
+    assert lib.spts_workspace_bytes(ctypes.byref(d), 32768) < 1.5 * 10 ** 9
+    assert 2 * 2 ** 20 < lib.spts_prepared_bytes(ctypes.byref(d)) < 4 * 2 ** 20
+
+
+def test_traffic_records_are_dropped_when_the_kernel_source_changes(tmp_path, monkeypatch):
+    """bench.py reports a captured DRAM-traffic figure only while the SHA-256 of the kernel's source files equals the
+    one stored with the capture."""
+    import json
+    from paper_2601_13155_b200 import ncu_summary
+    rec = {"workload": "cfg3", "op": "attention", "dram_bytes_per_launch": 1.0, "source_sha256": ncu_summary.source_digest("attention")}
+    f = tmp_path / "traffic.json"
+    f.write_text(json.dumps({"records": [rec]}))
+    monkeypatch.setattr(ncu_summary, "TRAFFIC_JSON", str(f))
+    assert ncu_summary.traffic_for("cfg3", "attention")["dram_bytes_per_launch"] == 1.0
+    assert ncu_summary.traffic_for("cfg4", "attention") is None and ncu_summary.traffic_for("cfg3", "topk") is None
+    rec["source_sha256"] = "0" * 64
+    f.write_text(json.dumps({"records": [rec]}))
+    assert ncu_summary.traffic_for("cfg3", "attention") is None
 
 
 def test_product_schedule_matches_budget_rule():
