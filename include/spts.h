@@ -33,8 +33,8 @@
  *     not overlap on the host.  Contexts on different streams are independent (each has its workspace).
  *     spts_layer_prefill_skip() and spts_prefill() use the context's workspace for every intermediate
  *     (K of all candidates, the selected rows' Q, the attention output, the SwiGLU intermediate, scores,
- *     index lists), so the workspace grows with max_seq: about 27 KiB per candidate at the 8B shape plus 0.47 GB for
- *     the SwiGLU intermediate of one 16384-row chunk (3.7 GB at 131072 candidates).
+ *     index lists), so the workspace grows with max_seq: about 24 KiB per candidate at the 8B shape plus 0.5 GB (of
+ *     which 0.47 GB is the SwiGLU intermediate of one 16384-row chunk): 1.30 GB at 32768 candidates, 3.68 GB at 131072.
  */
 #ifndef SPTS_H_
 #define SPTS_H_
