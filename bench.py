@@ -516,6 +516,14 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
 
     ms_e2e, _, _ = timed(plan, steps, from_host=True)
     e2e = N * world / (ms_e2e / steps * 1e-3)
+    # the host-to-device copy on its own (the same pinned buffer, the same stream), to show its share of an e2e step
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(3):
+        X.copy_(X0_host, non_blocking=True)
+    c1.record()
+    torch.cuda.synchronize()
+    h2d_ms = c0.elapsed_time(c1) / 3
 
     dense = None
     if not args.no_dense:
@@ -571,7 +579,7 @@ def prefill_line(args, rep, dev, wname, steps, warmup, dense_warmup, with_cpu):
                        "global_batch": world, "seq_len": N, "parallelism": f"replicas x{world}",
                        "l2": "inputs larger than L2 (14 GB of weights streamed per step)"},
             "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": int(X0_host.numel() * X0_host.element_size()),
-                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / steps},
+                    "d2h_bytes_per_step": 4, "ms_per_step": ms_e2e / steps, "h2d_ms_alone": h2d_ms},
             "gpu_launches": int(launches),
             "clocks": clk,
             "roofline": roof,
